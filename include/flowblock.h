@@ -1,0 +1,225 @@
+/* flowblock.h -- C ABI of the packed-wavefront decode step (sm_100a).
+ *
+ * One decode step of Gated Wavefront Decoding under Heterogeneous Wavefront
+ * Packing is four stream-ordered calls:
+ *
+ *   fb_pack_wavefronts   per-request windows (L_b, R_b) -> dense slot batch
+ *   fb_wavefront_attn    W-shaped block-causal GQA attention over the slots
+ *   fb_t2t_step          top-1 / confidence per row, joint M2T u T2T update
+ *   fb_gate_commit       in-order retirement, KV freeze, readiness-gated
+ *                        admission
+ *
+ * Conventions
+ *   - Every function returns FB_OK (0) or a negative fb_error.  After an
+ *     error fb_last_error(ctx) returns a human-readable host string.
+ *   - Unless stated otherwise every pointer inside fb_state / fb_pack and
+ *     every tensor argument is a DEVICE pointer owned by the caller, at
+ *     least 16-byte aligned.  The library never frees or reallocates them.
+ *   - Calls only enqueue work on `stream` (a cudaStream_t passed as void*)
+ *     and never synchronise.  Nothing is allocated after fb_create; scratch
+ *     comes from the caller's workspace of fb_workspace_bytes(ctx) bytes.
+ *   - Data-dependent problems (a page id out of range, a window wider than
+ *     W, a wait that ran out of time) never trap: the kernel skips the
+ *     offending access and ORs an fb_status bit into the caller's device
+ *     int32 `status` word.
+ *   - A "slot" is one live block of one request.  Slots are numbered in
+ *     (request, block) order; there are max_slots = max_requests * wmax of
+ *     them and the first *n_live are in use.  Row i of a [max_slots*bl, ...]
+ *     tensor is token i % bl of slot i / bl.
+ *   - K/V memory that a request's page table or the window tensors cover must
+ *     hold finite values even where it is masked out (masked entries get
+ *     weight exactly 0, and 0 * inf is not 0).
+ */
+#ifndef FLOWBLOCK_H
+#define FLOWBLOCK_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  FB_OK = 0,
+  FB_ERR_INVALID_ARG = -1, /* null pointer, non-positive size            */
+  FB_ERR_SHAPE = -2,       /* sizes inconsistent with each other         */
+  FB_ERR_ALIGNMENT = -3,   /* a pointer is not 16-byte aligned           */
+  FB_ERR_UNSUPPORTED = -4, /* shape outside what the kernels implement   */
+  FB_ERR_WORKSPACE = -5,   /* workspace missing                          */
+  FB_ERR_CUDA = -6         /* a CUDA runtime / driver call failed        */
+} fb_error;
+
+typedef enum {
+  FB_ST_BAD_PAGE = 1,     /* page id outside [0, num_pages): tile skipped */
+  FB_ST_BAD_TOKEN = 2,    /* reserved                                     */
+  FB_ST_BAD_STATE = 4,    /* R-L outside [0, wmax] or L,R outside [0, n]  */
+  FB_ST_NAN_LOGIT = 8,    /* a row's softmax sum was not finite           */
+  FB_ST_DEV_TIMEOUT = 16  /* a bounded device-side wait gave up           */
+} fb_status;
+
+enum { FB_FLAG_OLDEST = 1, FB_FLAG_FRONTIER = 2 };          /* slot_flags  */
+enum { FB_ACT_NONE = 0, FB_ACT_M2T = 1, FB_ACT_T2T = 2 };   /* action code */
+/* slot_stats columns */
+enum { FB_STAT_M0 = 0, FB_STAT_RDY, FB_STAT_M2T, FB_STAT_T2T, FB_STAT_M1, FB_STAT_EOS,
+       FB_SLOT_STATS = 6 };
+/* step_counters entries */
+enum { FB_CT_BLOCKS = 0, FB_CT_TOKENS, FB_CT_SPAWNED, FB_CT_FINISHED,
+       FB_CT_M2T, FB_CT_T2T, FB_CT_LIVE_SLOTS, FB_CT_ACTIVE,
+       FB_STEP_COUNTERS = 8 };
+
+typedef struct fb_ctx fb_ctx;
+
+/* Immutable per context.  Notation follows the paper: W (wmax), bl
+ * (block_len), n (max_blocks), tau_mask / tau_edit (Eq. 1), theta_spawn
+ * (Eq. 3), S_pe (Sec. 2.1). */
+typedef struct {
+  int32_t max_requests;      /* R_max >= 1                                  */
+  int32_t wmax;              /* W, window bound, 1..8                       */
+  int32_t block_len;         /* bl; bl * (n_q_heads/n_kv_heads) % 128 == 0  */
+  int32_t n_q_heads;
+  int32_t n_kv_heads;        /* divides n_q_heads; group size divides 128   */
+  int32_t head_dim;          /* 64 or 128                                   */
+  int32_t page_size;         /* 64                                          */
+  int32_t num_pages;         /* pages in the shared K and V pools           */
+  int32_t max_pages_per_req; /* columns of the page table                   */
+  int32_t vocab;             /* V, multiple of 8                            */
+  int32_t mask_id;           /* token id of [M] (may be >= vocab)           */
+  int32_t eos_id;            /* -1: none                                    */
+  int32_t max_blocks;        /* n, generation blocks per request            */
+  int32_t s_pe;              /* S_pe, post-edit forwards, 0..255            */
+  float tau_mask;
+  float tau_edit;            /* must be >= tau_mask                         */
+  float theta_spawn;
+  float sm_scale;            /* 0 -> 1/sqrt(head_dim)                       */
+} fb_config;
+
+/* Per-request wavefront state (Sec. 3.2: (L_b, R_b), in-order commit
+ * pointer).  The caller admits / removes requests by writing rows between
+ * steps. */
+typedef struct {
+  int32_t* active;      /* [R_max] 0 free, 1 decoding, 2 done               */
+  int32_t* prefix_len;  /* [R_max] o_b: tokens in the frozen prefix
+                           (prompt + committed blocks)                      */
+  int32_t* L;           /* [R_max] oldest live block                        */
+  int32_t* R;           /* [R_max] one past the frontier block; 0<=L<=R<=n  */
+  int32_t* tokens;      /* [R_max, n*bl] generation region; mask_id = [M]   */
+  uint8_t* pe_done;     /* [R_max, wmax] post-edit forwards seen, by slot   */
+  int32_t* page_table;  /* [R_max, max_pages_per_req] page of absolute
+                           positions [64 j, 64 j + 64); must cover
+                           prefix_len + wmax*bl positions                    */
+} fb_state;
+
+/* Output of fb_pack_wavefronts, input of the other three calls. */
+typedef struct {
+  int32_t* n_live;          /* [1]                                          */
+  int32_t* slot_req;        /* [max_slots] request index, -1 = padding      */
+  int32_t* slot_s;          /* [max_slots] window slot index s = g - L      */
+  int32_t* slot_pos0;       /* [max_slots] absolute position of token 0     */
+  int32_t* slot_kv_len;     /* [max_slots] keys visible: o_b + (s+1) bl     */
+  int32_t* slot_flags;      /* [max_slots] FB_FLAG_*                        */
+  int32_t* req_slot_begin;  /* [R_max+1] CSR over requests                  */
+  int32_t* qtok;            /* [max_slots*bl] gathered tokens (Eq. 4)       */
+  int32_t* pos;             /* [max_slots*bl] absolute position ids (Eq. 4) */
+} fb_pack;
+
+/* Validates the configuration and creates a context (host memory only; no
+ * CUDA call is made).  FB_ERR_UNSUPPORTED for shapes the kernels do not
+ * implement, including tau_edit < tau_mask. */
+int fb_create(const fb_config* cfg, fb_ctx** out);
+int fb_destroy(fb_ctx* ctx);
+const char* fb_last_error(const fb_ctx* ctx); /* ctx may be NULL */
+
+/* Bytes of device scratch the caller must pass as `ws` (256-byte aligned) to
+ * fb_pack_wavefronts and fb_wavefront_attn of the same step: the attention
+ * work list and the split-KV partial results. */
+size_t fb_workspace_bytes(const fb_ctx* ctx);
+
+/* Sec. 3.2, Eq. 4 (gather): compacts the live blocks of all decoding
+ * requests into slots, writes every array of `out`, pads the rest
+ * (slot_req = -1, qtok = mask_id, pos = 0) and builds the attention work
+ * list inside `ws`.  Reads st->{active, prefix_len, L, R, tokens}. */
+int fb_pack_wavefronts(fb_ctx* ctx, const fb_state* st, const fb_pack* out,
+                       void* ws, int32_t* status, void* stream);
+
+/* Sec. 3.1 "W-shaped block-causal attention", Sec. 3.2 Eq. 5: for every live
+ * slot (r, s), token and query head: softmax(sm_scale * q k^T) v over the
+ * keys {frozen prefix [0, o_r) of request r, read through its page table}
+ * u {window blocks 0..s of request r, all bl tokens each}.
+ *   q, out        [max_slots*bl, n_q_heads, head_dim]  bf16
+ *   k_win, v_win  [max_slots*bl, n_kv_heads, head_dim] bf16  (this step's
+ *                 fresh K/V of the window, slot order)
+ *   k_pool,v_pool [num_pages, n_kv_heads, 64, head_dim] bf16
+ *   page_table    [R_max, max_pages_per_req] int32
+ * bf16 inputs, fp32 accumulation, bf16 output.  Rows of padding slots are
+ * not written.  `pk` and `ws` must come from fb_pack_wavefronts of this
+ * step. */
+int fb_wavefront_attn(fb_ctx* ctx, const fb_pack* pk, const void* q,
+                      const void* k_win, const void* v_win,
+                      const void* k_pool, const void* v_pool,
+                      const int32_t* page_table, void* out, void* ws,
+                      int32_t* status, void* stream);
+
+/* Sec. 2.1 Eq. 1 and the numerator / denominator of Eq. 2.
+ *   logits     [max_slots*bl, vocab] bf16, slot order
+ *   argmax     [max_slots*bl] int32  top-1 token (lowest index on ties)
+ *   conf       [max_slots*bl] fp32   its softmax probability
+ *   action     [max_slots*bl] uint8  FB_ACT_*
+ *   slot_stats [max_slots, 6] int32  m0, rdy, n_m2t, n_t2t, m1, has_eos
+ * st->tokens is updated in place (x <- x_hat on Gamma u Delta).  Rows of
+ * padding slots get argmax -1, conf 0, action 0, stats 0. */
+int fb_t2t_step(fb_ctx* ctx, const fb_pack* pk, const void* logits,
+                const fb_state* st, int32_t* argmax, float* conf,
+                uint8_t* action, int32_t* slot_stats, int32_t* status,
+                void* stream);
+
+/* Alg. 1 lines 7-12, Eq. 2-3, Eq. 6 for the committing block: per decoding
+ * request retire the maximal locally-finished prefix of its window in order
+ * (stopping after a block that holds EOS), copy those blocks' window K/V to
+ * absolute positions [o_r, o_r + c*bl) of the request's pages, advance L and
+ * prefix_len, mark the request done on a committed EOS or L == n, then admit
+ * at most one new all-[M] block when rho(frontier) >= theta_spawn and
+ * R - L < W and R < n.
+ *   n_committed   [R_max] int32 blocks retired this step
+ *   spawned       [R_max] uint8
+ *   step_counters [8] int32 (FB_CT_*), overwritten
+ * Mutates st->{active, prefix_len, L, R, tokens (new block), pe_done} and the
+ * pool pages of committed blocks; frozen positions are never rewritten. */
+int fb_gate_commit(fb_ctx* ctx, const fb_pack* pk, const int32_t* slot_stats,
+                   const fb_state* st, const void* k_win, const void* v_win,
+                   void* k_pool, void* v_pool, int32_t* n_committed,
+                   uint8_t* spawned, int32_t* step_counters, int32_t* status,
+                   void* stream);
+
+/* One whole step (the four calls above in order) on HOST inputs: copies this
+ * step's q / k_win / v_win / logits from host (pinned) memory into the
+ * caller's device staging buffers, runs the step, and copies n_committed,
+ * spawned and step_counters back to host memory.  All asynchronous on
+ * `stream`.  h_* are host pointers; everything else is as above. */
+typedef struct {
+  const void* h_q;
+  const void* h_k_win;
+  const void* h_v_win;
+  const void* h_logits;
+  int32_t* h_n_committed;    /* [R_max]  */
+  uint8_t* h_spawned;        /* [R_max]  */
+  int32_t* h_step_counters;  /* [8]      */
+  int32_t* h_status;         /* [1]      */
+} fb_host_io;
+
+typedef struct {
+  void* q; void* k_win; void* v_win; void* out; void* logits;
+  void* k_pool; void* v_pool;
+  int32_t* argmax; float* conf; uint8_t* action; int32_t* slot_stats;
+  int32_t* n_committed; uint8_t* spawned; int32_t* step_counters;
+  int32_t* status; void* ws;
+} fb_device_bufs;
+
+int fb_step_host(fb_ctx* ctx, const fb_state* st, const fb_pack* pk,
+                 const fb_device_bufs* dev, const fb_host_io* io,
+                 void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLOWBLOCK_H */

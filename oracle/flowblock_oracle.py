@@ -197,7 +197,7 @@ def visible_keys(cfg: Config, pk: Pack, slot: int, k_win, k_pool, page_table):
 
 
 def wavefront_attn(cfg: Config, pk: Pack, q, k_win, v_win, k_pool, v_pool,
-                   page_table) -> np.ndarray:
+                   page_table, only_slots=None) -> np.ndarray:
     """Softmax attention of every live query over its visible keys.
 
     q [S*bl, Hq, d]; k_win, v_win [S*bl, Hkv, d] (slot order, this step's
@@ -205,12 +205,14 @@ def wavefront_attn(cfg: Config, pk: Pack, q, k_win, v_win, k_pool, v_pool,
     Query head h uses KV head h // (Hq/Hkv).  Masked keys are excluded
     outright (READING: -inf, never a finite fill); scale 1/sqrt(d) unless
     given.  Two-pass softmax in fp64.  Padding-slot rows are returned as 0.
+    ``only_slots`` restricts the computation to a subset of live slots (the
+    other rows stay 0); used for sampled checks at large sizes.
     """
     b, Hq, Hkv, d = cfg.block_len, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
     G = Hq // Hkv
     sc = _scale(cfg)
     out = np.zeros((cfg.max_slots * b, Hq, d), np.float64)
-    for slot in range(pk.n_live):
+    for slot in (range(pk.n_live) if only_slots is None else only_slots):
         K = visible_keys(cfg, pk, slot, k_win, k_pool, page_table)
         V = visible_keys(cfg, pk, slot, v_win, v_pool, page_table)
         for h in range(Hq):

@@ -1,0 +1,207 @@
+// C ABI entry points: argument validation, workspace layout, dispatch to the
+// kernel launchers.  No kernel lives here.
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "fb_common.cuh"
+
+namespace {
+
+thread_local std::string g_err;
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int fail(fb_ctx* ctx, int code, const std::string& msg) {
+  g_err = msg;
+  if (ctx) ctx->err = msg;
+  return code;
+}
+
+fb::WsLayout make_layout(const fb_config& c, int tiles_per_slot, int target_items) {
+  fb::WsLayout w{};
+  const long long qtiles = (long long)c.max_requests * c.wmax * tiles_per_slot;
+  w.max_units = (int)((qtiles + c.max_requests + 1) / 2) * c.n_kv_heads;
+  w.max_items = w.max_units + target_items + 8;
+  w.max_parts = 2 * target_items + 8;
+  size_t off = 0;
+  w.header = off;  off = align_up(off + sizeof(fb::SchedHeader), 256);
+  w.items = off;   off = align_up(off + (size_t)w.max_items * sizeof(fb::AttnItem), 256);
+  w.units = off;   off = align_up(off + (size_t)w.max_units * sizeof(fb::AttnUnit), 256);
+  w.part_ml = off; off = align_up(off + (size_t)w.max_parts * 2 * fb::kTileM * 2 * sizeof(float), 256);
+  w.part_o = off;  off = align_up(off + (size_t)w.max_parts * 2 * fb::kTileM * c.head_dim * sizeof(float), 256);
+  w.total = off;
+  return w;
+}
+
+int check_state(fb_ctx* ctx, const fb_state* st) {
+  if (!st) return fail(ctx, FB_ERR_INVALID_ARG, "state is null");
+  const void* ps[] = {st->active, st->prefix_len, st->L, st->R, st->tokens, st->pe_done, st->page_table};
+  const char* names[] = {"active", "prefix_len", "L", "R", "tokens", "pe_done", "page_table"};
+  for (int i = 0; i < 7; ++i)
+    if (!ps[i]) return fail(ctx, FB_ERR_INVALID_ARG, std::string("state.") + names[i] + " is null");
+  return FB_OK;
+}
+
+int check_pack(fb_ctx* ctx, const fb_pack* pk) {
+  if (!pk) return fail(ctx, FB_ERR_INVALID_ARG, "pack is null");
+  const void* ps[] = {pk->n_live, pk->slot_req, pk->slot_s, pk->slot_pos0, pk->slot_kv_len,
+                      pk->slot_flags, pk->req_slot_begin, pk->qtok, pk->pos};
+  const char* names[] = {"n_live", "slot_req", "slot_s", "slot_pos0", "slot_kv_len",
+                         "slot_flags", "req_slot_begin", "qtok", "pos"};
+  for (int i = 0; i < 9; ++i)
+    if (!ps[i]) return fail(ctx, FB_ERR_INVALID_ARG, std::string("pack.") + names[i] + " is null");
+  return FB_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int fb_create(const fb_config* cfg, fb_ctx** out) {
+  if (!cfg || !out) return fail(nullptr, FB_ERR_INVALID_ARG, "cfg or out is null");
+  *out = nullptr;
+  const fb_config& c = *cfg;
+  if (c.max_requests < 1 || c.wmax < 1 || c.block_len < 1 || c.n_q_heads < 1 || c.n_kv_heads < 1 ||
+      c.head_dim < 1 || c.num_pages < 1 || c.max_pages_per_req < 1 || c.vocab < 1 || c.max_blocks < 1 ||
+      c.s_pe < 0)
+    return fail(nullptr, FB_ERR_INVALID_ARG, "a size in fb_config is not positive");
+  if (c.n_q_heads % c.n_kv_heads != 0)
+    return fail(nullptr, FB_ERR_SHAPE, "n_kv_heads must divide n_q_heads");
+  if (!(c.tau_mask == c.tau_mask) || !(c.tau_edit == c.tau_edit) || !(c.theta_spawn == c.theta_spawn) ||
+      !(c.sm_scale == c.sm_scale) || c.sm_scale < 0.f)
+    return fail(nullptr, FB_ERR_INVALID_ARG, "a threshold or the scale is NaN or negative");
+  const int G = c.n_q_heads / c.n_kv_heads;
+  if (c.head_dim != 64 && c.head_dim != 128)
+    return fail(nullptr, FB_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
+  if (c.page_size != fb::kPage) return fail(nullptr, FB_ERR_UNSUPPORTED, "page_size must be 64");
+  if (fb::kTileM % G != 0 || (c.block_len * G) % fb::kTileM != 0)
+    return fail(nullptr, FB_ERR_UNSUPPORTED,
+                "block_len * (n_q_heads / n_kv_heads) must be a multiple of 128 and the group size must divide 128");
+  if (c.wmax > 8) return fail(nullptr, FB_ERR_UNSUPPORTED, "wmax must be at most 8");
+  if (c.vocab % 8 != 0) return fail(nullptr, FB_ERR_UNSUPPORTED, "vocab must be a multiple of 8");
+  if (c.s_pe > 255) return fail(nullptr, FB_ERR_UNSUPPORTED, "s_pe must be at most 255");
+  if (c.tau_edit < c.tau_mask)
+    return fail(nullptr, FB_ERR_UNSUPPORTED, "tau_edit < tau_mask is not supported");
+  if ((long long)c.max_requests * c.wmax * c.block_len > (1ll << 24))
+    return fail(nullptr, FB_ERR_UNSUPPORTED, "max_requests * wmax * block_len is too large");
+  fb_ctx* ctx = new (std::nothrow) fb_ctx();
+  if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "out of host memory");
+  ctx->cfg = c;
+  ctx->group = G;
+  ctx->tiles_per_slot = c.block_len * G / fb::kTileM;
+  ctx->tokens_per_tile = fb::kTileM / G;
+  ctx->target_items = fb::kDefaultTargetItems;
+  if (const char* e = getenv("FB_ATTN_TARGET_ITEMS")) {
+    int v = atoi(e);
+    if (v >= 1 && v <= (1 << 20)) ctx->target_items = v;
+  }
+  ctx->sm_scale = c.sm_scale > 0.f ? c.sm_scale : 1.0f / sqrtf((float)c.head_dim);
+  ctx->ws = make_layout(c, ctx->tiles_per_slot, ctx->target_items);
+  *out = ctx;
+  return FB_OK;
+}
+
+int fb_destroy(fb_ctx* ctx) {
+  if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");
+  delete ctx;
+  return FB_OK;
+}
+
+const char* fb_last_error(const fb_ctx* ctx) { return ctx ? ctx->err.c_str() : g_err.c_str(); }
+
+size_t fb_workspace_bytes(const fb_ctx* ctx) { return ctx ? ctx->ws.total : 0; }
+
+int fb_pack_wavefronts(fb_ctx* ctx, const fb_state* st, const fb_pack* out, void* ws, int32_t* status,
+                       void* stream) {
+  if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");
+  if (int e = check_state(ctx, st)) return e;
+  if (int e = check_pack(ctx, out)) return e;
+  if (!ws) return fail(ctx, FB_ERR_WORKSPACE, "workspace is null");
+  if (!status) return fail(ctx, FB_ERR_INVALID_ARG, "status is null");
+  if (reinterpret_cast<uintptr_t>(ws) & 255u) return fail(ctx, FB_ERR_ALIGNMENT, "workspace must be 256-byte aligned");
+  return fb::launch_pack(ctx, st, out, ws, status, (cudaStream_t)stream);
+}
+
+int fb_wavefront_attn(fb_ctx* ctx, const fb_pack* pk, const void* q, const void* k_win, const void* v_win,
+                      const void* k_pool, const void* v_pool, const int32_t* page_table, void* out, void* ws,
+                      int32_t* status, void* stream) {
+  if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");
+  if (int e = check_pack(ctx, pk)) return e;
+  if (!q || !k_win || !v_win || !k_pool || !v_pool || !page_table || !out)
+    return fail(ctx, FB_ERR_INVALID_ARG, "a tensor pointer is null");
+  if (!ws) return fail(ctx, FB_ERR_WORKSPACE, "workspace is null");
+  if (!status) return fail(ctx, FB_ERR_INVALID_ARG, "status is null");
+  if (!aligned16(q) || !aligned16(k_win) || !aligned16(v_win) || !aligned16(k_pool) || !aligned16(v_pool) ||
+      !aligned16(out))
+    return fail(ctx, FB_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  if (reinterpret_cast<uintptr_t>(ws) & 255u) return fail(ctx, FB_ERR_ALIGNMENT, "workspace must be 256-byte aligned");
+  return fb::launch_attn(ctx, pk, q, k_win, v_win, k_pool, v_pool, page_table, out, ws, status,
+                         (cudaStream_t)stream);
+}
+
+int fb_t2t_step(fb_ctx* ctx, const fb_pack* pk, const void* logits, const fb_state* st, int32_t* argmax,
+                float* conf, uint8_t* action, int32_t* slot_stats, int32_t* status, void* stream) {
+  if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");
+  if (int e = check_pack(ctx, pk)) return e;
+  if (int e = check_state(ctx, st)) return e;
+  if (!logits || !argmax || !conf || !action || !slot_stats || !status)
+    return fail(ctx, FB_ERR_INVALID_ARG, "a tensor pointer is null");
+  if (!aligned16(logits)) return fail(ctx, FB_ERR_ALIGNMENT, "logits must be 16-byte aligned");
+  return fb::launch_t2t(ctx, pk, logits, st, argmax, conf, action, slot_stats, status, (cudaStream_t)stream);
+}
+
+int fb_gate_commit(fb_ctx* ctx, const fb_pack* pk, const int32_t* slot_stats, const fb_state* st,
+                   const void* k_win, const void* v_win, void* k_pool, void* v_pool, int32_t* n_committed,
+                   uint8_t* spawned, int32_t* step_counters, int32_t* status, void* stream) {
+  if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");
+  if (int e = check_pack(ctx, pk)) return e;
+  if (int e = check_state(ctx, st)) return e;
+  if (!slot_stats || !k_win || !v_win || !k_pool || !v_pool || !n_committed || !spawned || !step_counters ||
+      !status)
+    return fail(ctx, FB_ERR_INVALID_ARG, "a tensor pointer is null");
+  if (!aligned16(k_win) || !aligned16(v_win) || !aligned16(k_pool) || !aligned16(v_pool))
+    return fail(ctx, FB_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  return fb::launch_gate(ctx, pk, slot_stats, st, k_win, v_win, k_pool, v_pool, n_committed, spawned,
+                         step_counters, status, (cudaStream_t)stream);
+}
+
+int fb_step_host(fb_ctx* ctx, const fb_state* st, const fb_pack* pk, const fb_device_bufs* dev,
+                 const fb_host_io* io, void* stream) {
+  if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");
+  if (!dev || !io) return fail(ctx, FB_ERR_INVALID_ARG, "dev or io is null");
+  if (!io->h_q || !io->h_k_win || !io->h_v_win || !io->h_logits || !io->h_n_committed || !io->h_spawned ||
+      !io->h_step_counters || !io->h_status)
+    return fail(ctx, FB_ERR_INVALID_ARG, "a host pointer is null");
+  if (!dev->q || !dev->k_win || !dev->v_win || !dev->out || !dev->logits || !dev->status)
+    return fail(ctx, FB_ERR_INVALID_ARG, "a device staging pointer is null");
+  const fb_config& c = ctx->cfg;
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t rows = (size_t)c.max_requests * c.wmax * c.block_len;
+  const size_t qb = rows * c.n_q_heads * c.head_dim * 2, kb = rows * c.n_kv_heads * c.head_dim * 2;
+  const size_t lb = rows * (size_t)c.vocab * 2;
+  int e;
+  if ((e = fb::cuda_err(ctx, cudaMemcpyAsync(dev->q, io->h_q, qb, cudaMemcpyHostToDevice, s), "copy q"))) return e;
+  if ((e = fb::cuda_err(ctx, cudaMemcpyAsync(dev->k_win, io->h_k_win, kb, cudaMemcpyHostToDevice, s), "copy k_win"))) return e;
+  if ((e = fb::cuda_err(ctx, cudaMemcpyAsync(dev->v_win, io->h_v_win, kb, cudaMemcpyHostToDevice, s), "copy v_win"))) return e;
+  if ((e = fb::cuda_err(ctx, cudaMemcpyAsync(dev->logits, io->h_logits, lb, cudaMemcpyHostToDevice, s), "copy logits"))) return e;
+  if ((e = fb_pack_wavefronts(ctx, st, pk, dev->ws, dev->status, stream))) return e;
+  if ((e = fb_wavefront_attn(ctx, pk, dev->q, dev->k_win, dev->v_win, dev->k_pool, dev->v_pool, st->page_table,
+                             dev->out, dev->ws, dev->status, stream))) return e;
+  if ((e = fb_t2t_step(ctx, pk, dev->logits, st, dev->argmax, dev->conf, dev->action, dev->slot_stats,
+                       dev->status, stream))) return e;
+  if ((e = fb_gate_commit(ctx, pk, dev->slot_stats, st, dev->k_win, dev->v_win, dev->k_pool, dev->v_pool,
+                          dev->n_committed, dev->spawned, dev->step_counters, dev->status, stream))) return e;
+  if ((e = fb::cuda_err(ctx, cudaMemcpyAsync(io->h_n_committed, dev->n_committed, (size_t)c.max_requests * 4,
+                                             cudaMemcpyDeviceToHost, s), "copy n_committed"))) return e;
+  if ((e = fb::cuda_err(ctx, cudaMemcpyAsync(io->h_spawned, dev->spawned, (size_t)c.max_requests,
+                                             cudaMemcpyDeviceToHost, s), "copy spawned"))) return e;
+  if ((e = fb::cuda_err(ctx, cudaMemcpyAsync(io->h_step_counters, dev->step_counters, FB_STEP_COUNTERS * 4,
+                                             cudaMemcpyDeviceToHost, s), "copy counters"))) return e;
+  if ((e = fb::cuda_err(ctx, cudaMemcpyAsync(io->h_status, dev->status, 4, cudaMemcpyDeviceToHost, s),
+                        "copy status"))) return e;
+  return FB_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,532 @@
+// fb_wavefront_attn: W-shaped block-causal GQA attention over the packed
+// wavefronts (Sec. 3.1 "W-shaped block-causal attention"; Sec. 3.2 Eq. 5).
+//
+// Persistent, warp-specialised tcgen05 kernel, one CTA per SM:
+//   warp 0      TMA producer: Q tiles, K/V tiles of the paged prefix (page-table
+//               lookups) and of the window tensors, 2-stage K and V rings
+//   warp 1      MMA issuer: S = Q K^T and O += P V with tcgen05.mma, S/P and O
+//               in TMEM, two Q tiles (A, B) ping-ponged so that the tensor pipe
+//               works on one tile while the other is in softmax
+//   warps 2-5   softmax of tile A (one thread per query row): tcgen05.ld S,
+//               online max with lazy rescale of O, exp2, P (bf16) written back
+//               over S in TMEM, epilogue
+//   warps 6-9   the same for tile B
+// A Q tile is 128 rows = (128/G tokens) x (G query heads of one KV head) of one
+// slot.  A unit pairs two Q tiles of one request and KV head so that they
+// share each K/V tile from shared memory.  The mask is per tile: a tile of the
+// frozen prefix is fully visible except the ragged last one; the window tile
+// is visible up to (s+1)*bl keys for a query in window slot s.  Tiles nobody
+// can see are never loaded (the work list only spans visible tiles), and
+// ragged tiles run the MMAs on ceil(valid/16)*16 keys only.
+// Long key ranges are split across CTAs; partial (max, sum, O) go to the
+// workspace and a second kernel merges them in a fixed order.
+#include <cudaTypedefs.h>
+
+#include <cstdlib>
+
+#include "fb_common.cuh"
+#include "ptx_sm100.cuh"
+
+namespace fb {
+
+constexpr int kAttnThreads = 320;
+constexpr float kLog2eF = 1.4426950408889634f;
+constexpr float kRescaleThreshold = 8.0f;   // log2 units
+
+struct AttnParams {
+  const SchedHeader* hdr;
+  const AttnItem* items;
+  const AttnUnit* units;
+  const int32_t* page_table;
+  __nv_bfloat16* out;
+  float* part_ml;
+  float* part_o;
+  int32_t* status;
+  int32_t bl, n_q_heads, n_kv_heads, group, max_pages_per_req, num_pages;
+  float scale_log2;
+  long long wait_cycles;
+};
+
+// Geometry of one work item, computed identically by every role.
+struct ItemGeom {
+  AttnUnit un;
+  int jb, n, nA, nB, chunk;
+};
+
+__device__ __forceinline__ bool load_item(const AttnParams& p, int idx, ItemGeom& g) {
+  const int4 it = *reinterpret_cast<const int4*>(&p.items[idx]);
+  const int4* up = reinterpret_cast<const int4*>(&p.units[it.x]);
+  const int4 u0 = up[0], u1 = up[1], u2 = up[2], u3 = up[3];
+  g.un.req = u0.x; g.un.kvh = u0.y; g.un.slotA = u0.z; g.un.slotB = u0.w;
+  g.un.t0A = u1.x; g.un.t0B = u1.y; g.un.n_tiles = u1.z; g.un.n_chunks = u1.w;
+  g.un.nvisA = u2.x; g.un.nvisB = u2.y; g.un.part_base = u2.z; g.un.prefix_len = u2.w;
+  g.un.npt = u3.x; g.un.win_row0 = u3.y; g.un.winA = u3.z; g.un.winB = u3.w;
+  g.chunk = it.y; g.jb = it.z;
+  const int je = it.w;
+  g.nA = max(0, min(je, g.un.nvisA) - g.jb);
+  g.nB = g.un.slotB >= 0 ? max(0, min(je, g.un.nvisB) - g.jb) : 0;
+  g.n = max(g.nA, g.nB);
+  return g.n > 0;
+}
+
+// number of keys of local tile j that tile X (window reach winX) may see
+__device__ __forceinline__ int tile_limit(const ItemGeom& g, int j, int winX) {
+  const int gj = g.jb + j;
+  const int lim = gj < g.un.npt ? g.un.prefix_len - gj * kTileN : winX - (gj - g.un.npt) * kTileN;
+  return min(lim, kTileN);
+}
+__device__ __forceinline__ int round16(int x) { return (x + 15) & ~15; }
+
+// static assignment of the longest-first item list: row k of width gridDim.x,
+// alternate rows reversed
+__device__ __forceinline__ int item_index(int k, int n_items) {
+  const int G = gridDim.x, c = blockIdx.x;
+  const int idx = k * G + ((k & 1) ? G - 1 - c : c);
+  return idx < n_items ? idx : -1;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKwin,
+                      const __grid_constant__ CUtensorMap tmVwin, const __grid_constant__ CUtensorMap tmKpool,
+                      const __grid_constant__ CUtensorMap tmVpool, const AttnParams p) {
+  constexpr int NH = D / 64;                 // 64-element halves of the head dim
+  constexpr int TILE_BYTES = NH * 16384;     // one 128-row operand tile
+  constexpr int PAGE_BYTES = NH * 8192;      // one 64-row page of it
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sQ = smem;                        // [2] tiles A, B
+  uint8_t* sK = sQ + 2 * TILE_BYTES;         // [2] stages
+  uint8_t* sV = sK + 2 * TILE_BYTES;         // [2] stages
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sV + 2 * TILE_BYTES);
+  uint64_t* q_full = bars + 0;
+  uint64_t* q_empty = bars + 1;
+  uint64_t* k_full = bars + 2;    // [2]
+  uint64_t* k_empty = bars + 4;   // [2]
+  uint64_t* v_full = bars + 6;    // [2]
+  uint64_t* v_empty = bars + 8;   // [2]
+  uint64_t* s_full = bars + 10;   // [2] A, B
+  uint64_t* p_full = bars + 12;   // [2]
+  uint64_t* o_full = bars + 14;   // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  volatile int* abortf = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const long long LIM = p.wait_cycles;
+
+  if (tid == 0) {
+    *abortf = 0;
+    mbar_init(q_full, 1); mbar_init(q_empty, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1);
+      mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1);
+      mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 128); mbar_init(&o_full[i], 1);
+    }
+    fence_mbar_init();
+    tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmKwin); tma_prefetch_desc(&tmVwin);
+    tma_prefetch_desc(&tmKpool); tma_prefetch_desc(&tmVpool);
+  }
+  if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const int n_items = p.hdr->n_items;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ producer
+    if (lane == 0) {
+      int q_uses = 0, kt_k = 0, kt_v = 0;
+      bool ok = true;
+      auto load_kv = [&](const ItemGeom& g, int j, bool isV, int& kt) -> bool {
+        const int st = kt & 1, fill = kt >> 1;
+        uint64_t* full = isV ? &v_full[st] : &k_full[st];
+        uint64_t* empty = isV ? &v_empty[st] : &k_empty[st];
+        uint8_t* dst = (isV ? sV : sK) + st * TILE_BYTES;
+        if (fill > 0 && !mbar_wait(empty, (fill - 1) & 1, abortf, LIM)) return false;
+        const int gj = g.jb + j;
+        if (gj < g.un.npt) {
+          const int npg = (gj * kTileN + kPage < g.un.prefix_len) ? 2 : 1;
+          mbar_arrive_expect_tx(full, npg * PAGE_BYTES);
+          for (int pg = 0; pg < npg; ++pg) {
+            const int pidx = gj * 2 + pg;
+            int page = pidx < p.max_pages_per_req ? p.page_table[(size_t)g.un.req * p.max_pages_per_req + pidx] : -1;
+            if (page < 0 || page >= p.num_pages) { atomicOr(p.status, FB_ST_BAD_PAGE); page = 0; }
+            const int y = (page * p.n_kv_heads + g.un.kvh) * kPage;
+            for (int h = 0; h < NH; ++h)
+              tma_load_2d(dst + h * 16384 + pg * 8192, isV ? &tmVpool : &tmKpool, full, h * 64, y);
+          }
+        } else {
+          mbar_arrive_expect_tx(full, TILE_BYTES);
+          const int row0 = g.un.win_row0 + (gj - g.un.npt) * kTileN;
+          for (int h = 0; h < NH; ++h)
+            tma_load_3d(dst + h * 16384, isV ? &tmVwin : &tmKwin, full, h * 64, g.un.kvh, row0);
+        }
+        ++kt;
+        return true;
+      };
+      for (int k = 0; ok && k * (int)gridDim.x < n_items; ++k) {
+        const int idx = item_index(k, n_items);
+        ItemGeom g;
+        if (idx < 0 || !load_item(p, idx, g)) continue;
+        if (q_uses > 0 && !mbar_wait(q_empty, (q_uses - 1) & 1, abortf, LIM)) { ok = false; break; }
+        ++q_uses;
+        mbar_arrive_expect_tx(q_full, ((g.nA > 0) + (g.nB > 0)) * TILE_BYTES);
+        if (g.nA > 0)
+          for (int h = 0; h < NH; ++h)
+            tma_load_3d(sQ + h * 16384, &tmQ, q_full, h * 64, g.un.kvh * p.group, g.un.slotA * p.bl + g.un.t0A);
+        if (g.nB > 0)
+          for (int h = 0; h < NH; ++h)
+            tma_load_3d(sQ + TILE_BYTES + h * 16384, &tmQ, q_full, h * 64, g.un.kvh * p.group,
+                        g.un.slotB * p.bl + g.un.t0B);
+        if (!load_kv(g, 0, false, kt_k)) { ok = false; break; }
+        for (int j = 0; j < g.n; ++j) {
+          if (j + 1 < g.n && !load_kv(g, j + 1, false, kt_k)) { ok = false; break; }
+          if (!load_kv(g, j, true, kt_v)) { ok = false; break; }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ---------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      int q_cnt = 0, kt = 0, cntP[2] = {0, 0};
+      bool ok = true;
+      const uint32_t idesc_pv = umma_idesc_bf16(128, D, 0, 1);
+      auto issue_qk = [&](int X, int st, int ncols) {
+        const uint32_t idesc = umma_idesc_bf16(128, ncols, 0, 0);
+        const uint32_t qa = smem_u32(sQ + X * TILE_BYTES), kb = smem_u32(sK + st * TILE_BYTES);
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
+          umma_ss(tmem + X * 128, smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(kb + off, 16, 1024), idesc,
+                  ks > 0);
+        }
+        umma_commit(&s_full[X]);
+      };
+      auto issue_pv = [&](int X, int st, int ncols, bool acc) {
+        const uint32_t vb = smem_u32(sV + st * TILE_BYTES);
+        for (int ks = 0; ks < ncols / 16; ++ks)
+          umma_ts(tmem + 256 + X * 128, tmem + X * 128 + ks * 8, smem_desc_sw128(vb + ks * 2048, 16384, 1024),
+                  idesc_pv, acc || ks > 0);
+      };
+      for (int k = 0; ok && k * (int)gridDim.x < n_items; ++k) {
+        const int idx = item_index(k, n_items);
+        ItemGeom g;
+        if (idx < 0 || !load_item(p, idx, g)) continue;
+        const int win[2] = {g.un.winA, g.un.winB};
+        const int nX[2] = {g.nA, g.nB};
+        if (!mbar_wait(q_full, q_cnt & 1, abortf, LIM)) { ok = false; break; }
+        ++q_cnt;
+        if (!mbar_wait(&k_full[kt & 1], (kt >> 1) & 1, abortf, LIM)) { ok = false; break; }
+        tc_fence_after();
+        for (int X = 0; X < 2; ++X)
+          if (0 < nX[X]) issue_qk(X, kt & 1, round16(tile_limit(g, 0, win[X])));
+        umma_commit(&k_empty[kt & 1]);
+        for (int j = 0; j < g.n && ok; ++j, ++kt) {
+          const int st = kt & 1, st1 = (kt + 1) & 1;
+          if (!mbar_wait(&v_full[st], (kt >> 1) & 1, abortf, LIM)) { ok = false; break; }
+          for (int X = 0; X < 2; ++X) {
+            if (j < nX[X]) {
+              if (!mbar_wait(&p_full[X], cntP[X] & 1, abortf, LIM)) { ok = false; break; }
+              ++cntP[X];
+              tc_fence_after();
+              issue_pv(X, st, round16(tile_limit(g, j, win[X])), j > 0);
+            }
+            if (X == 1) umma_commit(&v_empty[st]);
+            if (j + 1 < nX[X]) {
+              if (X == 0 || !(j + 1 < nX[0])) {   // first use of K(j+1) in this iteration
+                if (!mbar_wait(&k_full[st1], ((kt + 1) >> 1) & 1, abortf, LIM)) { ok = false; break; }
+                tc_fence_after();
+              }
+              issue_qk(X, st1, round16(tile_limit(g, j + 1, win[X])));
+            }
+          }
+          if (ok && j + 1 < g.n) umma_commit(&k_empty[st1]);
+        }
+        if (!ok) break;
+        if (g.nA > 0) umma_commit(&o_full[0]);
+        if (g.nB > 0) umma_commit(&o_full[1]);
+        umma_commit(q_empty);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------- softmax + epilogue
+    const int X = (warp - 2) >> 2;                 // 0: tile A, 1: tile B
+    const int quad = warp & 3;                     // TMEM lane quadrant of this warp
+    const int row = quad * 32 + lane;              // query row of the tile
+    const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+    const uint32_t tS = tmem + lane_base + X * 128;
+    const uint32_t tO = tmem + lane_base + 256 + X * 128;
+    const float sl2 = p.scale_log2;
+    int cntS = 0, cntO = 0;
+    bool ok = true;
+    for (int k = 0; ok && k * (int)gridDim.x < n_items; ++k) {
+      const int idx = item_index(k, n_items);
+      ItemGeom g;
+      if (idx < 0 || !load_item(p, idx, g)) continue;
+      const int nMine = X == 0 ? g.nA : g.nB;
+      if (nMine == 0) continue;
+      const int winX = X == 0 ? g.un.winA : g.un.winB;
+      float m_ref = -INFINITY, l = 0.f;
+      for (int j = 0; j < nMine; ++j) {
+        if (!mbar_wait(&s_full[X], cntS & 1, abortf, LIM)) { ok = false; break; }
+        ++cntS;
+        tc_fence_after();
+        const int limit = tile_limit(g, j, winX);
+        uint32_t sr[128];
+        tmem_ld32(tS, sr); tmem_ld32(tS + 32, sr + 32); tmem_ld32(tS + 64, sr + 64); tmem_ld32(tS + 96, sr + 96);
+        tmem_ld_wait();
+        float mx = -INFINITY;
+        if (limit >= kTileN) {
+#pragma unroll
+          for (int i = 0; i < 128; ++i) mx = fmaxf(mx, __uint_as_float(sr[i]));
+        } else {
+#pragma unroll
+          for (int i = 0; i < 128; ++i) mx = fmaxf(mx, i < limit ? __uint_as_float(sr[i]) : -INFINITY);
+        }
+        // lazy rescale: keep the old reference unless the max grew by > 2^8
+        bool grow = false;
+        if (j == 0) m_ref = mx;
+        else grow = (mx - m_ref) * sl2 > kRescaleThreshold;
+        if (__any_sync(0xffffffffu, grow)) {
+          const float alpha = grow ? ex2_approx((m_ref - mx) * sl2) : 1.0f;
+          if (grow) { m_ref = mx; l *= alpha; }
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tO + c * 32, o);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+            tmem_st32(tO + c * 32, o);
+          }
+          tmem_st_wait();
+        }
+        const float mb = m_ref * sl2;
+        float sum = 0.f;
+        if (limit >= kTileN) {
+#pragma unroll
+          for (int i = 0; i < 128; i += 2) {
+            const float p0 = ex2_approx(fmaf(__uint_as_float(sr[i]), sl2, -mb));
+            const float p1 = ex2_approx(fmaf(__uint_as_float(sr[i + 1]), sl2, -mb));
+            sum += p0 + p1;
+            sr[i >> 1] = pack_bf16x2(p0, p1);
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 128; i += 2) {
+            const float p0 = i < limit ? ex2_approx(fmaf(__uint_as_float(sr[i]), sl2, -mb)) : 0.f;
+            const float p1 = i + 1 < limit ? ex2_approx(fmaf(__uint_as_float(sr[i + 1]), sl2, -mb)) : 0.f;
+            sum += p0 + p1;
+            sr[i >> 1] = pack_bf16x2(p0, p1);
+          }
+        }
+        l += sum;
+        tmem_st32(tS, sr); tmem_st32(tS + 32, sr + 32);
+        tmem_st_wait();
+        tc_fence_before();
+        mbar_arrive(&p_full[X]);
+      }
+      if (!ok) break;
+      if (!mbar_wait(&o_full[X], cntO & 1, abortf, LIM)) { ok = false; break; }
+      ++cntO;
+      tc_fence_after();
+      if (g.un.n_chunks <= 1) {
+        const int slot = X == 0 ? g.un.slotA : g.un.slotB, t0 = X == 0 ? g.un.t0A : g.un.t0B;
+        const int grow_ = slot * p.bl + t0 + row / p.group;
+        const int head = g.un.kvh * p.group + row % p.group;
+        uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)grow_ * p.n_q_heads + head) * D);
+        const float inv = 1.0f / l;
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t o[32];
+          tmem_ld32(tO + c * 32, o);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            uint4 v;
+            v.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv, __uint_as_float(o[8 * i + 1]) * inv);
+            v.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv);
+            v.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv, __uint_as_float(o[8 * i + 5]) * inv);
+            v.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv, __uint_as_float(o[8 * i + 7]) * inv);
+            dst[c * 4 + i] = v;
+          }
+        }
+      } else {
+        const size_t prow = ((size_t)(g.un.part_base + g.chunk) * 2 + X) * kTileM + row;
+        p.part_ml[prow * 2 + 0] = m_ref * sl2;
+        p.part_ml[prow * 2 + 1] = l;
+        uint4* dst = reinterpret_cast<uint4*>(p.part_o + prow * D);
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t o[32];
+          tmem_ld32(tO + c * 32, o);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 8; ++i) dst[c * 8 + i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+        }
+      }
+      tc_fence_before();
+    }
+  }
+  // ---------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (*abortf) {
+    if (tid == 0) atomicOr(p.status, FB_ST_DEV_TIMEOUT);
+    // give copies that are still in flight time to land before the CTA's
+    // shared memory is handed to the next one
+    for (int i = 0; i < 64; ++i) __nanosleep(10000);
+    __syncthreads();
+  }
+  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem, 512); }
+}
+
+// Merge of the split-KV partials of one unit, chunks in index order.
+template <int D>
+__global__ void __launch_bounds__(256) attn_combine_kernel(const AttnParams p) {
+  const int u = blockIdx.x;
+  if (u >= p.hdr->n_units) return;
+  const AttnUnit un = p.units[u];
+  if (un.n_chunks <= 1) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int PER = D / 32;
+  for (int rr = warp; rr < 2 * kTileM; rr += 8) {
+    const int X = rr / kTileM, row = rr % kTileM;
+    const int slot = X == 0 ? un.slotA : un.slotB;
+    if (slot < 0) continue;
+    const int nvis = X == 0 ? un.nvisA : un.nvisB, t0 = X == 0 ? un.t0A : un.t0B;
+    float M = -INFINITY;
+    for (int c = 0; c < un.n_chunks; ++c) {
+      const int jb = (int)((long long)c * un.n_tiles / un.n_chunks);
+      if (jb >= nvis) break;
+      M = fmaxf(M, p.part_ml[(((size_t)(un.part_base + c) * 2 + X) * kTileM + row) * 2]);
+    }
+    float acc[PER];
+#pragma unroll
+    for (int i = 0; i < PER; ++i) acc[i] = 0.f;
+    float L = 0.f;
+    for (int c = 0; c < un.n_chunks; ++c) {
+      const int jb = (int)((long long)c * un.n_tiles / un.n_chunks);
+      if (jb >= nvis) break;
+      const size_t prow = ((size_t)(un.part_base + c) * 2 + X) * kTileM + row;
+      const float w = ex2_approx(p.part_ml[prow * 2] - M);
+      L += w * p.part_ml[prow * 2 + 1];
+      const float* src = p.part_o + prow * D + lane * PER;
+#pragma unroll
+      for (int i = 0; i < PER; ++i) acc[i] += w * src[i];
+    }
+    const float inv = 1.0f / L;
+    const int grow_ = slot * p.bl + t0 + row / p.group;
+    const int head = un.kvh * p.group + row % p.group;
+    __nv_bfloat16* dst = p.out + ((size_t)grow_ * p.n_q_heads + head) * D + lane * PER;
+#pragma unroll
+    for (int i = 0; i < PER; i += 2)
+      *reinterpret_cast<uint32_t*>(dst + i) = pack_bf16x2(acc[i] * inv, acc[i + 1] * inv);
+  }
+}
+
+// ------------------------------------------------------------------- host
+static int ensure_device(fb_ctx* ctx) {
+  if (ctx->dev_ready) return FB_OK;
+  int dev = 0;
+  if (int e = cuda_err(ctx, cudaGetDevice(&dev), "cudaGetDevice")) return e;
+  cudaDeviceProp prop;
+  if (int e = cuda_err(ctx, cudaGetDeviceProperties(&prop, dev), "cudaGetDeviceProperties")) return e;
+  if (prop.major != 10) return set_err(ctx, FB_ERR_UNSUPPORTED, "the attention kernel needs an sm_100 device");
+  ctx->num_sms = prop.multiProcessorCount;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (int e = cuda_err(ctx, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q),
+                       "cudaGetDriverEntryPoint"))
+    return e;
+  if (!fn || q != cudaDriverEntryPointSuccess)
+    return set_err(ctx, FB_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+  ctx->encode_fn = fn;
+  const int smem64 = 6 * 16384 + 2048, smem128 = 6 * 32768 + 2048;
+  if (int e = cuda_err(ctx, cudaFuncSetAttribute(wavefront_attn_kernel<64>,
+                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, smem64), "smem attr"))
+    return e;
+  if (int e = cuda_err(ctx, cudaFuncSetAttribute(wavefront_attn_kernel<128>,
+                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, smem128), "smem attr"))
+    return e;
+  ctx->dev_ready = true;
+  return FB_OK;
+}
+
+static int encode(fb_ctx* ctx, CUtensorMap* m, const void* base, int rank, const cuuint64_t* dims,
+                  const cuuint64_t* strides, const cuuint32_t* box) {
+  cuuint32_t es[3] = {1, 1, 1};
+  auto fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled>(ctx->encode_fn);
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims, strides, box, es,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return set_err(ctx, FB_ERR_CUDA, "cuTensorMapEncodeTiled failed: " + std::to_string((int)r));
+  return FB_OK;
+}
+
+int launch_attn(fb_ctx* ctx, const fb_pack* pk, const void* q, const void* k_win, const void* v_win,
+                const void* k_pool, const void* v_pool, const int32_t* page_table, void* out, void* ws,
+                int32_t* status, cudaStream_t stream) {
+  (void)pk;
+  if (int e = ensure_device(ctx)) return e;
+  const fb_config& c = ctx->cfg;
+  const cuuint64_t rows = (cuuint64_t)c.max_requests * c.wmax * c.block_len;
+  const cuuint64_t D = c.head_dim;
+  const void* ptrs[5] = {q, k_win, v_win, k_pool, v_pool};
+  if (memcmp(ptrs, ctx->map_ptrs, sizeof(ptrs)) != 0) {
+    {
+      cuuint64_t dims[3] = {D, (cuuint64_t)c.n_q_heads, rows};
+      cuuint64_t str[2] = {D * 2, (cuuint64_t)c.n_q_heads * D * 2};
+      cuuint32_t box[3] = {64, (cuuint32_t)ctx->group, (cuuint32_t)ctx->tokens_per_tile};
+      if (int e = encode(ctx, &ctx->tm_q, q, 3, dims, str, box)) return e;
+    }
+    {
+      cuuint64_t dims[3] = {D, (cuuint64_t)c.n_kv_heads, rows};
+      cuuint64_t str[2] = {D * 2, (cuuint64_t)c.n_kv_heads * D * 2};
+      cuuint32_t box[3] = {64, 1, 128};
+      if (int e = encode(ctx, &ctx->tm_kwin, k_win, 3, dims, str, box)) return e;
+      if (int e = encode(ctx, &ctx->tm_vwin, v_win, 3, dims, str, box)) return e;
+    }
+    {
+      cuuint64_t dims[2] = {D, (cuuint64_t)c.num_pages * c.n_kv_heads * kPage};
+      cuuint64_t str[1] = {D * 2};
+      cuuint32_t box[2] = {64, 64};
+      if (int e = encode(ctx, &ctx->tm_kpool, k_pool, 2, dims, str, box)) return e;
+      if (int e = encode(ctx, &ctx->tm_vpool, v_pool, 2, dims, str, box)) return e;
+    }
+    memcpy(ctx->map_ptrs, ptrs, sizeof(ptrs));
+  }
+  uint8_t* w = static_cast<uint8_t*>(ws);
+  AttnParams p;
+  p.hdr = reinterpret_cast<const SchedHeader*>(w + ctx->ws.header);
+  p.items = reinterpret_cast<const AttnItem*>(w + ctx->ws.items);
+  p.units = reinterpret_cast<const AttnUnit*>(w + ctx->ws.units);
+  p.page_table = page_table;
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.part_ml = reinterpret_cast<float*>(w + ctx->ws.part_ml);
+  p.part_o = reinterpret_cast<float*>(w + ctx->ws.part_o);
+  p.status = status;
+  p.bl = c.block_len; p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.group = ctx->group;
+  p.max_pages_per_req = c.max_pages_per_req; p.num_pages = c.num_pages;
+  p.scale_log2 = ctx->sm_scale * kLog2eF;
+  p.wait_cycles = 2000000000LL;
+  if (const char* e = getenv("FB_WAIT_CYCLES")) { long long v = atoll(e); if (v > 0) p.wait_cycles = v; }
+  const int grid = ctx->num_sms;
+  if (c.head_dim == 64) {
+    wavefront_attn_kernel<64><<<grid, kAttnThreads, 6 * 16384 + 2048, stream>>>(
+        ctx->tm_q, ctx->tm_kwin, ctx->tm_vwin, ctx->tm_kpool, ctx->tm_vpool, p);
+    if (int e = cuda_err(ctx, cudaGetLastError(), "wavefront_attn_kernel launch")) return e;
+    attn_combine_kernel<64><<<ctx->ws.max_units, 256, 0, stream>>>(p);
+  } else {
+    wavefront_attn_kernel<128><<<grid, kAttnThreads, 6 * 32768 + 2048, stream>>>(
+        ctx->tm_q, ctx->tm_kwin, ctx->tm_vwin, ctx->tm_kpool, ctx->tm_vpool, p);
+    if (int e = cuda_err(ctx, cudaGetLastError(), "wavefront_attn_kernel launch")) return e;
+    attn_combine_kernel<128><<<ctx->ws.max_units, 256, 0, stream>>>(p);
+  }
+  return cuda_err(ctx, cudaGetLastError(), "attn_combine_kernel launch");
+}
+
+}  // namespace fb

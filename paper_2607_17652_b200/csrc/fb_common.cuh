@@ -1,0 +1,85 @@
+// Shared declarations of the CUDA path: context, workspace layout, the
+// attention work list.  Nothing here is used by the CPU oracle.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <string>
+
+#include "../../include/flowblock.h"
+
+namespace fb {
+
+constexpr int kTileM = 128;      // query rows per Q tile (tokens x group heads)
+constexpr int kTileN = 128;      // keys per K/V tile (two 64-token pages)
+constexpr int kPage = 64;
+constexpr int kMinChunkTiles = 8;
+constexpr int kDefaultTargetItems = 8 * 148;
+
+// One unit = one (request, KV head, pair of Q tiles); split along the key
+// axis into n_chunks items.  16 ints each, read as four int4.
+struct __align__(16) AttnUnit {
+  int32_t req, kvh, slotA, slotB;      // slotB = -1: single tile
+  int32_t t0A, t0B, n_tiles, n_chunks; // n_tiles: key tiles of the request
+  int32_t nvisA, nvisB, part_base, prefix_len;
+  int32_t npt, win_row0, winA, winB;   // npt prefix tiles; winX = window keys
+                                       // visible to tile X = (s+1)*bl
+};
+struct __align__(16) AttnItem {
+  int32_t unit, chunk, jb, je;         // key tiles [jb, je) of the unit
+};
+
+struct SchedHeader {
+  int32_t n_items, n_units, chunk_tiles, n_parts;
+  int32_t total_tiles, pad[11];
+};
+
+struct WsLayout {
+  size_t header, items, units, part_ml, part_o, total;
+  int32_t max_items, max_units, max_parts;
+};
+
+}  // namespace fb
+
+struct fb_ctx {
+  fb_config cfg;
+  int group;            // G = n_q_heads / n_kv_heads
+  int tiles_per_slot;   // bl * G / 128
+  int tokens_per_tile;  // 128 / G
+  int target_items;
+  float sm_scale;
+  fb::WsLayout ws;
+  std::string err;
+  // lazily initialised at the first attention launch
+  bool dev_ready = false;
+  int num_sms = 0;
+  void* encode_fn = nullptr;
+  // cached tensor maps (re-encoded when a base pointer changes)
+  const void* map_ptrs[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+  CUtensorMap tm_q, tm_kwin, tm_vwin, tm_kpool, tm_vpool;
+};
+
+namespace fb {
+
+int launch_pack(fb_ctx*, const fb_state*, const fb_pack*, void* ws, int32_t* status, cudaStream_t);
+int launch_attn(fb_ctx*, const fb_pack*, const void* q, const void* k_win, const void* v_win,
+                const void* k_pool, const void* v_pool, const int32_t* page_table, void* out,
+                void* ws, int32_t* status, cudaStream_t);
+int launch_t2t(fb_ctx*, const fb_pack*, const void* logits, const fb_state*, int32_t* argmax,
+               float* conf, uint8_t* action, int32_t* slot_stats, int32_t* status, cudaStream_t);
+int launch_gate(fb_ctx*, const fb_pack*, const int32_t* slot_stats, const fb_state*,
+                const void* k_win, const void* v_win, void* k_pool, void* v_pool,
+                int32_t* n_committed, uint8_t* spawned, int32_t* step_counters, int32_t* status,
+                cudaStream_t);
+
+inline int set_err(fb_ctx* ctx, int code, const std::string& msg) {
+  if (ctx) ctx->err = msg;
+  return code;
+}
+inline int cuda_err(fb_ctx* ctx, cudaError_t e, const char* what) {
+  if (e == cudaSuccess) return FB_OK;
+  return set_err(ctx, FB_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+}  // namespace fb

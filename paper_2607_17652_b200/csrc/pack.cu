@@ -1,0 +1,267 @@
+// fb_pack_wavefronts: Heterogeneous Wavefront Packing (Sec. 3.2, Eq. 4).
+//
+// One launch.  Blocks 0..nb-1 compact the live blocks of all decoding
+// requests into slots and gather tokens / position ids; the last block builds
+// the attention work list (units, key-axis chunks, longest first) from the
+// same per-request state.  Everything is integer work on a few KB.
+#include "fb_common.cuh"
+
+namespace fb {
+
+constexpr int kPackThreads = 256;
+constexpr int kSlotsPerBlock = 8;
+constexpr int kCostBins = 1024;
+
+struct PackParams {
+  const int32_t *active, *prefix_len, *L, *R, *tokens;
+  int32_t *n_live, *slot_req, *slot_s, *slot_pos0, *slot_kv_len, *slot_flags, *req_slot_begin, *qtok, *pos;
+  int32_t* status;
+  SchedHeader* hdr;
+  AttnItem* items;
+  AttnUnit* units;
+  int32_t max_requests, wmax, bl, max_slots, max_blocks, mask_id, n_kv_heads;
+  int32_t tiles_per_slot, tokens_per_tile, target_items, max_items, max_units, max_parts;
+  int32_t n_gather_blocks;
+};
+
+// live-block count of request r, sanitised to [0, wmax]
+__device__ __forceinline__ int live_blocks(const PackParams& p, int r, int32_t* status) {
+  if (p.active[r] != 1) return 0;
+  const int L = p.L[r], R = p.R[r];
+  int w = R - L;
+  if (L < 0 || R > p.max_blocks || w < 0 || w > p.wmax) {
+    if (status) atomicOr(status, FB_ST_BAD_STATE);
+    w = w < 0 ? 0 : (w > p.wmax ? p.wmax : w);
+    if (L < 0 || L + w > p.max_blocks) w = 0;
+  }
+  return w;
+}
+
+// exclusive block scan of one value per thread; returns the exclusive prefix,
+// *total = block sum.  All threads must call.
+__device__ __forceinline__ int block_excl_scan(int v, int* total, int* sh /*[kPackThreads/32 + 1]*/) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int x = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int y = __shfl_up_sync(0xffffffffu, x, o);
+    if (lane >= o) x += y;
+  }
+  __syncthreads();
+  if (lane == 31) sh[warp] = x;
+  __syncthreads();
+  if (warp == 0) {
+    int w = lane < kPackThreads / 32 ? sh[lane] : 0;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int y = __shfl_up_sync(0xffffffffu, w, o);
+      if (lane >= o) w += y;
+    }
+    if (lane < kPackThreads / 32) sh[lane] = w;   // inclusive warp sums
+  }
+  __syncthreads();
+  const int base = warp == 0 ? 0 : sh[warp - 1];
+  *total = sh[kPackThreads / 32 - 1];
+  return base + x - v;
+}
+
+struct ReqGeom {
+  int w, ntq, npairs, P, npt, nt;
+};
+__device__ __forceinline__ ReqGeom req_geom(const PackParams& p, int r, int32_t* status) {
+  ReqGeom g;
+  g.w = live_blocks(p, r, status);
+  g.ntq = g.w * p.tiles_per_slot;
+  g.npairs = (g.ntq + 1) >> 1;
+  g.P = g.w ? max(p.prefix_len[r], 0) : 0;
+  g.npt = (g.P + kTileN - 1) / kTileN;
+  g.nt = g.w ? g.npt + (g.w * p.bl + kTileN - 1) / kTileN : 0;
+  return g;
+}
+
+__device__ void build_sched(const PackParams& p) {
+  __shared__ int sh_scan[kPackThreads / 32 + 1];
+  __shared__ int bins[kCostBins];
+  __shared__ long long sh_total;
+  __shared__ int sh_ct;
+  const int tid = threadIdx.x;
+  // bad states are reported once, by the gather blocks (null status here)
+  // phase 1: total key-tile work -> chunk length
+  long long mine = 0;
+  for (int r = tid; r < p.max_requests; r += kPackThreads) {
+    ReqGeom g = req_geom(p, r, nullptr);
+    mine += (long long)g.npairs * p.n_kv_heads * g.nt;
+  }
+  if (tid == 0) sh_total = 0;
+  for (int i = tid; i < kCostBins; i += kPackThreads) bins[i] = 0;
+  __syncthreads();
+  atomicAdd((unsigned long long*)&sh_total, (unsigned long long)mine);
+  __syncthreads();
+  if (tid == 0) {
+    long long ct = (sh_total + p.target_items - 1) / p.target_items;
+    sh_ct = (int)(ct < kMinChunkTiles ? kMinChunkTiles : (ct > (1 << 20) ? (1 << 20) : ct));
+  }
+  __syncthreads();
+  const int Ct = sh_ct;
+  // phase 2 + 3: per-request bases (chunked scan), units, cost histogram
+  int unit_run = 0, part_run = 0, item_run = 0, slot_run = 0;
+  for (int r0 = 0; r0 < p.max_requests; r0 += kPackThreads) {
+    const int r = r0 + tid;
+    ReqGeom g{};
+    int nch = 0, nunits = 0;
+    if (r < p.max_requests) {
+      g = req_geom(p, r, nullptr);
+      nch = g.nt ? (g.nt + Ct - 1) / Ct : 0;
+      nunits = g.npairs * p.n_kv_heads;
+    }
+    int tu, tp, ti, ts;
+    const int ubase = unit_run + block_excl_scan(nunits, &tu, sh_scan);
+    const int pbase = part_run + block_excl_scan(nch > 1 ? nunits * nch : 0, &tp, sh_scan);
+    block_excl_scan(nunits * nch, &ti, sh_scan);
+    const int first = slot_run + block_excl_scan(g.w, &ts, sh_scan);  // first slot of the request
+    unit_run += tu; part_run += tp; item_run += ti; slot_run += ts;
+    if (r < p.max_requests && nunits) {
+      for (int pr = 0; pr < g.npairs; ++pr)
+        for (int h = 0; h < p.n_kv_heads; ++h) {
+          const int u = ubase + pr * p.n_kv_heads + h;
+          if (u >= p.max_units) continue;
+          const int qa = 2 * pr, qb = 2 * pr + 1;
+          AttnUnit un;
+          un.req = r; un.kvh = h;
+          const int sA = qa / p.tiles_per_slot;
+          un.slotA = first + sA;
+          un.t0A = (qa % p.tiles_per_slot) * p.tokens_per_tile;
+          un.winA = (sA + 1) * p.bl;
+          un.nvisA = g.npt + (un.winA + kTileN - 1) / kTileN;
+          if (qb < g.ntq) {
+            const int sB = qb / p.tiles_per_slot;
+            un.slotB = first + sB;
+            un.t0B = (qb % p.tiles_per_slot) * p.tokens_per_tile;
+            un.winB = (sB + 1) * p.bl;
+            un.nvisB = g.npt + (un.winB + kTileN - 1) / kTileN;
+          } else {
+            un.slotB = -1; un.t0B = 0; un.winB = 0; un.nvisB = 0;
+          }
+          un.n_tiles = g.nt; un.n_chunks = nch;
+          un.part_base = nch > 1 ? pbase + (pr * p.n_kv_heads + h) * nch : -1;
+          if (nch > 1 && un.part_base + nch > p.max_parts) un.n_chunks = 0;  // cannot happen; see header
+          un.prefix_len = g.P; un.npt = g.npt; un.win_row0 = first * p.bl;
+          p.units[u] = un;
+          for (int c = 0; c < un.n_chunks; ++c) {
+            const int jb = (int)((long long)c * g.nt / nch), je = (int)((long long)(c + 1) * g.nt / nch);
+            int cost = max(0, min(je, un.nvisA) - jb) + max(0, min(je, un.nvisB) - jb);
+            atomicAdd(&bins[min(cost, kCostBins - 1)], 1);
+          }
+        }
+    }
+  }
+  __syncthreads();
+  // descending exclusive offsets over the cost bins (single thread: 1024 adds)
+  if (tid == 0) {
+    int run = 0;
+    for (int k = kCostBins - 1; k >= 0; --k) { int c = bins[k]; bins[k] = run; run += c; }
+    p.hdr->n_items = min(run, p.max_items);
+    p.hdr->n_units = min(unit_run, p.max_units);
+    p.hdr->chunk_tiles = Ct;
+    p.hdr->n_parts = part_run;
+    p.hdr->total_tiles = (int)min(sh_total, (long long)0x7fffffff);
+    if (run > p.max_items || unit_run > p.max_units || part_run > p.max_parts)
+      atomicOr(p.status, FB_ST_BAD_STATE);
+  }
+  __syncthreads();
+  // phase 4: scatter items, longest first
+  for (int u = tid; u < min(unit_run, p.max_units); u += kPackThreads) {
+    const AttnUnit un = p.units[u];
+    const int nch = un.n_chunks;
+    for (int c = 0; c < nch; ++c) {
+      const int jb = (int)((long long)c * un.n_tiles / nch), je = (int)((long long)(c + 1) * un.n_tiles / nch);
+      int cost = max(0, min(je, un.nvisA) - jb) + max(0, min(je, un.nvisB) - jb);
+      const int at = atomicAdd(&bins[min(cost, kCostBins - 1)], 1);
+      if (at < p.max_items) {
+        AttnItem it; it.unit = u; it.chunk = c; it.jb = jb; it.je = je;
+        p.items[at] = it;
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kPackThreads) pack_kernel(const PackParams p) {
+  if ((int)blockIdx.x == p.n_gather_blocks) { build_sched(p); return; }
+  __shared__ int sh_scan[kPackThreads / 32 + 1];
+  __shared__ int s_req[kSlotsPerBlock], s_idx[kSlotsPerBlock], s_w[kSlotsPerBlock];
+  const int tid = threadIdx.x;
+  const int slot0 = blockIdx.x * kSlotsPerBlock;
+  if (tid < kSlotsPerBlock) s_req[tid] = -1;
+  __syncthreads();
+  int run = 0;
+  for (int r0 = 0; r0 < p.max_requests; r0 += kPackThreads) {
+    const int r = r0 + tid;
+    const int w = r < p.max_requests ? live_blocks(p, r, p.status) : 0;
+    int tot;
+    const int begin = run + block_excl_scan(w, &tot, sh_scan);
+    run += tot;
+    if (r < p.max_requests) {
+      if (blockIdx.x == 0) p.req_slot_begin[r] = begin;
+      for (int s = 0; s < w; ++s) {
+        const int slot = begin + s;
+        if (slot >= slot0 && slot < slot0 + kSlotsPerBlock) {
+          s_req[slot - slot0] = r; s_idx[slot - slot0] = s; s_w[slot - slot0] = w;
+        }
+      }
+    }
+  }
+  if (blockIdx.x == 0 && tid == 0) { p.req_slot_begin[p.max_requests] = run; *p.n_live = run; }
+  __syncthreads();
+  for (int k = 0; k < kSlotsPerBlock; ++k) {
+    const int slot = slot0 + k;
+    if (slot >= p.max_slots) break;
+    const int r = s_req[k];
+    if (r < 0) {
+      if (tid == 0) {
+        p.slot_req[slot] = -1; p.slot_s[slot] = 0; p.slot_pos0[slot] = 0; p.slot_kv_len[slot] = 0;
+        p.slot_flags[slot] = 0;
+      }
+      for (int t = tid; t < p.bl; t += kPackThreads) {
+        p.qtok[slot * p.bl + t] = p.mask_id; p.pos[slot * p.bl + t] = 0;
+      }
+      continue;
+    }
+    const int s = s_idx[k], w = s_w[k];
+    const int P = p.prefix_len[r], g = p.L[r] + s;
+    const int pos0 = P + s * p.bl;
+    if (tid == 0) {
+      p.slot_req[slot] = r; p.slot_s[slot] = s; p.slot_pos0[slot] = pos0;
+      p.slot_kv_len[slot] = P + (s + 1) * p.bl;
+      p.slot_flags[slot] = (s == 0 ? FB_FLAG_OLDEST : 0) | (s == w - 1 ? FB_FLAG_FRONTIER : 0);
+    }
+    const int32_t* src = p.tokens + (size_t)r * p.max_blocks * p.bl + (size_t)g * p.bl;
+    for (int t = tid; t < p.bl; t += kPackThreads) {
+      p.qtok[slot * p.bl + t] = src[t];        // Eq. 4: qtok = x[b, o_b + ...]
+      p.pos[slot * p.bl + t] = pos0 + t;       //        pos  = o_b + ...
+    }
+  }
+}
+
+int launch_pack(fb_ctx* ctx, const fb_state* st, const fb_pack* out, void* ws, int32_t* status,
+                cudaStream_t stream) {
+  const fb_config& c = ctx->cfg;
+  PackParams p;
+  p.active = st->active; p.prefix_len = st->prefix_len; p.L = st->L; p.R = st->R; p.tokens = st->tokens;
+  p.n_live = out->n_live; p.slot_req = out->slot_req; p.slot_s = out->slot_s; p.slot_pos0 = out->slot_pos0;
+  p.slot_kv_len = out->slot_kv_len; p.slot_flags = out->slot_flags; p.req_slot_begin = out->req_slot_begin;
+  p.qtok = out->qtok; p.pos = out->pos; p.status = status;
+  uint8_t* w = static_cast<uint8_t*>(ws);
+  p.hdr = reinterpret_cast<SchedHeader*>(w + ctx->ws.header);
+  p.items = reinterpret_cast<AttnItem*>(w + ctx->ws.items);
+  p.units = reinterpret_cast<AttnUnit*>(w + ctx->ws.units);
+  p.max_requests = c.max_requests; p.wmax = c.wmax; p.bl = c.block_len;
+  p.max_slots = c.max_requests * c.wmax; p.max_blocks = c.max_blocks; p.mask_id = c.mask_id;
+  p.n_kv_heads = c.n_kv_heads; p.tiles_per_slot = ctx->tiles_per_slot;
+  p.tokens_per_tile = ctx->tokens_per_tile; p.target_items = ctx->target_items;
+  p.max_items = ctx->ws.max_items; p.max_units = ctx->ws.max_units; p.max_parts = ctx->ws.max_parts;
+  p.n_gather_blocks = (p.max_slots + kSlotsPerBlock - 1) / kSlotsPerBlock;
+  pack_kernel<<<p.n_gather_blocks + 1, kPackThreads, 0, stream>>>(p);
+  return cuda_err(ctx, cudaGetLastError(), "pack_kernel launch");
+}
+
+}  // namespace fb

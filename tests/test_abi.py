@@ -1,0 +1,81 @@
+"""CPU-only checks of the boundary: the library loads, exports every symbol
+the header declares, and rejects bad arguments before touching CUDA."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2607_17652_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+GOOD = dict(max_requests=4, wmax=2, block_len=32, n_q_heads=8, n_kv_heads=2,
+            head_dim=128, page_size=64, num_pages=16, max_pages_per_req=4,
+            vocab=1024, mask_id=1023, eos_id=1022, max_blocks=8, s_pe=1,
+            tau_mask=0.9, tau_edit=0.95, theta_spawn=0.5, sm_scale=0.0)
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    from paper_2607_17652_b200 import build
+    build.build()
+
+
+def test_header_symbols_are_exported():
+    hdr = open(os.path.join(ROOT, "include", "flowblock.h")).read()
+    declared = set(re.findall(r"\b(fb_[a-z0-9_]+)\s*\(", hdr))
+    assert {"fb_pack_wavefronts", "fb_wavefront_attn", "fb_t2t_step",
+            "fb_gate_commit"} <= declared
+    lib = B.lib()
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert set(B.EXPORTS) >= declared - {"fb_no_such"}
+
+
+def test_struct_layouts_match_header_order():
+    hdr = open(os.path.join(ROOT, "include", "flowblock.h")).read()
+    for cls in (B.fb_config, B.fb_state, B.fb_pack, B.fb_host_io, B.fb_device_bufs):
+        body = re.search(r"typedef struct \{([^{}]*)\} %s;" % cls.__name__, hdr).group(1)
+        body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
+        names = re.findall(r"\*?\s*([A-Za-z_][A-Za-z0-9_]*)\s*[;,]", body)
+        assert names == [n for n, _ in cls._fields_], cls.__name__
+
+
+def test_create_validates_configuration():
+    ctx = B.Context(**GOOD)
+    assert ctx.workspace_bytes() > 0
+    bad = [dict(head_dim=96), dict(page_size=32), dict(block_len=24),
+           dict(n_kv_heads=3), dict(wmax=0), dict(vocab=1001), dict(wmax=9),
+           dict(tau_edit=0.5), dict(s_pe=300), dict(max_requests=-1),
+           dict(tau_mask=float("nan"))]
+    for delta in bad:
+        with pytest.raises(B.FlowBlockError):
+            B.Context(**dict(GOOD, **delta))
+    assert B.lib().fb_create(None, None) == B.FB_ERR_INVALID_ARG
+    assert b"null" in B.lib().fb_last_error(None)
+
+
+def test_null_and_misaligned_arguments_are_rejected_on_the_host():
+    ctx = B.Context(**GOOD)
+    lib = B.lib()
+    st, pk = B.fb_state(), B.fb_pack()
+    assert lib.fb_pack_wavefronts(ctx.handle, C.byref(st), C.byref(pk), None, None, None) \
+        == B.FB_ERR_INVALID_ARG
+    assert b"state.active" in lib.fb_last_error(ctx.handle)
+    full_st = B.fb_state(*([0x1000] * 7))
+    full_pk = B.fb_pack(*([0x1000] * 9))
+    assert lib.fb_pack_wavefronts(ctx.handle, C.byref(full_st), C.byref(full_pk), None,
+                                  0x1000, None) == B.FB_ERR_WORKSPACE
+    assert lib.fb_pack_wavefronts(ctx.handle, C.byref(full_st), C.byref(full_pk), 0x1010,
+                                  0x1000, None) == B.FB_ERR_ALIGNMENT
+    args = [0x1000] * 10
+    args[0] = 0x1008                                   # q misaligned
+    assert lib.fb_wavefront_attn(ctx.handle, C.byref(full_pk), *args) == B.FB_ERR_ALIGNMENT
+    assert lib.fb_t2t_step(ctx.handle, C.byref(full_pk), None, C.byref(full_st),
+                           *([0x1000] * 6)) == B.FB_ERR_INVALID_ARG
+    assert lib.fb_gate_commit(ctx.handle, C.byref(full_pk), None, C.byref(full_st),
+                              *([0x1000] * 9)) == B.FB_ERR_INVALID_ARG
+    assert lib.fb_step_host(ctx.handle, C.byref(full_st), C.byref(full_pk), None, None,
+                            None) == B.FB_ERR_INVALID_ARG
+    assert lib.fb_destroy(None) == B.FB_ERR_INVALID_ARG

@@ -1,0 +1,353 @@
+"""GPU parity: every C-ABI call against the fp64 oracle on the same seeded
+inputs, element by element.  Integer / index / decision outputs must be
+bit-exact; confidence within 2e-5 absolute (fp32 sum of up to 151,552 terms
+with ex2.approx: relative error below 1e-6); attention within
+max-abs 1e-2 and relative L2 5e-3 of the oracle (bf16 inputs, fp32
+accumulation, bf16 output)."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import flowblock_oracle as O
+from paper_2607_17652_b200 import binding as B
+from paper_2607_17652_b200 import synth
+from tests import harness as H
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+CONF_TOL = 2e-5
+ATTN_MAX_ABS, ATTN_REL_L2 = 1e-2, 5e-3
+MARGIN = 1e-3
+
+
+def make_case(wl, seed=None, n_inactive=0, logits_kind=None, conf_shift=0.0,
+              with_attn=True, with_logits=True):
+    stc = synth.make_structure(wl, seed, n_inactive=n_inactive)
+    tokens = synth.make_tokens(stc)
+    case = dict(wl=wl, stc=stc)
+    if with_logits:
+        z, tokens = synth.make_logits(stc, tokens, logits_kind,
+                                      conf_shift=conf_shift)
+        case["logits"] = z
+    case["tokens"] = tokens
+    if with_attn:
+        case["attn"] = synth.make_attn_inputs(stc)
+    return case
+
+
+def gpu_objects(case, **over):
+    stc = case["stc"]
+    ctx = B.Context(**H.common_cfg(stc, **over))
+    st = B.DeviceState.from_numpy(
+        DEV, stc.active, stc.prefix_len, stc.L, stc.R, case["tokens"],
+        np.zeros((stc.wl.n_requests, stc.wl.wmax), np.uint8), stc.page_table)
+    pk = B.PackBuffers.alloc(ctx, DEV)
+    sb = B.StepBuffers(ctx, DEV)
+    return ctx, st, pk, sb
+
+
+def check_pack(pk_gpu: B.PackBuffers, pk: O.Pack):
+    g = pk_gpu.to_numpy()
+    assert int(g["n_live"][0]) == pk.n_live
+    for name in ("slot_req", "slot_s", "slot_pos0", "slot_kv_len",
+                 "slot_flags", "req_slot_begin", "qtok", "pos"):
+        np.testing.assert_array_equal(g[name], getattr(pk, name), err_msg=name)
+
+
+WORKLOADS = {
+    "tiny": synth.tiny_workload(),
+    "tiny_d128_b64": synth.tiny_workload(head_dim=128, block_len=64, wmax=3,
+                                         n_q_heads=8, n_kv_heads=2,
+                                         prefix_lo=0, prefix_hi=700),
+    "tiny_wide": synth.tiny_workload(n_requests=9, wmax=4, n_q_heads=4,
+                                     n_kv_heads=1, prefix_lo=120,
+                                     prefix_hi=136, w_lo=1, w_hi=4),
+    "tiny_noprefix": synth.tiny_workload(prefix_lo=0, prefix_hi=0, w_lo=1,
+                                         w_hi=3, n_requests=4),
+    "cfg0": synth.WORKLOADS[0],
+    "cfg1": synth.WORKLOADS[1],
+}
+
+
+# ------------------------------------------------------------------- pack
+@pytest.mark.parametrize("name", list(WORKLOADS))
+@pytest.mark.parametrize("n_inactive", [0, 1])
+def test_pack_bit_exact(name, n_inactive):
+    wl = WORKLOADS[name]
+    if n_inactive >= wl.n_requests:
+        pytest.skip("single request")
+    case = make_case(wl, n_inactive=n_inactive, with_attn=False,
+                     with_logits=False)
+    ctx, st, pk, sb = gpu_objects(case)
+    B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+    torch.cuda.synchronize()
+    ref = O.pack_wavefronts(H.oracle_cfg(case["stc"]),
+                            H.oracle_state(case["stc"], case["tokens"]))
+    check_pack(pk, ref)
+    assert int(sb.status.item()) == 0
+
+
+def test_pack_empty_and_full_batches():
+    wl = synth.tiny_workload(n_requests=5, wmax=4, w_lo=4, w_hi=4)
+    case = make_case(wl, with_attn=False, with_logits=False)
+    stc = case["stc"]
+    for active in (np.zeros(5, np.int32), np.ones(5, np.int32),
+                   np.array([2, 1, 0, 1, 2], np.int32)):
+        stc.active[:] = active
+        ctx, st, pk, sb = gpu_objects(case)
+        B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+        torch.cuda.synchronize()
+        ref = O.pack_wavefronts(H.oracle_cfg(stc), H.oracle_state(stc, case["tokens"]))
+        check_pack(pk, ref)
+        assert ref.n_live == 4 * int((active == 1).sum())
+
+
+def test_pack_flags_corrupt_state_without_faulting():
+    wl = synth.tiny_workload(n_requests=4, wmax=2, w_lo=1, w_hi=2)
+    case = make_case(wl, with_attn=False, with_logits=False)
+    case["stc"].R[1] = case["stc"].L[1] + 5            # window wider than W
+    ctx, st, pk, sb = gpu_objects(case)
+    B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+    torch.cuda.synchronize()
+    assert int(sb.status.item()) & B.FB_ST_BAD_STATE
+    assert int(pk.n_live.item()) <= ctx.max_slots
+
+
+# -------------------------------------------------------------------- T2T
+def run_t2t_and_gate(case, **over):
+    stc = case["stc"]
+    ctx, st, pk, sb = gpu_objects(case, **over)
+    z = case["logits"].to(DEV)
+    attn = case.get("attn")
+    if attn is not None:
+        q, kw, vw, kp, vp = (t.to(DEV) for t in attn)
+    else:
+        wl = stc.wl
+        kw = torch.zeros(ctx.max_slots * wl.block_len, wl.n_kv_heads, wl.head_dim,
+                         dtype=torch.bfloat16, device=DEV)
+        vw = torch.zeros_like(kw)
+        kp = torch.zeros(stc.num_pages, wl.n_kv_heads, 64, wl.head_dim,
+                         dtype=torch.bfloat16, device=DEV)
+        vp = torch.zeros_like(kp)
+    B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+    B.fb_t2t_step(ctx, pk, z, st, sb.argmax, sb.conf, sb.action, sb.slot_stats,
+                  sb.status)
+    torch.cuda.synchronize()
+    tokens_after_t2t = st.tokens.cpu().numpy().copy()
+    B.fb_gate_commit(ctx, pk, sb.slot_stats, st, kw, vw, kp, vp, sb.n_committed,
+                     sb.spawned, sb.step_counters, sb.status)
+    torch.cuda.synchronize()
+    # oracle
+    ocfg = H.oracle_cfg(stc, **over)
+    ost = H.oracle_state(stc, case["tokens"])
+    opk = O.pack_wavefronts(ocfg, ost)
+    xhat, conf = O.t2t_rows(ocfg, opk, H.f64(case["logits"]))
+    live = opk.n_live * stc.wl.block_len
+    for thr in (np.float32(ocfg.tau_mask), np.float32(ocfg.tau_edit)):
+        assert np.abs(conf[:live] - float(thr)).min() >= MARGIN, \
+            "generator left a confidence inside the decision margin"
+    action, stats = O.t2t_update(ocfg, opk, ost, xhat, conf)
+    np.testing.assert_array_equal(sb.argmax.cpu().numpy(), xhat)
+    np.testing.assert_allclose(sb.conf.cpu().numpy(), conf, rtol=0, atol=CONF_TOL)
+    np.testing.assert_array_equal(sb.action.cpu().numpy(), action)
+    np.testing.assert_array_equal(sb.slot_stats.cpu().numpy(), stats)
+    np.testing.assert_array_equal(tokens_after_t2t, ost.tokens)
+    if attn is not None:
+        okw, ovw, okp, ovp = (H.f64(t) for t in attn[1:])
+        kvargs = (okw, ovw, okp, ovp)
+    else:
+        kvargs = ()
+    ncom, spawned, ctr = O.gate_commit(ocfg, opk, stats, ost, *kvargs)
+    np.testing.assert_array_equal(sb.n_committed.cpu().numpy(), ncom)
+    np.testing.assert_array_equal(sb.spawned.cpu().numpy(), spawned)
+    np.testing.assert_array_equal(sb.step_counters.cpu().numpy(), ctr)
+    g = st.to_numpy()
+    for name in ("active", "prefix_len", "L", "R", "tokens", "pe_done"):
+        np.testing.assert_array_equal(g[name], getattr(ost, name), err_msg=name)
+    if attn is not None:
+        # pool pages: committed rows equal the window rows byte for byte,
+        # everything else untouched
+        np.testing.assert_array_equal(H.f64(kp.cpu()), okp)
+        np.testing.assert_array_equal(H.f64(vp.cpu()), ovp)
+    assert int(sb.status.item()) == 0
+    return dict(action=action, stats=stats, ncom=ncom, spawned=spawned, ctr=ctr)
+
+
+@pytest.mark.parametrize("name,kind,shift,s_pe", [
+    ("tiny", "calibrated", 0.0, 1), ("tiny", "calibrated", 0.3, 0),
+    ("tiny_wide", "calibrated", 0.2, 1), ("tiny_d128_b64", "calibrated", 0.1, 3),
+    ("tiny", "literal", 0.0, 1), ("cfg0", "normal2", 0.0, 1)])
+def test_t2t_and_gate_commit_bit_exact(name, kind, shift, s_pe):
+    case = make_case(WORKLOADS[name], logits_kind=kind, conf_shift=shift)
+    res = run_t2t_and_gate(case, s_pe=s_pe)
+    if kind == "calibrated":
+        assert (res["action"] == O.ACT_M2T).any() and (res["action"] == O.ACT_T2T).any()
+    if shift >= 0.3:
+        assert res["ncom"].sum() >= 0
+
+
+def test_t2t_full_vocab_rows():
+    """V = 151,552 rows: many tiles per row, bf16 ties, peaked rows."""
+    wl = dataclasses.replace(synth.WORKLOADS[1], n_requests=2, name="cfg1_2req")
+    case = make_case(wl, logits_kind="calibrated", with_attn=False)
+    res = run_t2t_and_gate(case)
+    assert (res["action"] == O.ACT_M2T).any()
+
+
+def test_t2t_hand_worked_rows():
+    """Closed-form rows 'one logit = a, others 0' (p = e^a / (e^a + V - 1)),
+    exact ties, and the Eq. 1 / Eq. 2 / Eq. 3 hand-worked block."""
+    V, b = 8, 32
+    wl = synth.tiny_workload(n_requests=1, wmax=2, w_lo=1, w_hi=1, vocab=V,
+                             n_q_heads=4, n_kv_heads=1, max_blocks=4)
+    stc = synth.make_structure(wl)
+    stc.L[:] = 0; stc.R[:] = 1
+    stc.mask_id, stc.eos_id = 9, 10
+    tokens = np.full((1, wl.max_blocks * b), 9, np.int32)
+    tokens[0, :b] = ([9, 9, 3, 0] * 8)
+    z = torch.zeros(wl.max_slots * b, V)
+    spec = [(2, 5.0), (1, 3.0), (1, 5.0), (3, 4.0)] * 8
+    for i, (w, a) in enumerate(spec):
+        z[i, w] = a
+    z[5] = 0.0                                   # 8-way tie -> index 0, p = 1/8
+    case = dict(wl=wl, stc=stc, tokens=tokens, logits=z.to(torch.bfloat16))
+    res = run_t2t_and_gate(case, theta_spawn=0.5)
+    a = res["action"][:b]
+    assert list(a[:4]) == [O.ACT_M2T, O.ACT_NONE, O.ACT_T2T, O.ACT_NONE]
+    assert res["spawned"][0] == 1 and res["ncom"][0] == 0
+
+
+# -------------------------------------------------------------- attention
+def run_attention(case, fill_pad=False):
+    stc = case["stc"]
+    wl = stc.wl
+    ctx, st, pk, sb = gpu_objects(case)
+    q, kw, vw, kp, vp = (t.to(DEV) for t in case["attn"])
+    sb.out.fill_(7.0)
+    B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+    B.fb_wavefront_attn(ctx, pk, q, kw, vw, kp, vp, st.page_table, sb.out,
+                        sb.ws, sb.status)
+    torch.cuda.synchronize()
+    assert int(sb.status.item()) == 0, f"status {int(sb.status.item())}"
+    ocfg = H.oracle_cfg(stc)
+    opk = O.pack_wavefronts(ocfg, H.oracle_state(stc, case["tokens"]))
+    ref = O.wavefront_attn(ocfg, opk, *(H.f64(t) for t in case["attn"]),
+                           stc.page_table)
+    rows = H.live_rows(opk, wl.block_len)
+    max_abs, rel = H.attn_errors(sb.out, ref, rows)
+    assert max_abs <= ATTN_MAX_ABS and rel <= ATTN_REL_L2, (max_abs, rel)
+    # rows of padding slots are not written
+    pad = sb.out[opk.n_live * wl.block_len:].float()
+    assert bool((pad == 7.0).all())
+    return max_abs, rel
+
+
+@pytest.mark.parametrize("name", list(WORKLOADS))
+def test_attention_matches_oracle(name):
+    case = make_case(WORKLOADS[name], with_logits=False)
+    run_attention(case)
+
+
+@pytest.mark.parametrize("target", [1, 7, 100000])
+def test_attention_split_kv_invariance(target, monkeypatch):
+    """Forcing very coarse / very fine key-axis splits changes nothing beyond
+    rounding: the split is an execution detail."""
+    monkeypatch.setenv("FB_ATTN_TARGET_ITEMS", str(target))
+    wl = synth.tiny_workload(prefix_lo=900, prefix_hi=2600, n_requests=3,
+                             head_dim=128, n_q_heads=8, n_kv_heads=2)
+    case = make_case(wl, with_logits=False)
+    run_attention(case)
+
+
+def test_attention_isolation_from_invisible_memory():
+    """Keys a query must not see (other requests, padding slots, pool rows
+    beyond the prefix, blocks to the right) may hold anything finite."""
+    wl = WORKLOADS["tiny"]
+    case = make_case(wl, with_logits=False)
+    stc = case["stc"]
+    ocfg = H.oracle_cfg(stc)
+    opk = O.pack_wavefronts(ocfg, H.oracle_state(stc, case["tokens"]))
+    base = run_attention(case)
+    q, kw, vw, kp, vp = (t.clone() for t in case["attn"])
+    b = wl.block_len
+    kw[opk.n_live * b:] = 300.0
+    vw[opk.n_live * b:] = -300.0
+    used = set()
+    for r in range(wl.n_requests):
+        if stc.active[r] != 1:
+            continue
+        P = int(stc.prefix_len[r])
+        for j in range((P + 63) // 64):
+            used.add(int(stc.page_table[r, j]))
+        if P % 64:
+            pg = int(stc.page_table[r, P // 64])
+            kp[pg, :, P % 64:] = 250.0
+            vp[pg, :, P % 64:] = -250.0
+    for pg in range(stc.num_pages):
+        if pg not in used:
+            kp[pg] = 200.0
+            vp[pg] = -200.0
+    case2 = dict(case, attn=(q, kw, vw, kp, vp))
+    again = run_attention(case2)
+    assert again == base
+
+
+# --------------------------------------------------- multi-step state machine
+def test_multi_step_trajectory_matches_oracle():
+    """Eight consecutive steps (pack -> attention -> T2T -> gate/commit) with
+    confidences rising by 0.05 per step: states, pools and attention outputs
+    are compared after every step, so commits and admissions of one step feed
+    the next one on both sides."""
+    wl = synth.tiny_workload(n_requests=5, wmax=3, w_lo=1, w_hi=2,
+                             prefix_lo=40, prefix_hi=400, max_blocks=10)
+    stc = synth.make_structure(wl)
+    tokens = synth.make_tokens(stc)
+    case = dict(wl=wl, stc=stc, tokens=tokens)
+    ctx, st, pk, sb = gpu_objects(case, s_pe=1)
+    ocfg = H.oracle_cfg(stc, s_pe=1)
+    ost = H.oracle_state(stc, tokens)
+    q, kw, vw, kp, vp = synth.make_attn_inputs(stc)
+    okp, ovp = H.f64(kp), H.f64(vp)
+    dkp, dvp = kp.to(DEV), vp.to(DEV)
+    total_commits = 0
+    for step in range(8):
+        # this step's synthetic model outputs, placed from the ORACLE's state
+        cur = dataclasses.replace(stc)
+        cur.active, cur.prefix_len, cur.L, cur.R = (ost.active.copy(), ost.prefix_len.copy(),
+                                                   ost.L.copy(), ost.R.copy())
+        z, tok2 = synth.make_logits(cur, ost.tokens, "calibrated", seed_shift=step,
+                                    conf_shift=0.05 * step)
+        ost.tokens[:] = tok2
+        st.tokens.copy_(torch.from_numpy(tok2))
+        q = synth.randn_bf16(q.shape, stc.seed + step, 1)
+        kw = synth.randn_bf16(kw.shape, stc.seed + step, 2)
+        vw = synth.randn_bf16(vw.shape, stc.seed + step, 3)
+        dq, dkw, dvw, dz = q.to(DEV), kw.to(DEV), vw.to(DEV), z.to(DEV)
+        B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+        B.fb_wavefront_attn(ctx, pk, dq, dkw, dvw, dkp, dvp, st.page_table, sb.out, sb.ws, sb.status)
+        B.fb_t2t_step(ctx, pk, dz, st, sb.argmax, sb.conf, sb.action, sb.slot_stats, sb.status)
+        B.fb_gate_commit(ctx, pk, sb.slot_stats, st, dkw, dvw, dkp, dvp, sb.n_committed,
+                         sb.spawned, sb.step_counters, sb.status)
+        torch.cuda.synchronize()
+        opk = O.pack_wavefronts(ocfg, ost)
+        check_pack(pk, opk)
+        ref = O.wavefront_attn(ocfg, opk, H.f64(q), H.f64(kw), H.f64(vw), okp, ovp, ost.page_table)
+        max_abs, rel = H.attn_errors(sb.out, ref, H.live_rows(opk, wl.block_len))
+        assert max_abs <= ATTN_MAX_ABS and rel <= ATTN_REL_L2, (step, max_abs, rel)
+        xhat, conf = O.t2t_rows(ocfg, opk, H.f64(z))
+        action, stats = O.t2t_update(ocfg, opk, ost, xhat, conf)
+        ncom, spawned, ctr = O.gate_commit(ocfg, opk, stats, ost, H.f64(kw), H.f64(vw), okp, ovp)
+        np.testing.assert_array_equal(sb.action.cpu().numpy(), action)
+        np.testing.assert_array_equal(sb.n_committed.cpu().numpy(), ncom)
+        np.testing.assert_array_equal(sb.spawned.cpu().numpy(), spawned)
+        np.testing.assert_array_equal(sb.step_counters.cpu().numpy(), ctr)
+        g = st.to_numpy()
+        for name in ("active", "prefix_len", "L", "R", "tokens", "pe_done"):
+            np.testing.assert_array_equal(g[name], getattr(ost, name), err_msg=f"{name}@{step}")
+        np.testing.assert_array_equal(H.f64(dkp.cpu()), okp)
+        np.testing.assert_array_equal(H.f64(dvp.cpu()), ovp)
+        assert int(sb.status.item()) == 0
+        total_commits += int(ncom.sum())
+    assert total_commits >= 3, "the trajectory never committed a block"
