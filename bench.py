@@ -1,0 +1,473 @@
+#!/usr/bin/env python
+"""Benchmark of the packed-wavefront decode step on B200.
+
+A step = fb_pack_wavefronts -> fb_wavefront_attn -> fb_t2t_step ->
+fb_gate_commit over one batch of seeded synthetic input.  Prints ONE JSON line
+(rank 0).  `--impl reference` times the fp64 CPU oracle on a bounded sample
+of the same workload instead.
+
+Units
+  value      whole-step throughput: algorithmic attention FLOPs of one step
+             (4 d sum_live-slots bl Hq kv_len) / device time of the whole step,
+             in TFLOP/s, inputs resident in HBM
+  kernels    per-call device times inside the same timed steps, with the two
+             figures the metric names: attention TFLOP/s and T2T-step GB/s
+  e2e        the same step through fb_step_host: pinned host q / k_win / v_win
+             / logits copied in, decisions copied out, inside the timed region
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "packed-wavefront attn TFLOP/s & T2T-step GB/s (fraction of B200 peak)"
+DEFAULT_WORKLOAD = 2
+KERNELS_PER_STEP = 6   # pack, attention, split-KV combine, T2T rows, T2T update, gate/commit
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures
+# summarised under profiles/ (None until captured for that kernel / workload)
+NCU_TRAFFIC = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"],
+                    bf16_tflops_sustained=d.get("bf16_tflops_sustained"),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0,
+                source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while timing."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id: str):
+        self.gpu_id, self.proc, self.lines = gpu_id, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", self.gpu_id, f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "20"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ts, line in self.lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                c, m = float(f[0]), float(f[1])
+            except ValueError:
+                continue
+            mx = m
+            if t0 - 0.05 <= ts <= t1 + 0.15:
+                sm.append(c)
+                for n, v in zip(names, f[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def attn_flops(stc) -> float:
+    wl = stc.wl
+    tot = 0
+    for r in range(wl.n_requests):
+        if stc.active[r] != 1:
+            continue
+        for s in range(int(stc.R[r] - stc.L[r])):
+            tot += wl.block_len * wl.n_q_heads * (int(stc.prefix_len[r]) + (s + 1) * wl.block_len)
+    return 4.0 * wl.head_dim * tot
+
+
+def attn_bytes(stc) -> float:
+    """K/V read once per request and KV head + Q read + O written."""
+    wl = stc.wl
+    kv = 0
+    rows = 0
+    for r in range(wl.n_requests):
+        if stc.active[r] != 1:
+            continue
+        w = int(stc.R[r] - stc.L[r])
+        kv += int(stc.prefix_len[r]) + w * wl.block_len
+        rows += w * wl.block_len
+    return 2.0 * (2 * kv * wl.n_kv_heads * wl.head_dim + 2 * rows * wl.n_q_heads * wl.head_dim)
+
+
+def t2t_bytes(stc, n_live) -> float:
+    wl = stc.wl
+    rows = n_live * wl.block_len
+    return rows * (2.0 * wl.vocab + 4 + 4 + 1 + 4) + n_live * 24
+
+
+def pick_workload(args):
+    import dataclasses
+    from paper_2607_17652_b200 import synth
+    wl = synth.WORKLOADS[args.workload]
+    if args.requests:
+        wl = dataclasses.replace(wl, n_requests=args.requests, name=f"{wl.name}[{args.requests} requests]")
+    return wl
+
+
+def build_inputs(wl, seed):
+    from paper_2607_17652_b200 import synth
+    stc = synth.make_structure(wl, seed)
+    tokens = synth.make_tokens(stc)
+    n_live = synth.n_live_slots(stc)
+    z, tokens = synth.make_logits(stc, tokens, n_rows=n_live * wl.block_len)
+    attn = synth.make_attn_inputs(stc)
+    return stc, tokens, n_live, z, attn
+
+
+# ---------------------------------------------------------------- our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2607_17652_b200 import binding as B, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    wl = pick_workload(args)
+    seed = synth.BASE_SEED + wl.index + 1000 * rank     # each rank its own batch
+    stc, tokens, n_live, z_live, attn = build_inputs(wl, seed)
+    stc_init = stc
+    ctx = B.Context(**synth.config_dict(stc))
+    st = B.DeviceState.from_numpy(dev, stc.active, stc.prefix_len, stc.L, stc.R, tokens,
+                                  np.zeros((wl.n_requests, wl.wmax), np.uint8), stc.page_table)
+    pk = B.PackBuffers.alloc(ctx, dev)
+    sb = B.StepBuffers(ctx, dev)
+    rows = ctx.max_slots * wl.block_len
+    logits = torch.zeros(rows, wl.vocab, dtype=torch.bfloat16, device=dev)
+    logits[:z_live.shape[0]].copy_(z_live)
+    q, kw, vw, kp, vp = (t.to(dev) for t in attn)
+    stream = torch.cuda.current_stream()
+
+    only = args.only
+
+    def step(ev=None):
+        if ev: ev[0].record(stream)
+        if only == "all" or ev is None:
+            B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status, stream)
+        if ev: ev[1].record(stream)
+        if only in ("all", "attn"):
+            B.fb_wavefront_attn(ctx, pk, q, kw, vw, kp, vp, st.page_table, sb.out, sb.ws, sb.status, stream)
+        if ev: ev[2].record(stream)
+        if only in ("all", "t2t"):
+            B.fb_t2t_step(ctx, pk, logits, st, sb.argmax, sb.conf, sb.action, sb.slot_stats, sb.status, stream)
+        if ev: ev[3].record(stream)
+        if only == "all":
+            B.fb_gate_commit(ctx, pk, sb.slot_stats, st, kw, vw, kp, vp, sb.n_committed, sb.spawned,
+                             sb.step_counters, sb.status, stream)
+        if ev: ev[4].record(stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def device_structure():
+        """The workload structure as it stands on the device (commits and
+        admissions of earlier steps move L, R and the prefix lengths)."""
+        import dataclasses
+        g = st.to_numpy()
+        cur = dataclasses.replace(stc)
+        cur.active, cur.prefix_len, cur.L, cur.R = g["active"], g["prefix_len"], g["L"], g["R"]
+        return cur
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    stc0 = device_structure()
+    uuid = str(torch.cuda.get_device_properties(local).uuid)
+    sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+    sampler.start()
+    time.sleep(0.2)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    barrier()
+    t0 = time.time()
+    for k in range(args.steps):
+        step(evs[k])
+    barrier()
+    t1 = time.time()
+    total_ms = evs[0][0].elapsed_time(evs[-1][4])
+    seg = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(4)] for e in evs])  # ms
+    status = int(sb.status.item())
+    counters = sb.step_counters.cpu().numpy().tolist()
+    stc1 = device_structure()
+
+    # ------------------------------------------------------------ end to end
+    e2e_ms, h2d, d2h = float("nan"), 0, 0
+    if not args.no_e2e and only == "all":
+        pin = lambda t: t.cpu().contiguous().pin_memory()
+        hq, hkw, hvw = pin(q), pin(kw), pin(vw)
+        hz = torch.zeros(rows, wl.vocab, dtype=torch.bfloat16).pin_memory()
+        hz[:z_live.shape[0]].copy_(z_live)
+        host = dict(h_q=hq, h_k_win=hkw, h_v_win=hvw, h_logits=hz,
+                    h_n_committed=torch.zeros(wl.n_requests, dtype=torch.int32).pin_memory(),
+                    h_spawned=torch.zeros(wl.n_requests, dtype=torch.uint8).pin_memory(),
+                    h_step_counters=torch.zeros(8, dtype=torch.int32).pin_memory(),
+                    h_status=torch.zeros(1, dtype=torch.int32).pin_memory())
+        devb = dict(q=q, k_win=kw, v_win=vw, out=sb.out, logits=logits, k_pool=kp, v_pool=vp,
+                    argmax=sb.argmax, conf=sb.conf, action=sb.action, slot_stats=sb.slot_stats,
+                    n_committed=sb.n_committed, spawned=sb.spawned, step_counters=sb.step_counters,
+                    status=sb.status, ws=sb.ws)
+        e2e_steps = max(3, min(args.steps, 5))
+        for _ in range(2):
+            B.fb_step_host(ctx, st, pk, devb, host, stream)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(e2e_steps):
+            B.fb_step_host(ctx, st, pk, devb, host, stream)
+            stream.synchronize()          # the caller reads the step's decisions
+        e1.record(stream)
+        barrier()
+        e2e_ms = e0.elapsed_time(e1) / e2e_steps
+        h2d = sum(t.numel() * t.element_size() for t in (hq, hkw, hvw, hz))
+        d2h = wl.n_requests * 4 + wl.n_requests + 8 * 4 + 4
+    t2 = time.time()
+    clocks = sampler.stop(t0, t2)
+    clocks["window"] = "timed steps + end-to-end steps"
+
+    # algorithmic work of the state the timed steps ran on (mean of the state
+    # before and after, equal once the literal-logit workload has settled)
+    n_live = (synth.n_live_slots(stc0) + synth.n_live_slots(stc1)) / 2.0
+    flops_state = (attn_flops(stc0) + attn_flops(stc1)) / 2.0
+    abytes_state = (attn_bytes(stc0) + attn_bytes(stc1)) / 2.0
+    stc = stc0
+    flops = flops_state
+    ms_step = total_ms / args.steps
+    tms = torch.tensor([ms_step, e2e_ms], dtype=torch.float64, device=dev)
+    fl = torch.tensor([flops, t2t_bytes(stc, n_live)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
+        dist.all_reduce(fl, op=dist.ReduceOp.SUM)
+    ms_step_max, e2e_ms_max = (float(x) for x in tms.cpu())
+    flops_all, t2tb_all = (float(x) for x in fl.cpu())
+
+    if rank == 0:
+        peaks = load_peaks()
+        attn_ms, t2t_ms = float(seg[:, 1].mean()), float(seg[:, 2].mean())
+        attn_tf = flops / attn_ms / 1e9
+        t2t_gbs = t2t_bytes(stc, n_live) / t2t_ms / 1e6
+        roof_attn = {"kernel": "wavefront_attn_kernel(+combine)", "bound": "tensor",
+                     "achieved": round(attn_tf, 2), "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                     "frac": round(attn_tf / peaks["bf16_tflops"], 4),
+                     "traffic": NCU_TRAFFIC.get(("attn", args.workload)),
+                     "peak_source": peaks["source"] + " cuBLAS bf16 burst",
+                     "hbm_floor_ms": round(abytes_state / peaks["hbm_gbs"] / 1e6, 4),
+                     "tensor_floor_ms": round(flops / peaks["bf16_tflops"] / 1e9, 4),
+                     "ms": round(attn_ms, 4)}
+        roof_t2t = {"kernel": "t2t_rows_kernel(+update)", "bound": "hbm", "achieved": round(t2t_gbs, 1),
+                    "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(t2t_gbs / peaks["hbm_gbs"], 4),
+                    "traffic": NCU_TRAFFIC.get(("t2t", args.workload)),
+                    "peak_source": peaks["source"] + " copy bandwidth", "ms": round(t2t_ms, 4)}
+        dominant = roof_attn if attn_ms >= t2t_ms else roof_t2t
+        line = {
+            "metric": METRIC, "value": round(flops_all / ms_step_max / 1e9, 3),
+            "unit": "TFLOP/s (attention FLOPs / whole-step time)",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": round(ms_step_max, 4), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "requests": wl.n_requests, "block_len": wl.block_len,
+                       "wmax": wl.wmax, "slots": ctx.max_slots, "live_slots": n_live, "state_settled": bool(synth.n_live_slots(stc0) == synth.n_live_slots(stc1)),
+                       "q_heads": wl.n_q_heads, "kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim,
+                       "vocab": wl.vocab, "prefix_range": [wl.prefix_lo, wl.prefix_hi],
+                       "logits": wl.logits_kind, "parallelism": f"replicas x{world}",
+                       "l2": "inputs larger than L2 (logits + KV pools >> 126 MB); no flush"},
+            "clocks": clocks,
+            "e2e": {"value": round(flops_all / e2e_ms_max / 1e9, 3),
+                    "unit": "TFLOP/s (attention FLOPs / whole-step time, host buffers)",
+                    "ms_per_step": round(e2e_ms_max, 3), "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h,
+                    "t2t_gbs": round(t2tb_all / e2e_ms_max / 1e6, 2)},
+            "gpu_launches": KERNELS_PER_STEP * args.steps,
+            "kernels": {"pack_ms": round(float(seg[:, 0].mean()), 4), "attn_ms": round(attn_ms, 4),
+                        "t2t_ms": round(t2t_ms, 4), "gate_commit_ms": round(float(seg[:, 3].mean()), 4),
+                        "attn_tflops": round(attn_tf, 2), "t2t_gbs": round(t2t_gbs, 1),
+                        "attn_frac_of_nominal_2250": round(attn_tf / 2250.0, 4),
+                        "t2t_frac_of_nominal_8000": round(t2t_gbs / 8000.0, 4)},
+            "roofline": {k: dominant[k] for k in ("bound", "achieved", "peak", "unit", "frac", "traffic")}
+                        | {"kernel": dominant["kernel"], "peak_source": dominant["peak_source"]},
+            "roofline_attn": roof_attn, "roofline_t2t": roof_t2t,
+            "device_status": status, "step_counters": counters,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(wl, stc_init, tokens, z_live, attn, budget_s=args.cpu_budget)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------- the oracle, timed
+def oracle_sample_step(wl, stc, tokens, z_live, attn, n_req):
+    """One oracle step (pack, attention, T2T, gate/commit) on the first n_req
+    decoding requests of the workload.  Returns (seconds, attention flops,
+    slots, rows)."""
+    import dataclasses
+    from oracle import flowblock_oracle as O
+    from tests import harness as H
+    import torch
+    sub = dataclasses.replace(stc)
+    act = stc.active.copy()
+    keep = np.flatnonzero(act == 1)[:n_req]
+    act[:] = 0
+    act[keep] = 1
+    sub.active = act
+    # compact pool holding only the pages of the kept requests (input layout
+    # only: the oracle still reads every key through a page table)
+    need = (stc.prefix_len + wl.wmax * wl.block_len + wl.page_size - 1) // wl.page_size
+    pages = np.concatenate([stc.page_table[r, :need[r]] for r in keep]) if len(keep) else np.zeros(1, np.int32)
+    remap = {int(pg): i for i, pg in enumerate(pages)}
+    pt = np.zeros_like(stc.page_table)
+    for r in keep:
+        pt[r, :need[r]] = [remap[int(pg)] for pg in stc.page_table[r, :need[r]]]
+    sub.page_table, sub.num_pages = pt, len(pages)
+    ocfg = H.oracle_cfg(sub)
+    ost = H.oracle_state(sub, tokens)
+    full_pk = O.pack_wavefronts(H.oracle_cfg(stc), H.oracle_state(stc, tokens))
+    b = wl.block_len
+    rows = np.concatenate([np.arange(full_pk.req_slot_begin[r] * b, full_pk.req_slot_begin[r + 1] * b)
+                           for r in keep]) if len(keep) else np.zeros(0, np.int64)
+    trows = torch.from_numpy(rows.astype(np.int64))
+    q, kw, vw, kp, vp = attn
+    pad = ocfg.max_slots * b - len(rows)
+    def take(t):
+        x = H.f64(t[trows])
+        return np.concatenate([x, np.zeros((pad,) + x.shape[1:])], axis=0)
+    fq, fkw, fvw = take(q), take(kw), take(vw)
+    fz = H.f64(z_live[trows])
+    fz = np.concatenate([fz, np.zeros((pad, wl.vocab))], axis=0) if pad else fz
+    tp = torch.from_numpy(pages.astype(np.int64))
+    fkp, fvp = H.f64(kp[tp]), H.f64(vp[tp])
+    t0 = time.perf_counter()
+    opk = O.pack_wavefronts(ocfg, ost)
+    O.wavefront_attn(ocfg, opk, fq, fkw, fvw, fkp, fvp, ost.page_table)
+    xhat, conf = O.t2t_rows(ocfg, opk, fz)
+    action, stats = O.t2t_update(ocfg, opk, ost, xhat, conf)
+    O.gate_commit(ocfg, opk, stats, ost, fkw, fvw, fkp, fvp)
+    dt = time.perf_counter() - t0
+    return dt, attn_flops(sub), opk.n_live, opk.n_live * b
+
+
+def cpu_baseline(wl, stc, tokens, z_live, attn, budget_s=12.0):
+    n_req, used = 1, None
+    total = int((stc.active == 1).sum())
+    while True:
+        dt, fl, slots, rows = oracle_sample_step(wl, stc, tokens, z_live, attn, n_req)
+        used = (dt, fl, slots, rows, n_req)
+        if dt >= budget_s or n_req >= total:
+            break
+        n_req = min(total, max(n_req + 1, int(n_req * min(4.0, budget_s / max(dt, 1e-3)))))
+    dt, fl, slots, rows, n_req = used
+    try:
+        import threadpoolctl
+        threads = max([p["num_threads"] for p in threadpoolctl.threadpool_info()] or [1])
+    except Exception:
+        threads = os.cpu_count()
+    return {"value": round(fl / dt / 1e12, 6), "unit": "TFLOP/s (attention FLOPs / whole-step time)",
+            "cores": threads, "host_cores": os.cpu_count(), "kind": "oracle", "seconds": round(dt, 2),
+            "sample": f"first {n_req} of {total} requests of {wl.name}: {slots} slots, {rows} rows x V={wl.vocab}"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2607_17652_b200 import synth
+    wl = pick_workload(args)
+    stc, tokens, n_live, z_live, attn = build_inputs(wl, synth.BASE_SEED + wl.index)
+    n_req = args.ref_requests
+    times, fl = [], 0.0
+    for k in range(args.warmup + args.steps):
+        dt, fl, slots, rows = oracle_sample_step(wl, stc, tokens, z_live, attn, n_req)
+        if k >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    val = round(fl / (ms / 1e3) / 1e12, 6)
+    unit = "TFLOP/s (attention FLOPs / whole-step time)"
+    try:
+        import threadpoolctl
+        threads = max([p["num_threads"] for p in threadpoolctl.threadpool_info()] or [1])
+    except Exception:
+        threads = os.cpu_count()
+    total = int((stc.active == 1).sum())
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": unit,
+            "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": round(ms, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "requests": wl.n_requests, "block_len": wl.block_len,
+                       "wmax": wl.wmax, "vocab": wl.vocab},
+            "cpu_baseline": {"value": val, "unit": unit, "kind": "oracle", "cores": threads,
+                             "host_cores": os.cpu_count(),
+                             "sample": f"each step: first {n_req} of {total} requests of {wl.name}: "
+                                       f"{slots} slots, {rows} rows x V={wl.vocab}"},
+            "e2e": {"value": val, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=DEFAULT_WORKLOAD)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--requests", type=int, default=0,
+                    help="override the workload's request count (small cases for profiler captures)")
+    ap.add_argument("--only", default="all", choices=["all", "attn", "t2t"],
+                    help="time one call only (profiler captures); the JSON line then has no step metric")
+    ap.add_argument("--cpu-budget", type=float, default=12.0)
+    ap.add_argument("--ref-requests", type=int, default=2)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

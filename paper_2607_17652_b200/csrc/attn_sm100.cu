@@ -7,10 +7,12 @@
 //   warp 1      MMA issuer: S = Q K^T and O += P V with tcgen05.mma, S/P and O
 //               in TMEM, two Q tiles (A, B) ping-ponged so that the tensor pipe
 //               works on one tile while the other is in softmax
-//   warps 2-5   softmax of tile A (one thread per query row): tcgen05.ld S,
+//   warps 2-3   idle (they complete the control warpgroup, which gives its
+//               registers to the softmax warpgroups with setmaxnreg)
+//   warps 4-7   softmax of tile A (one thread per query row): tcgen05.ld S,
 //               online max with lazy rescale of O, exp2, P (bf16) written back
 //               over S in TMEM, epilogue
-//   warps 6-9   the same for tile B
+//   warps 8-11  the same for tile B
 // A Q tile is 128 rows = (128/G tokens) x (G query heads of one KV head) of one
 // slot.  A unit pairs two Q tiles of one request and KV head so that they
 // share each K/V tile from shared memory.  The mask is per tile: a tile of the
@@ -29,7 +31,7 @@
 
 namespace fb {
 
-constexpr int kAttnThreads = 320;
+constexpr int kAttnThreads = 384;   // 3 warpgroups: control, softmax A, softmax B
 constexpr float kLog2eF = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
 
@@ -133,8 +135,11 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   const uint32_t tmem = *tmem_slot;
   const int n_items = p.hdr->n_items;
 
+  // The control warpgroup (warps 0-3) hands registers to the two softmax
+  // warpgroups; each role's code follows its own setmaxnreg.
   if (warp == 0) {
     // ------------------------------------------------------------ producer
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (lane == 0) {
       int q_uses = 0, kt_k = 0, kt_v = 0;
       bool ok = true;
@@ -150,7 +155,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           mbar_arrive_expect_tx(full, npg * PAGE_BYTES);
           for (int pg = 0; pg < npg; ++pg) {
             const int pidx = gj * 2 + pg;
-            int page = pidx < p.max_pages_per_req ? p.page_table[(size_t)g.un.req * p.max_pages_per_req + pidx] : -1;
+            int page = pidx < p.max_pages_per_req ? __ldg(&p.page_table[(size_t)g.un.req * p.max_pages_per_req + pidx]) : -1;
             if (page < 0 || page >= p.num_pages) { atomicOr(p.status, FB_ST_BAD_PAGE); page = 0; }
             const int y = (page * p.n_kv_heads + g.un.kvh) * kPage;
             for (int h = 0; h < NH; ++h)
@@ -189,13 +194,16 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     __syncwarp();
   } else if (warp == 1) {
     // ---------------------------------------------------------- MMA issuer
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (lane == 0) {
-      int q_cnt = 0, kt = 0, cntP[2] = {0, 0};
+      int q_cnt = 0, kt = 0, cntPA = 0, cntPB = 0;
       bool ok = true;
       const uint32_t idesc_pv = umma_idesc_bf16(128, D, 0, 1);
-      auto issue_qk = [&](int X, int st, int ncols) {
+      const uint32_t sQ_u = smem_u32(sQ), sK_u = smem_u32(sK), sV_u = smem_u32(sV);
+      // S_X = Q_X K^T over `ncols` keys of K stage `st`; X is 0 (tile A) or 1 (tile B)
+      auto issue_qk = [&](const int X, int st, int ncols) {
         const uint32_t idesc = umma_idesc_bf16(128, ncols, 0, 0);
-        const uint32_t qa = smem_u32(sQ + X * TILE_BYTES), kb = smem_u32(sK + st * TILE_BYTES);
+        const uint32_t qa = sQ_u + X * TILE_BYTES, kb = sK_u + st * TILE_BYTES;
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
           const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
@@ -204,8 +212,9 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         }
         umma_commit(&s_full[X]);
       };
-      auto issue_pv = [&](int X, int st, int ncols, bool acc) {
-        const uint32_t vb = smem_u32(sV + st * TILE_BYTES);
+      // O_X (+)= P_X V over `ncols` keys of V stage `st`; P_X is read from TMEM
+      auto issue_pv = [&](const int X, int st, int ncols, bool acc) {
+        const uint32_t vb = sV_u + st * TILE_BYTES;
         for (int ks = 0; ks < ncols / 16; ++ks)
           umma_ts(tmem + 256 + X * 128, tmem + X * 128 + ks * 8, smem_desc_sw128(vb + ks * 2048, 16384, 1024),
                   idesc_pv, acc || ks > 0);
@@ -214,46 +223,62 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         const int idx = item_index(k, n_items);
         ItemGeom g;
         if (idx < 0 || !load_item(p, idx, g)) continue;
-        const int win[2] = {g.un.winA, g.un.winB};
-        const int nX[2] = {g.nA, g.nB};
+        const int nA = g.nA, nB = g.nB, n = g.n, winA = g.un.winA, winB = g.un.winB;
         if (!mbar_wait(q_full, q_cnt & 1, abortf, LIM)) { ok = false; break; }
         ++q_cnt;
         if (!mbar_wait(&k_full[kt & 1], (kt >> 1) & 1, abortf, LIM)) { ok = false; break; }
         tc_fence_after();
-        for (int X = 0; X < 2; ++X)
-          if (0 < nX[X]) issue_qk(X, kt & 1, round16(tile_limit(g, 0, win[X])));
+        if (nA > 0) issue_qk(0, kt & 1, round16(tile_limit(g, 0, winA)));
+        if (nB > 0) issue_qk(1, kt & 1, round16(tile_limit(g, 0, winB)));
         umma_commit(&k_empty[kt & 1]);
-        for (int j = 0; j < g.n && ok; ++j, ++kt) {
+        if (n == 1) umma_commit(q_empty);        // Q is free once its last QK has run
+        for (int j = 0; j < n; ++j, ++kt) {
           const int st = kt & 1, st1 = (kt + 1) & 1;
           if (!mbar_wait(&v_full[st], (kt >> 1) & 1, abortf, LIM)) { ok = false; break; }
-          for (int X = 0; X < 2; ++X) {
-            if (j < nX[X]) {
-              if (!mbar_wait(&p_full[X], cntP[X] & 1, abortf, LIM)) { ok = false; break; }
-              ++cntP[X];
-              tc_fence_after();
-              issue_pv(X, st, round16(tile_limit(g, j, win[X])), j > 0);
-            }
-            if (X == 1) umma_commit(&v_empty[st]);
-            if (j + 1 < nX[X]) {
-              if (X == 0 || !(j + 1 < nX[0])) {   // first use of K(j+1) in this iteration
-                if (!mbar_wait(&k_full[st1], ((kt + 1) >> 1) & 1, abortf, LIM)) { ok = false; break; }
-                tc_fence_after();
-              }
-              issue_qk(X, st1, round16(tile_limit(g, j + 1, win[X])));
-            }
+          // tile A: O_A += P_A(j) V(j), then S_A(j+1) so that softmax A can go on
+          if (j < nA) {
+            if (!mbar_wait(&p_full[0], cntPA & 1, abortf, LIM)) { ok = false; break; }
+            ++cntPA;
+            tc_fence_after();
+            issue_pv(0, st, round16(tile_limit(g, j, winA)), j > 0);
           }
-          if (ok && j + 1 < g.n) umma_commit(&k_empty[st1]);
+          if (j + 1 < nA) {
+            if (!mbar_wait(&k_full[st1], ((kt + 1) >> 1) & 1, abortf, LIM)) { ok = false; break; }
+            tc_fence_after();
+            issue_qk(0, st1, round16(tile_limit(g, j + 1, winA)));
+          }
+          // tile B
+          if (j < nB) {
+            if (!mbar_wait(&p_full[1], cntPB & 1, abortf, LIM)) { ok = false; break; }
+            ++cntPB;
+            tc_fence_after();
+            issue_pv(1, st, round16(tile_limit(g, j, winB)), j > 0);
+          }
+          umma_commit(&v_empty[st]);
+          if (j + 1 < nB) {
+            if (!(j + 1 < nA)) {
+              if (!mbar_wait(&k_full[st1], ((kt + 1) >> 1) & 1, abortf, LIM)) { ok = false; break; }
+              tc_fence_after();
+            }
+            issue_qk(1, st1, round16(tile_limit(g, j + 1, winB)));
+          }
+          if (j + 1 < n) {
+            umma_commit(&k_empty[st1]);
+            if (j + 2 == n) umma_commit(q_empty);
+          }
         }
         if (!ok) break;
-        if (g.nA > 0) umma_commit(&o_full[0]);
-        if (g.nB > 0) umma_commit(&o_full[1]);
-        umma_commit(q_empty);
+        if (nA > 0) umma_commit(&o_full[0]);
+        if (nB > 0) umma_commit(&o_full[1]);
       }
     }
     __syncwarp();
+  } else if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
   } else {
     // ------------------------------------------------- softmax + epilogue
-    const int X = (warp - 2) >> 2;                 // 0: tile A, 1: tile B
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+    const int X = (warp - 4) >> 2;                 // 0: tile A, 1: tile B
     const int quad = warp & 3;                     // TMEM lane quadrant of this warp
     const int row = quad * 32 + lane;              // query row of the tile
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;

@@ -12,16 +12,7 @@ from paper_2607_17652_b200 import synth
 
 
 def common_cfg(stc: synth.Structure, **over) -> dict:
-    wl = stc.wl
-    d = dict(max_requests=wl.n_requests, wmax=wl.wmax, block_len=wl.block_len,
-             n_q_heads=wl.n_q_heads, n_kv_heads=wl.n_kv_heads,
-             head_dim=wl.head_dim, page_size=wl.page_size,
-             num_pages=stc.num_pages, max_pages_per_req=stc.max_pages_per_req,
-             vocab=wl.vocab, mask_id=stc.mask_id, eos_id=stc.eos_id,
-             max_blocks=wl.max_blocks, s_pe=wl.s_pe, tau_mask=wl.tau_mask,
-             tau_edit=wl.tau_edit, theta_spawn=wl.theta_spawn, sm_scale=0.0)
-    d.update(over)
-    return d
+    return synth.config_dict(stc, **over)
 
 
 def oracle_cfg(stc, **over) -> O.Config:
