@@ -34,6 +34,18 @@ namespace fb {
 constexpr int kAttnThreads = 384;   // 3 warpgroups: control, softmax A, softmax B
 constexpr float kLog2eF = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
+// Dynamic shared memory per CTA.  Both sizes exceed half of the 227 KB an SM
+// offers, so two CTAs never share an SM: each CTA allocates all 512 TMEM columns.
+constexpr int kSmem64 = 120 * 1024;
+constexpr int kSmem128 = 6 * 32768 + 2048;
+
+// Optional per-role timeline of CTA 0 (debug builds with -DFB_TRACE only).
+#ifdef FB_TRACE
+#define FB_TR(role, tag) do { if (blockIdx.x == 0 && tr_n < 4096) { p.trace[(role) * 8192 + 2 * tr_n] = (tag); \
+    p.trace[(role) * 8192 + 2 * tr_n + 1] = clock64(); ++tr_n; } } while (0)
+#else
+#define FB_TR(role, tag) do { } while (0)
+#endif
 
 struct AttnParams {
   const SchedHeader* hdr;
@@ -47,6 +59,9 @@ struct AttnParams {
   int32_t bl, n_q_heads, n_kv_heads, group, max_pages_per_req, num_pages;
   float scale_log2;
   long long wait_cycles;
+#ifdef FB_TRACE
+  long long* trace;
+#endif
 };
 
 // Geometry of one work item, computed identically by every role.
@@ -69,6 +84,36 @@ __device__ __forceinline__ bool load_item(const AttnParams& p, int idx, ItemGeom
   g.nB = g.un.slotB >= 0 ? max(0, min(je, g.un.nvisB) - g.jb) : 0;
   g.n = max(g.nA, g.nB);
   return g.n > 0;
+}
+
+__device__ __forceinline__ int uni(int x) { return __shfl_sync(0xffffffffu, x, 0); }
+
+// The subset of an item the control warps need, made warp-uniform (every lane
+// holds lane 0's copy) so that the compiler keeps it in uniform registers.
+struct ItemU {
+  int req, kvh, rowA, rowB, jb, n, nA, nB, npt, prefix_len, win_row0, winA, winB;
+  __device__ __forceinline__ int limit(int j, int winX) const {
+    const int gj = jb + j;
+    const int lim = gj < npt ? prefix_len - gj * kTileN : winX - (gj - npt) * kTileN;
+    return min(lim, kTileN);
+  }
+};
+
+__device__ __forceinline__ bool load_item_uniform(const AttnParams& p, int idx, ItemU& u) {
+  ItemGeom g;
+  load_item(p, idx, g);
+  u.req = uni(g.un.req); u.kvh = uni(g.un.kvh);
+  u.rowA = uni(g.un.slotA * p.bl + g.un.t0A); u.rowB = uni(g.un.slotB * p.bl + g.un.t0B);
+  u.jb = uni(g.jb); u.n = uni(g.n); u.nA = uni(g.nA); u.nB = uni(g.nB);
+  u.npt = uni(g.un.npt); u.prefix_len = uni(g.un.prefix_len); u.win_row0 = uni(g.un.win_row0);
+  u.winA = uni(g.un.winA); u.winB = uni(g.un.winB);
+  return u.n > 0;
+}
+
+// All lanes of a converged warp wait on the barrier; the result is uniform.
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort, long long limit) {
+  const bool ok = mbar_wait(bar, parity, abort, limit);
+  return __all_sync(0xffffffffu, ok);
 }
 
 // number of keys of local tile j that tile X (window reach winX) may see
@@ -110,7 +155,8 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   uint64_t* s_full = bars + 10;   // [2] A, B
   uint64_t* p_full = bars + 12;   // [2]
   uint64_t* o_full = bars + 14;   // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  uint64_t* p_half = bars + 16;   // [2] first 64 keys of P stored
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
   volatile int* abortf = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -123,6 +169,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1);
       mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1);
       mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 128); mbar_init(&o_full[i], 1);
+      mbar_init(&p_half[i], 128);
     }
     fence_mbar_init();
     tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmKwin); tma_prefetch_desc(&tmVwin);
@@ -139,140 +186,191 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   // warpgroups; each role's code follows its own setmaxnreg.
   if (warp == 0) {
     // ------------------------------------------------------------ producer
+    // The whole warp runs the loop converged and one elected lane issues the
+    // copies: operands of the TMA / MMA instructions then live in uniform
+    // registers (issuing from a single diverged lane costs ~200 cycles each).
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
-    if (lane == 0) {
-      int q_uses = 0, kt_k = 0, kt_v = 0;
-      bool ok = true;
-      auto load_kv = [&](const ItemGeom& g, int j, bool isV, int& kt) -> bool {
-        const int st = kt & 1, fill = kt >> 1;
-        uint64_t* full = isV ? &v_full[st] : &k_full[st];
-        uint64_t* empty = isV ? &v_empty[st] : &k_empty[st];
-        uint8_t* dst = (isV ? sV : sK) + st * TILE_BYTES;
-        if (fill > 0 && !mbar_wait(empty, (fill - 1) & 1, abortf, LIM)) return false;
-        const int gj = g.jb + j;
-        if (gj < g.un.npt) {
-          const int npg = (gj * kTileN + kPage < g.un.prefix_len) ? 2 : 1;
+    const bool leader = elect_one();
+    int q_uses = 0, kt_k = 0, kt_v = 0;
+    bool ok = true;
+    int tr_n = leader ? 0 : 1 << 30; (void)tr_n;
+    auto load_kv = [&](const ItemU& g, int j, bool isV, int& kt) -> bool {
+      const int st = kt & 1, fill = kt >> 1;
+      uint64_t* full = isV ? &v_full[st] : &k_full[st];
+      uint64_t* empty = isV ? &v_empty[st] : &k_empty[st];
+      uint8_t* dst = (isV ? sV : sK) + st * TILE_BYTES;
+      if (fill > 0 && !warp_wait(empty, (fill - 1) & 1, abortf, LIM)) return false;
+      FB_TR(0, isV ? 2 : 1);
+      const int gj = g.jb + j;
+      if (gj < g.npt) {
+        const int npg = (gj * kTileN + kPage < g.prefix_len) ? 2 : 1;
+        int page[2];
+#pragma unroll
+        for (int pg = 0; pg < 2; ++pg) {
+          const int pidx = gj * 2 + pg;
+          page[pg] = (pg < npg && pidx < p.max_pages_per_req)
+                         ? __ldg(&p.page_table[(size_t)g.req * p.max_pages_per_req + pidx]) : (pg < npg ? -1 : 0);
+          if (page[pg] < 0 || page[pg] >= p.num_pages) { if (leader) atomicOr(p.status, FB_ST_BAD_PAGE); page[pg] = 0; }
+          page[pg] = uni(page[pg]);
+        }
+        if (leader) {
           mbar_arrive_expect_tx(full, npg * PAGE_BYTES);
           for (int pg = 0; pg < npg; ++pg) {
-            const int pidx = gj * 2 + pg;
-            int page = pidx < p.max_pages_per_req ? __ldg(&p.page_table[(size_t)g.un.req * p.max_pages_per_req + pidx]) : -1;
-            if (page < 0 || page >= p.num_pages) { atomicOr(p.status, FB_ST_BAD_PAGE); page = 0; }
-            const int y = (page * p.n_kv_heads + g.un.kvh) * kPage;
+            const int y = (page[pg] * p.n_kv_heads + g.kvh) * kPage;
             for (int h = 0; h < NH; ++h)
               tma_load_2d(dst + h * 16384 + pg * 8192, isV ? &tmVpool : &tmKpool, full, h * 64, y);
           }
-        } else {
-          mbar_arrive_expect_tx(full, TILE_BYTES);
-          const int row0 = g.un.win_row0 + (gj - g.un.npt) * kTileN;
-          for (int h = 0; h < NH; ++h)
-            tma_load_3d(dst + h * 16384, isV ? &tmVwin : &tmKwin, full, h * 64, g.un.kvh, row0);
         }
-        ++kt;
-        return true;
-      };
-      for (int k = 0; ok && k * (int)gridDim.x < n_items; ++k) {
-        const int idx = item_index(k, n_items);
-        ItemGeom g;
-        if (idx < 0 || !load_item(p, idx, g)) continue;
-        if (q_uses > 0 && !mbar_wait(q_empty, (q_uses - 1) & 1, abortf, LIM)) { ok = false; break; }
-        ++q_uses;
+      } else if (leader) {
+        mbar_arrive_expect_tx(full, TILE_BYTES);
+        const int row0 = g.win_row0 + (gj - g.npt) * kTileN;
+        for (int h = 0; h < NH; ++h)
+          tma_load_3d(dst + h * 16384, isV ? &tmVwin : &tmKwin, full, h * 64, g.kvh, row0);
+      }
+      __syncwarp();
+      ++kt;
+      FB_TR(0, isV ? 4 : 3);
+      return true;
+    };
+    for (int k = 0; ok && k * (int)gridDim.x < n_items; ++k) {
+      const int idx = item_index(k, n_items);
+      ItemU g;
+      if (idx < 0 || !load_item_uniform(p, idx, g)) continue;
+      FB_TR(0, 10);
+      if (q_uses > 0 && !warp_wait(q_empty, (q_uses - 1) & 1, abortf, LIM)) { ok = false; break; }
+      FB_TR(0, 11);
+      ++q_uses;
+      if (leader) {
         mbar_arrive_expect_tx(q_full, ((g.nA > 0) + (g.nB > 0)) * TILE_BYTES);
         if (g.nA > 0)
           for (int h = 0; h < NH; ++h)
-            tma_load_3d(sQ + h * 16384, &tmQ, q_full, h * 64, g.un.kvh * p.group, g.un.slotA * p.bl + g.un.t0A);
+            tma_load_3d(sQ + h * 16384, &tmQ, q_full, h * 64, g.kvh * p.group, g.rowA);
         if (g.nB > 0)
           for (int h = 0; h < NH; ++h)
-            tma_load_3d(sQ + TILE_BYTES + h * 16384, &tmQ, q_full, h * 64, g.un.kvh * p.group,
-                        g.un.slotB * p.bl + g.un.t0B);
-        if (!load_kv(g, 0, false, kt_k)) { ok = false; break; }
-        for (int j = 0; j < g.n; ++j) {
-          if (j + 1 < g.n && !load_kv(g, j + 1, false, kt_k)) { ok = false; break; }
-          if (!load_kv(g, j, true, kt_v)) { ok = false; break; }
-        }
+            tma_load_3d(sQ + TILE_BYTES + h * 16384, &tmQ, q_full, h * 64, g.kvh * p.group, g.rowB);
+      }
+      __syncwarp();
+      if (!load_kv(g, 0, false, kt_k)) { ok = false; break; }
+      for (int j = 0; j < g.n; ++j) {
+        if (j + 1 < g.n && !load_kv(g, j + 1, false, kt_k)) { ok = false; break; }
+        if (!load_kv(g, j, true, kt_v)) { ok = false; break; }
       }
     }
-    __syncwarp();
   } else if (warp == 1) {
     // ---------------------------------------------------------- MMA issuer
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
-    if (lane == 0) {
-      int q_cnt = 0, kt = 0, cntPA = 0, cntPB = 0;
-      bool ok = true;
-      const uint32_t idesc_pv = umma_idesc_bf16(128, D, 0, 1);
-      const uint32_t sQ_u = smem_u32(sQ), sK_u = smem_u32(sK), sV_u = smem_u32(sV);
-      // S_X = Q_X K^T over `ncols` keys of K stage `st`; X is 0 (tile A) or 1 (tile B)
-      auto issue_qk = [&](const int X, int st, int ncols) {
-        const uint32_t idesc = umma_idesc_bf16(128, ncols, 0, 0);
-        const uint32_t qa = sQ_u + X * TILE_BYTES, kb = sK_u + st * TILE_BYTES;
+    const bool leader = elect_one();
+    int q_cnt = 0, kt = 0, cntPA = 0, cntPB = 0;
+    bool ok = true;
+    int tr_n = leader ? 0 : 1 << 30; (void)tr_n;
+    // All descriptors are built once; a k-step only adds a constant to the
+    // address field (low word, no carry: shared-memory addresses fit the
+    // 14-bit field).
+    const uint32_t idesc_pv = umma_idesc_bf16(128, D, 0, 1);
+    const uint32_t idesc_qk_full = umma_idesc_bf16(128, kTileN, 0, 0);
+    const uint64_t dQ0 = smem_desc_sw128(smem_u32(sQ), 16, 1024);
+    const uint64_t dK0 = smem_desc_sw128(smem_u32(sK), 16, 1024);
+    const uint64_t dV0 = smem_desc_sw128(smem_u32(sV), 16384, 1024);
+    // S_X = Q_X K^T over `ncols` keys of K stage `st`; X is 0 (tile A) or 1 (tile B)
+    auto issue_qk = [&](const int X, int st, int ncols) {
+      const uint32_t idesc = ncols == kTileN ? idesc_qk_full : umma_idesc_bf16(128, ncols, 0, 0);
+      const uint64_t qa = dQ0 + (uint32_t)((X * TILE_BYTES) >> 4), kb = dK0 + (uint32_t)((st * TILE_BYTES) >> 4);
+      const uint32_t d = tmem + X * 128;
+      if (leader) {
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
-          const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
-          umma_ss(tmem + X * 128, smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(kb + off, 16, 1024), idesc,
-                  ks > 0);
+          const uint32_t off = ((ks >> 2) * 16384 + (ks & 3) * 32) >> 4;
+          umma_ss(d, qa + off, kb + off, idesc, ks > 0 ? 1u : 0u);
         }
         umma_commit(&s_full[X]);
-      };
-      // O_X (+)= P_X V over `ncols` keys of V stage `st`; P_X is read from TMEM
-      auto issue_pv = [&](const int X, int st, int ncols, bool acc) {
-        const uint32_t vb = sV_u + st * TILE_BYTES;
-        for (int ks = 0; ks < ncols / 16; ++ks)
-          umma_ts(tmem + 256 + X * 128, tmem + X * 128 + ks * 8, smem_desc_sw128(vb + ks * 2048, 16384, 1024),
-                  idesc_pv, acc || ks > 0);
-      };
-      for (int k = 0; ok && k * (int)gridDim.x < n_items; ++k) {
-        const int idx = item_index(k, n_items);
-        ItemGeom g;
-        if (idx < 0 || !load_item(p, idx, g)) continue;
-        const int nA = g.nA, nB = g.nB, n = g.n, winA = g.un.winA, winB = g.un.winB;
-        if (!mbar_wait(q_full, q_cnt & 1, abortf, LIM)) { ok = false; break; }
-        ++q_cnt;
-        if (!mbar_wait(&k_full[kt & 1], (kt >> 1) & 1, abortf, LIM)) { ok = false; break; }
-        tc_fence_after();
-        if (nA > 0) issue_qk(0, kt & 1, round16(tile_limit(g, 0, winA)));
-        if (nB > 0) issue_qk(1, kt & 1, round16(tile_limit(g, 0, winB)));
-        umma_commit(&k_empty[kt & 1]);
-        if (n == 1) umma_commit(q_empty);        // Q is free once its last QK has run
-        for (int j = 0; j < n; ++j, ++kt) {
-          const int st = kt & 1, st1 = (kt + 1) & 1;
-          if (!mbar_wait(&v_full[st], (kt >> 1) & 1, abortf, LIM)) { ok = false; break; }
-          // tile A: O_A += P_A(j) V(j), then S_A(j+1) so that softmax A can go on
-          if (j < nA) {
-            if (!mbar_wait(&p_full[0], cntPA & 1, abortf, LIM)) { ok = false; break; }
-            ++cntPA;
-            tc_fence_after();
-            issue_pv(0, st, round16(tile_limit(g, j, winA)), j > 0);
-          }
-          if (j + 1 < nA) {
-            if (!mbar_wait(&k_full[st1], ((kt + 1) >> 1) & 1, abortf, LIM)) { ok = false; break; }
-            tc_fence_after();
-            issue_qk(0, st1, round16(tile_limit(g, j + 1, winA)));
-          }
-          // tile B
-          if (j < nB) {
-            if (!mbar_wait(&p_full[1], cntPB & 1, abortf, LIM)) { ok = false; break; }
-            ++cntPB;
-            tc_fence_after();
-            issue_pv(1, st, round16(tile_limit(g, j, winB)), j > 0);
-          }
-          umma_commit(&v_empty[st]);
-          if (j + 1 < nB) {
-            if (!(j + 1 < nA)) {
-              if (!mbar_wait(&k_full[st1], ((kt + 1) >> 1) & 1, abortf, LIM)) { ok = false; break; }
-              tc_fence_after();
-            }
-            issue_qk(1, st1, round16(tile_limit(g, j + 1, winB)));
-          }
-          if (j + 1 < n) {
-            umma_commit(&k_empty[st1]);
-            if (j + 2 == n) umma_commit(q_empty);
-          }
-        }
-        if (!ok) break;
-        if (nA > 0) umma_commit(&o_full[0]);
-        if (nB > 0) umma_commit(&o_full[1]);
       }
+      __syncwarp();
+    };
+    // O_X (+)= P_X V over k-steps [ks0, ks1) of V stage `st`; P_X is read from TMEM
+    auto issue_pv = [&](const int X, int st, int ks0, int ks1, bool acc) {
+      const uint64_t vb = dV0 + (uint32_t)((st * TILE_BYTES) >> 4);
+      const uint32_t d = tmem + 256 + X * 128, a = tmem + X * 128;
+      if (leader) {
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+          if (ks >= ks0 && ks < ks1)
+            umma_ts(d, a + ks * 8, vb + (uint32_t)((ks * 2048) >> 4), idesc_pv, (acc || ks > 0) ? 1u : 0u);
+      }
+      __syncwarp();
+    };
+    auto commit = [&](uint64_t* bar) { if (leader) umma_commit(bar); __syncwarp(); };
+    for (int k = 0; ok && k * (int)gridDim.x < n_items; ++k) {
+      const int idx = item_index(k, n_items);
+      ItemU g;
+      if (idx < 0 || !load_item_uniform(p, idx, g)) continue;
+      const int nA = g.nA, nB = g.nB, n = g.n;
+      FB_TR(1, 10);
+      if (!warp_wait(q_full, q_cnt & 1, abortf, LIM)) { ok = false; break; }
+      ++q_cnt;
+      FB_TR(1, 11);
+      if (!warp_wait(&k_full[kt & 1], (kt >> 1) & 1, abortf, LIM)) { ok = false; break; }
+      FB_TR(1, 12);
+      tc_fence_after();
+      if (nA > 0) issue_qk(0, kt & 1, round16(g.limit(0, g.winA)));
+      if (nB > 0) issue_qk(1, kt & 1, round16(g.limit(0, g.winB)));
+      commit(&k_empty[kt & 1]);
+      if (n == 1) commit(q_empty);               // Q is free once its last QK has run
+      for (int j = 0; j < n; ++j, ++kt) {
+        const int st = kt & 1, st1 = (kt + 1) & 1;
+        FB_TR(1, 20);
+        if (!warp_wait(&v_full[st], (kt >> 1) & 1, abortf, LIM)) { ok = false; break; }
+        FB_TR(1, 21);
+        // tile A: O_A += P_A(j) V(j), then S_A(j+1) so that softmax A can go on
+        if (j < nA) {
+          const int nks = round16(g.limit(j, g.winA)) >> 4;
+          if (!warp_wait(&p_half[0], cntPA & 1, abortf, LIM)) { ok = false; break; }
+          FB_TR(1, 22);
+          tc_fence_after();
+          issue_pv(0, st, 0, min(nks, 4), j > 0);
+          if (!warp_wait(&p_full[0], cntPA & 1, abortf, LIM)) { ok = false; break; }
+          FB_TR(1, 23);
+          ++cntPA;
+          tc_fence_after();
+          issue_pv(0, st, 4, nks, j > 0);
+          FB_TR(1, 24);
+        }
+        if (j + 1 < nA) {
+          if (!warp_wait(&k_full[st1], ((kt + 1) >> 1) & 1, abortf, LIM)) { ok = false; break; }
+          FB_TR(1, 25);
+          tc_fence_after();
+          issue_qk(0, st1, round16(g.limit(j + 1, g.winA)));
+          FB_TR(1, 26);
+        }
+        // tile B
+        if (j < nB) {
+          const int nks = round16(g.limit(j, g.winB)) >> 4;
+          if (!warp_wait(&p_half[1], cntPB & 1, abortf, LIM)) { ok = false; break; }
+          FB_TR(1, 32);
+          tc_fence_after();
+          issue_pv(1, st, 0, min(nks, 4), j > 0);
+          if (!warp_wait(&p_full[1], cntPB & 1, abortf, LIM)) { ok = false; break; }
+          FB_TR(1, 33);
+          ++cntPB;
+          tc_fence_after();
+          issue_pv(1, st, 4, nks, j > 0);
+        }
+        commit(&v_empty[st]);
+        if (j + 1 < nB) {
+          if (!(j + 1 < nA)) {
+            if (!warp_wait(&k_full[st1], ((kt + 1) >> 1) & 1, abortf, LIM)) { ok = false; break; }
+            tc_fence_after();
+          }
+          issue_qk(1, st1, round16(g.limit(j + 1, g.winB)));
+        }
+        if (j + 1 < n) {
+          commit(&k_empty[st1]);
+          if (j + 2 == n) commit(q_empty);
+        }
+      }
+      if (!ok) break;
+      if (nA > 0) commit(&o_full[0]);
+      if (nB > 0) commit(&o_full[1]);
     }
-    __syncwarp();
   } else if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
   } else {
@@ -287,6 +385,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     const float sl2 = p.scale_log2;
     int cntS = 0, cntO = 0;
     bool ok = true;
+    int tr_n = (quad == 0 && lane == 0) ? 0 : 1 << 30; (void)tr_n;
     for (int k = 0; ok && k * (int)gridDim.x < n_items; ++k) {
       const int idx = item_index(k, n_items);
       ItemGeom g;
@@ -296,20 +395,35 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       const int winX = X == 0 ? g.un.winA : g.un.winB;
       float m_ref = -INFINITY, l = 0.f;
       for (int j = 0; j < nMine; ++j) {
+        FB_TR(2 + X, 40);
         if (!mbar_wait(&s_full[X], cntS & 1, abortf, LIM)) { ok = false; break; }
+        FB_TR(2 + X, 41);
         ++cntS;
         tc_fence_after();
         const int limit = tile_limit(g, j, winX);
         uint32_t sr[128];
         tmem_ld32(tS, sr); tmem_ld32(tS + 32, sr + 32); tmem_ld32(tS + 64, sr + 64); tmem_ld32(tS + 96, sr + 96);
         tmem_ld_wait();
-        float mx = -INFINITY;
-        if (limit >= kTileN) {
+        FB_TR(2 + X, 42);
+        // row max over the visible columns; 8 independent chains
+        float mx;
+        {
+          float m8[8];
 #pragma unroll
-          for (int i = 0; i < 128; ++i) mx = fmaxf(mx, __uint_as_float(sr[i]));
-        } else {
+          for (int t = 0; t < 8; ++t) m8[t] = -INFINITY;
+          if (limit >= kTileN) {
 #pragma unroll
-          for (int i = 0; i < 128; ++i) mx = fmaxf(mx, i < limit ? __uint_as_float(sr[i]) : -INFINITY);
+            for (int i = 0; i < 128; i += 8)
+#pragma unroll
+              for (int t = 0; t < 8; ++t) m8[t] = fmaxf(m8[t], __uint_as_float(sr[i + t]));
+          } else {
+#pragma unroll
+            for (int i = 0; i < 128; i += 8)
+#pragma unroll
+              for (int t = 0; t < 8; ++t)
+                m8[t] = fmaxf(m8[t], i + t < limit ? __uint_as_float(sr[i + t]) : -INFINITY);
+          }
+          mx = fmaxf(fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3])), fmaxf(fmaxf(m8[4], m8[5]), fmaxf(m8[6], m8[7])));
         }
         // lazy rescale: keep the old reference unless the max grew by > 2^8
         bool grow = false;
@@ -329,33 +443,44 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           }
           tmem_st_wait();
         }
+        FB_TR(2 + X, 43);
         const float mb = m_ref * sl2;
-        float sum = 0.f;
-        if (limit >= kTileN) {
+        float s4[4] = {0.f, 0.f, 0.f, 0.f};
+        // P is handed to the MMA warp in two halves of 64 keys so that the first
+        // PV k-steps run while the second half is still being exponentiated
 #pragma unroll
-          for (int i = 0; i < 128; i += 2) {
-            const float p0 = ex2_approx(fmaf(__uint_as_float(sr[i]), sl2, -mb));
-            const float p1 = ex2_approx(fmaf(__uint_as_float(sr[i + 1]), sl2, -mb));
-            sum += p0 + p1;
-            sr[i >> 1] = pack_bf16x2(p0, p1);
-          }
-        } else {
+        for (int half = 0; half < 2; ++half) {
+          if (limit >= kTileN) {
 #pragma unroll
-          for (int i = 0; i < 128; i += 2) {
-            const float p0 = i < limit ? ex2_approx(fmaf(__uint_as_float(sr[i]), sl2, -mb)) : 0.f;
-            const float p1 = i + 1 < limit ? ex2_approx(fmaf(__uint_as_float(sr[i + 1]), sl2, -mb)) : 0.f;
-            sum += p0 + p1;
-            sr[i >> 1] = pack_bf16x2(p0, p1);
+            for (int i = 64 * half; i < 64 * half + 64; i += 2) {
+              const float p0 = ex2_approx(fmaf(__uint_as_float(sr[i]), sl2, -mb));
+              const float p1 = ex2_approx(fmaf(__uint_as_float(sr[i + 1]), sl2, -mb));
+              s4[(i >> 1) & 3] += p0 + p1;
+              sr[i >> 1] = pack_bf16x2(p0, p1);
+            }
+          } else {
+#pragma unroll
+            for (int i = 64 * half; i < 64 * half + 64; i += 2) {
+              const float p0 = i < limit ? ex2_approx(fmaf(__uint_as_float(sr[i]), sl2, -mb)) : 0.f;
+              const float p1 = i + 1 < limit ? ex2_approx(fmaf(__uint_as_float(sr[i + 1]), sl2, -mb)) : 0.f;
+              s4[(i >> 1) & 3] += p0 + p1;
+              sr[i >> 1] = pack_bf16x2(p0, p1);
+            }
           }
+          FB_TR(2 + X, 44 + 3 * half);
+          tmem_st32(tS + 32 * half, sr + 32 * half);
+          tmem_st_wait();
+          FB_TR(2 + X, 45 + 3 * half);
+          tc_fence_before();
+          mbar_arrive(half == 0 ? &p_half[X] : &p_full[X]);
+          FB_TR(2 + X, 46 + 3 * half);
         }
-        l += sum;
-        tmem_st32(tS, sr); tmem_st32(tS + 32, sr + 32);
-        tmem_st_wait();
-        tc_fence_before();
-        mbar_arrive(&p_full[X]);
+        l += (s4[0] + s4[1]) + (s4[2] + s4[3]);
       }
       if (!ok) break;
+      FB_TR(2 + X, 50);
       if (!mbar_wait(&o_full[X], cntO & 1, abortf, LIM)) { ok = false; break; }
+      FB_TR(2 + X, 51);
       ++cntO;
       tc_fence_after();
       if (g.un.n_chunks <= 1) {
@@ -394,6 +519,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         }
       }
       tc_fence_before();
+      FB_TR(2 + X, 52);
     }
   }
   // ---------------------------------------------------------------- teardown
@@ -454,6 +580,12 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const AttnParams p) {
 }
 
 // ------------------------------------------------------------------- host
+#ifdef FB_TRACE
+static long long* g_trace_ptr = nullptr;
+extern "C" int fb_debug_trace(long long* host_out) {
+  return (int)cudaMemcpy(host_out, g_trace_ptr, 4 * 8192 * sizeof(long long), cudaMemcpyDeviceToHost);
+}
+#endif
 static int ensure_device(fb_ctx* ctx) {
   if (ctx->dev_ready) return FB_OK;
   int dev = 0;
@@ -470,7 +602,7 @@ static int ensure_device(fb_ctx* ctx) {
   if (!fn || q != cudaDriverEntryPointSuccess)
     return set_err(ctx, FB_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
   ctx->encode_fn = fn;
-  const int smem64 = 6 * 16384 + 2048, smem128 = 6 * 32768 + 2048;
+  const int smem64 = kSmem64, smem128 = kSmem128;
   if (int e = cuda_err(ctx, cudaFuncSetAttribute(wavefront_attn_kernel<64>,
                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, smem64), "smem attr"))
     return e;
@@ -537,16 +669,23 @@ int launch_attn(fb_ctx* ctx, const fb_pack* pk, const void* q, const void* k_win
   p.bl = c.block_len; p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.group = ctx->group;
   p.max_pages_per_req = c.max_pages_per_req; p.num_pages = c.num_pages;
   p.scale_log2 = ctx->sm_scale * kLog2eF;
+#ifdef FB_TRACE
+  static long long* g_trace = nullptr;
+  if (!g_trace) { cudaMalloc(&g_trace, 4 * 8192 * sizeof(long long)); }
+  cudaMemsetAsync(g_trace, 0, 4 * 8192 * sizeof(long long), stream);
+  p.trace = g_trace;
+  g_trace_ptr = g_trace;
+#endif
   p.wait_cycles = 2000000000LL;
   if (const char* e = getenv("FB_WAIT_CYCLES")) { long long v = atoll(e); if (v > 0) p.wait_cycles = v; }
   const int grid = ctx->num_sms;
   if (c.head_dim == 64) {
-    wavefront_attn_kernel<64><<<grid, kAttnThreads, 6 * 16384 + 2048, stream>>>(
+    wavefront_attn_kernel<64><<<grid, kAttnThreads, kSmem64, stream>>>(
         ctx->tm_q, ctx->tm_kwin, ctx->tm_vwin, ctx->tm_kpool, ctx->tm_vpool, p);
     if (int e = cuda_err(ctx, cudaGetLastError(), "wavefront_attn_kernel launch")) return e;
     attn_combine_kernel<64><<<ctx->ws.max_units, 256, 0, stream>>>(p);
   } else {
-    wavefront_attn_kernel<128><<<grid, kAttnThreads, 6 * 32768 + 2048, stream>>>(
+    wavefront_attn_kernel<128><<<grid, kAttnThreads, kSmem128, stream>>>(
         ctx->tm_q, ctx->tm_kwin, ctx->tm_vwin, ctx->tm_kpool, ctx->tm_vpool, p);
     if (int e = cuda_err(ctx, cudaGetLastError(), "wavefront_attn_kernel launch")) return e;
     attn_combine_kernel<128><<<ctx->ws.max_units, 256, 0, stream>>>(p);
