@@ -9,11 +9,12 @@
 //               works on one tile while the other is in softmax
 //   warps 2-3   idle (they complete the control warpgroup, which gives its
 //               registers to the softmax warpgroups with setmaxnreg)
-//   warps 4-11  softmax of tile A: two threads per query row, 64 key columns
-//               each: tcgen05.ld S, online max with lazy rescale of O, exp2
-//               (part of it as a polynomial on the FMA pipe), P (bf16) written
-//               back over S in TMEM, epilogue
-//   warps 12-19 the same for tile B
+//   warps 4-7   softmax of tile A, one thread per query row: tcgen05.ld S (once
+//               for the row max, once more in 32-column chunks for the
+//               exponentials), lazy rescale of O, exp2 (part of it as a
+//               polynomial on the FMA pipe), P (bf16) written back over S in
+//               TMEM, epilogue
+//   warps 8-11  the same for tile B
 // A Q tile is 128 rows = (128/G tokens) x (G query heads of one KV head) of one
 // slot.  A unit pairs two Q tiles of one request and KV head so that they
 // share each K/V tile from shared memory.  The mask is per tile: a tile of the
@@ -32,7 +33,7 @@
 
 namespace fb {
 
-constexpr int kAttnThreads = 640;   // 5 warpgroups: control, 2 x softmax A, 2 x softmax B
+constexpr int kAttnThreads = 384;   // 3 warpgroups: control, softmax A, softmax B
 constexpr float kLog2eF = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
 // Dynamic shared memory per CTA.  Both sizes exceed half of the 227 KB an SM
@@ -181,10 +182,8 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   uint64_t* p_full = bars + 12;   // [2]
   uint64_t* o_full = bars + 14;   // [2]
   uint64_t* p_half = bars + 16;   // [2] first 64 keys of P stored
-  uint64_t* x_bar = bars + 20;    // [8] max / sum exchange of a softmax warp pair
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
   volatile int* abortf = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* xbuf = reinterpret_cast<float*>(bars + 64);   // [2 parity][2 tiles][2 halves][128 rows]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const long long LIM = p.wait_cycles;
@@ -198,7 +197,6 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 128); mbar_init(&o_full[i], 1);
       mbar_init(&p_half[i], 128);
     }
-    for (int i = 0; i < 8; ++i) mbar_init(&x_bar[i], 64);
     fence_mbar_init();
     tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmKwin); tma_prefetch_desc(&tmVwin);
     tma_prefetch_desc(&tmKpool); tma_prefetch_desc(&tmVpool);
@@ -214,10 +212,10 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   // warpgroups.  All four warps of a warpgroup execute the same setmaxnreg
   // instruction, and each role's code is dominated by its warpgroup's one.
   // Registers only move inside the CTA: what the four softmax warpgroups take
-  // (4 x 128 x (104 - 96)) must not exceed what the control warpgroup gives up
-  // (128 x (96 - 56)), or setmaxnreg.inc blocks for good.
+  // (2 x 128 x (216 - 168)) must not exceed what the control warpgroup gives up
+  // (128 x (168 - 72)), or setmaxnreg.inc blocks for good.
   if (warp < 4) {
-  asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
   if (warp == 0) {
     // ------------------------------------------------------------ producer
     // The whole warp runs the loop converged and one elected lane issues the
@@ -326,8 +324,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
           if (ks >= ks0 && ks < ks1)
-            umma_ts(d, a + (ks < 4 ? ks * 8 : 64 + (ks - 4) * 8), vb + (uint32_t)((ks * 2048) >> 4), idesc_pv,
-                    (acc || ks > 0) ? 1u : 0u);
+            umma_ts(d, a + ks * 8, vb + (uint32_t)((ks * 2048) >> 4), idesc_pv, (acc || ks > 0) ? 1u : 0u);
       }
       __syncwarp();
     };
@@ -407,36 +404,18 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   }
   } else {
     // ------------------------------------------------- softmax + epilogue
-    // Eight warps per Q tile: two warps share a TMEM lane quadrant (32 query
-    // rows) and split the tile's 128 key columns, so a thread owns 64 scores
-    // of one row.  The pair exchanges its row max and row sum through shared
-    // memory under a 64-thread named barrier.
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 104;");
-    const int a = warp - 4;
-    const int X = a >> 3;                          // 0: tile A, 1: tile B
-    const int quad = a & 3;                        // TMEM lane quadrant (== warp % 4)
-    const int ch = (a >> 2) & 1;                   // column half: keys [64 ch, 64 ch + 64)
+    // Four warps per Q tile, one thread per query row (its TMEM lane).
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+    const int X = (warp - 4) >> 2;                 // 0: tile A, 1: tile B
+    const int quad = warp & 3;                     // TMEM lane quadrant of this warp
     const int row = quad * 32 + lane;              // query row of the tile
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-    const uint32_t tS = tmem + lane_base + X * 128 + ch * 64;        // my 64 fp32 score columns
-    const uint32_t tP = tS;   // my 32 packed bf16x2 P columns overwrite the start of my score columns
-    const uint32_t tO = tmem + lane_base + 256 + X * 128 + ch * (D / 2);
-    float* xrow = xbuf + X * 256 + row;            // [parity][ch] strides: 1024, 128 floats
+    const uint32_t tS = tmem + lane_base + X * 128;
+    const uint32_t tO = tmem + lane_base + 256 + X * 128;
     const float sl2 = p.scale_log2;
-    int cntS = 0, cntO = 0, xcnt = 0;
+    int cntS = 0, cntO = 0;
     bool ok = true;
-    int tr_n = (quad == 0 && lane == 0 && ch == 0) ? 0 : 1 << 30; (void)tr_n;
-    // exchange one float with the partner thread (same row, other column
-    // half): write, arrive on the pair's mbarrier (64 arrivals), bounded wait
-    uint64_t* xbar = &x_bar[X * 4 + quad];
-    auto exchange = [&](float v, float& other) -> bool {
-      xrow[(xcnt & 1) * 1024 + ch * 128] = v;
-      mbar_arrive(xbar);
-      if (!mbar_wait(xbar, xcnt & 1, abortf, LIM)) return false;
-      other = xrow[(xcnt & 1) * 1024 + (ch ^ 1) * 128];
-      ++xcnt;
-      return true;
-    };
+    int tr_n = (quad == 0 && lane == 0) ? 0 : 1 << 30; (void)tr_n;
     for (int k = 0; ok && k * (int)gridDim.x < n_items; ++k) {
       const int idx = item_index(k, n_items);
       ItemGeom g;
@@ -451,37 +430,44 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         FB_TR(2 + X, 41);
         ++cntS;
         tc_fence_after();
-        const int limit = tile_limit(g, j, winX) - ch * 64;   // visible columns of my half
-        // pass 1: row max over my visible columns (TMEM reads are cheap, so the
-        // scores are read again in pass 2 instead of being kept in registers)
+        const int limit = tile_limit(g, j, winX);
+        // pass 1: row max over the visible columns.  TMEM reads are cheap, so
+        // the scores are read again in pass 2 instead of living in registers.
         float mx;
         {
-          uint32_t sr[64];
-          tmem_ld32(tS, sr); tmem_ld32(tS + 32, sr + 32);
-          tmem_ld_wait();
-          FB_TR(2 + X, 42);
           float m8[8];
 #pragma unroll
           for (int t = 0; t < 8; ++t) m8[t] = -INFINITY;
-          if (limit >= 64) {
+          uint32_t sa[64], sb[64];
+          tmem_ld32(tS, sa); tmem_ld32(tS + 32, sa + 32);
+          tmem_ld_wait();
+          FB_TR(2 + X, 47);
+          tmem_ld32(tS + 64, sb); tmem_ld32(tS + 96, sb + 32);     // in flight during the first half
+          if (limit >= kTileN) {
 #pragma unroll
             for (int i = 0; i < 64; i += 8)
 #pragma unroll
-              for (int t = 0; t < 8; ++t) m8[t] = fmaxf(m8[t], __uint_as_float(sr[i + t]));
+              for (int t = 0; t < 8; ++t) m8[t] = fmaxf(m8[t], __uint_as_float(sa[i + t]));
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 64; i += 8)
+#pragma unroll
+              for (int t = 0; t < 8; ++t) m8[t] = fmaxf(m8[t], __uint_as_float(sb[i + t]));
           } else {
 #pragma unroll
             for (int i = 0; i < 64; i += 8)
 #pragma unroll
+              for (int t = 0; t < 8; ++t) m8[t] = fmaxf(m8[t], i + t < limit ? __uint_as_float(sa[i + t]) : -INFINITY);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 64; i += 8)
+#pragma unroll
               for (int t = 0; t < 8; ++t)
-                m8[t] = fmaxf(m8[t], i + t < limit ? __uint_as_float(sr[i + t]) : -INFINITY);
+                m8[t] = fmaxf(m8[t], 64 + i + t < limit ? __uint_as_float(sb[i + t]) : -INFINITY);
           }
           mx = fmaxf(fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3])), fmaxf(fmaxf(m8[4], m8[5]), fmaxf(m8[6], m8[7])));
         }
-        {
-          float other;
-          if (!exchange(mx, other)) { ok = false; break; }
-          mx = fmaxf(mx, other);
-        }
+        FB_TR(2 + X, 42);
         // lazy rescale: keep the old reference unless the max grew by > 2^8
         bool grow = false;
         if (j == 0) m_ref = mx;
@@ -490,7 +476,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           const float alpha = grow ? ex2_approx((m_ref - mx) * sl2) : 1.0f;
           if (grow) { m_ref = mx; l *= alpha; }
 #pragma unroll
-          for (int c = 0; c < D / 64; ++c) {
+          for (int c = 0; c < D / 32; ++c) {
             uint32_t o[32];
             tmem_ld32(tO + c * 32, o);
             tmem_ld_wait();
@@ -502,16 +488,19 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         }
         FB_TR(2 + X, 43);
         // pass 2: P = 2^(s * scale - m) in 32-column chunks; a chunk's 16 packed
-        // columns overwrite score columns this warp has already consumed
+        // columns overwrite score columns that have already been consumed.  The
+        // MMA warp is told after keys 0-63 and again after keys 64-127.
         const float mb = m_ref * sl2;
         float2 acc2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
         const float2 sl2v = make_float2(sl2, sl2), nmb = make_float2(-mb, -mb);
+        uint32_t sc[2][32];
+        tmem_ld32(tS, sc[0]);
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          if (limit <= 32 * c) break;              // nothing visible: the MMA warp skips these k-steps
-          uint32_t sr[32];
-          tmem_ld32(tS + 32 * c, sr);
+        for (int c = 0; c < 4; ++c) {
+          uint32_t* sr = sc[c & 1];
           tmem_ld_wait();
+          FB_TR(2 + X, 60 + c);
+          if (c < 3) tmem_ld32(tS + 32 * (c + 1), sc[(c + 1) & 1]);   // next chunk in flight
           if (limit >= 32 * c + 32) {
 #pragma unroll
             for (int i = 0; i < 32; i += 2) {
@@ -531,14 +520,16 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
               sr[i >> 1] = pack_bf16x2(p0, p1);
             }
           }
-          tmem_st16(tP + 16 * c, sr);
+          FB_TR(2 + X, 70 + c);
+          tmem_st16(tS + 16 * c, sr);
+          if (c == 1 || c == 3) {
+            tmem_st_wait();
+            FB_TR(2 + X, c == 1 ? 44 : 45);
+            tc_fence_before();
+            mbar_arrive(c == 1 ? &p_half[X] : &p_full[X]);
+          }
         }
         l += (acc2[0].x + acc2[0].y) + (acc2[1].x + acc2[1].y);
-        FB_TR(2 + X, 44);
-        tmem_st_wait();
-        FB_TR(2 + X, 45);
-        tc_fence_before();
-        mbar_arrive(ch == 0 ? &p_half[X] : &p_full[X]);
         FB_TR(2 + X, 46);
       }
       if (!ok) break;
@@ -547,19 +538,14 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       FB_TR(2 + X, 51);
       ++cntO;
       tc_fence_after();
-      {
-        float other;                               // row sum over both column halves
-        if (!exchange(l, other)) { ok = false; break; }
-        l += other;
-      }
       if (g.un.n_chunks <= 1) {
         const int slot = X == 0 ? g.un.slotA : g.un.slotB, t0 = X == 0 ? g.un.t0A : g.un.t0B;
         const int grow_ = slot * p.bl + t0 + row / p.group;
         const int head = g.un.kvh * p.group + row % p.group;
-        uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)grow_ * p.n_q_heads + head) * D + ch * (D / 2));
+        uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)grow_ * p.n_q_heads + head) * D);
         const float inv = 1.0f / l;
 #pragma unroll
-        for (int c = 0; c < D / 64; ++c) {
+        for (int c = 0; c < D / 32; ++c) {
           uint32_t o[32];
           tmem_ld32(tO + c * 32, o);
           tmem_ld_wait();
@@ -575,13 +561,11 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         }
       } else {
         const size_t prow = ((size_t)(g.un.part_base + g.chunk) * 2 + X) * kTileM + row;
-        if (ch == 0) {
-          p.part_ml[prow * 2 + 0] = m_ref * sl2;
-          p.part_ml[prow * 2 + 1] = l;
-        }
-        uint4* dst = reinterpret_cast<uint4*>(p.part_o + prow * D + ch * (D / 2));
+        p.part_ml[prow * 2 + 0] = m_ref * sl2;
+        p.part_ml[prow * 2 + 1] = l;
+        uint4* dst = reinterpret_cast<uint4*>(p.part_o + prow * D);
 #pragma unroll
-        for (int c = 0; c < D / 64; ++c) {
+        for (int c = 0; c < D / 32; ++c) {
           uint32_t o[32];
           tmem_ld32(tO + c * 32, o);
           tmem_ld_wait();
