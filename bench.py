@@ -344,42 +344,13 @@ def oracle_sample_step(wl, stc, tokens, z_live, attn, n_req):
     """One oracle step (pack, attention, T2T, gate/commit) on the first n_req
     decoding requests of the workload.  Returns (seconds, attention flops,
     slots, rows)."""
-    import dataclasses
     from oracle import flowblock_oracle as O
     from tests import harness as H
-    import torch
-    sub = dataclasses.replace(stc)
-    act = stc.active.copy()
-    keep = np.flatnonzero(act == 1)[:n_req]
-    act[:] = 0
-    act[keep] = 1
-    sub.active = act
-    # compact pool holding only the pages of the kept requests (input layout
-    # only: the oracle still reads every key through a page table)
-    need = (stc.prefix_len + wl.wmax * wl.block_len + wl.page_size - 1) // wl.page_size
-    pages = np.concatenate([stc.page_table[r, :need[r]] for r in keep]) if len(keep) else np.zeros(1, np.int32)
-    remap = {int(pg): i for i, pg in enumerate(pages)}
-    pt = np.zeros_like(stc.page_table)
-    for r in keep:
-        pt[r, :need[r]] = [remap[int(pg)] for pg in stc.page_table[r, :need[r]]]
-    sub.page_table, sub.num_pages = pt, len(pages)
-    ocfg = H.oracle_cfg(sub)
-    ost = H.oracle_state(sub, tokens)
-    full_pk = O.pack_wavefronts(H.oracle_cfg(stc), H.oracle_state(stc, tokens))
+    keep = np.flatnonzero(stc.active == 1)[:n_req]
+    sp = H.sub_problem(stc, tokens, attn, z_live, keep)
+    ocfg, ost, sub = sp["ocfg"], sp["ost"], sp["sub"]
+    fq, fkw, fvw, fkp, fvp, fz = sp["q"], sp["k_win"], sp["v_win"], sp["k_pool"], sp["v_pool"], sp["logits"]
     b = wl.block_len
-    rows = np.concatenate([np.arange(full_pk.req_slot_begin[r] * b, full_pk.req_slot_begin[r + 1] * b)
-                           for r in keep]) if len(keep) else np.zeros(0, np.int64)
-    trows = torch.from_numpy(rows.astype(np.int64))
-    q, kw, vw, kp, vp = attn
-    pad = ocfg.max_slots * b - len(rows)
-    def take(t):
-        x = H.f64(t[trows])
-        return np.concatenate([x, np.zeros((pad,) + x.shape[1:])], axis=0)
-    fq, fkw, fvw = take(q), take(kw), take(vw)
-    fz = H.f64(z_live[trows])
-    fz = np.concatenate([fz, np.zeros((pad, wl.vocab))], axis=0) if pad else fz
-    tp = torch.from_numpy(pages.astype(np.int64))
-    fkp, fvp = H.f64(kp[tp]), H.f64(vp[tp])
     t0 = time.perf_counter()
     opk = O.pack_wavefronts(ocfg, ost)
     O.wavefront_attn(ocfg, opk, fq, fkw, fvw, fkp, fvp, ost.page_table)

@@ -44,3 +44,50 @@ def live_rows(pk: O.Pack, b: int, slots=None) -> np.ndarray:
     if slots is None:
         return np.arange(pk.n_live * b)
     return np.concatenate([np.arange(s * b, (s + 1) * b) for s in slots])
+
+
+def sub_problem(stc, tokens, attn, z_live, keep):
+    """The oracle's view of a few requests of a large workload.
+
+    ``keep``: request indices (ascending).  Builds a structure in which only
+    those requests are decoding, a compact pool that holds just their pages
+    (the oracle still reads every key through a page table) and the slot-order
+    rows of q / k_win / v_win / logits that belong to them.  Returns a dict
+    with the oracle Config/State, float64 inputs and ``rows``: the row indices
+    of the FULL slot-order tensors the sub-problem's live rows correspond to.
+    """
+    import dataclasses
+    wl = stc.wl
+    b = wl.block_len
+    keep = [int(r) for r in keep if stc.active[r] == 1]
+    sub = dataclasses.replace(stc)
+    act = np.zeros_like(stc.active)
+    act[keep] = 1
+    sub.active = act
+    need = (stc.prefix_len + wl.wmax * b + wl.page_size - 1) // wl.page_size
+    pages = np.concatenate([stc.page_table[r, :need[r]] for r in keep]) if keep else np.zeros(1, np.int32)
+    remap = {int(pg): i for i, pg in enumerate(pages)}
+    pt = np.zeros_like(stc.page_table)
+    for r in keep:
+        pt[r, :need[r]] = [remap[int(pg)] for pg in stc.page_table[r, :need[r]]]
+    sub.page_table, sub.num_pages = pt, len(pages)
+    ocfg = oracle_cfg(sub)
+    ost = oracle_state(sub, tokens)
+    full_pk = O.pack_wavefronts(oracle_cfg(stc), oracle_state(stc, tokens))
+    rows = np.concatenate([np.arange(full_pk.req_slot_begin[r] * b, full_pk.req_slot_begin[r + 1] * b)
+                           for r in keep]) if keep else np.zeros(0, np.int64)
+    trows = torch.from_numpy(rows.astype(np.int64))
+    pad = ocfg.max_slots * b - len(rows)
+
+    def take(t):
+        x = f64(t[trows])
+        return np.concatenate([x, np.zeros((pad,) + x.shape[1:])], axis=0)
+
+    out = dict(ocfg=ocfg, ost=ost, rows=rows, sub=sub)
+    if attn is not None:
+        q, kw, vw, kp, vp = attn
+        tp = torch.from_numpy(pages.astype(np.int64))
+        out.update(q=take(q), k_win=take(kw), v_win=take(vw), k_pool=f64(kp[tp]), v_pool=f64(vp[tp]))
+    if z_live is not None:
+        out["logits"] = take(z_live)
+    return out

@@ -1,0 +1,139 @@
+"""Parity at the benchmark's full size (64 heterogeneous requests, prefixes
+1K-8K, V = 151,552), in the launch configuration bench.py times.  The oracle
+cannot do the whole batch in seconds, so it recomputes sampled requests (all
+their slots, rows and heads; every logits row of those slots) one by one, and
+the rest is covered by properties that hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import flowblock_oracle as O
+from paper_2607_17652_b200 import binding as B
+from paper_2607_17652_b200 import synth
+from tests import harness as H
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def full():
+    wl = synth.WORKLOADS[2]
+    stc = synth.make_structure(wl)
+    tokens = synth.make_tokens(stc)
+    n_live = synth.n_live_slots(stc)
+    z_live, tokens = synth.make_logits(stc, tokens, "calibrated", n_rows=n_live * wl.block_len)
+    attn = synth.make_attn_inputs(stc)
+    ctx = B.Context(**synth.config_dict(stc))
+    st = B.DeviceState.from_numpy(DEV, stc.active, stc.prefix_len, stc.L, stc.R, tokens,
+                                  np.zeros((wl.n_requests, wl.wmax), np.uint8), stc.page_table)
+    pk = B.PackBuffers.alloc(ctx, DEV)
+    sb = B.StepBuffers(ctx, DEV)
+    rows = ctx.max_slots * wl.block_len
+    logits = torch.zeros(rows, wl.vocab, dtype=torch.bfloat16, device=DEV)
+    logits[:z_live.shape[0]].copy_(z_live)
+    q, kw, vw, kp, vp = (t.to(DEV) for t in attn)
+    sb.out.fill_(7.0)
+    B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+    B.fb_wavefront_attn(ctx, pk, q, kw, vw, kp, vp, st.page_table, sb.out, sb.ws, sb.status)
+    B.fb_t2t_step(ctx, pk, logits, st, sb.argmax, sb.conf, sb.action, sb.slot_stats, sb.status)
+    torch.cuda.synchronize()
+    tokens_after = st.tokens.cpu().numpy().copy()
+    kp_before = kp[:64].clone()
+    B.fb_gate_commit(ctx, pk, sb.slot_stats, st, kw, vw, kp, vp, sb.n_committed, sb.spawned,
+                     sb.step_counters, sb.status)
+    torch.cuda.synchronize()
+    assert int(sb.status.item()) == 0
+    # requests to recompute: the longest and the shortest prefix, the widest window, a few more
+    order = np.argsort(stc.prefix_len)
+    keep = sorted({int(order[0]), int(order[-1]), int(np.argmax(stc.R - stc.L)), 5, 23, 41})
+    return dict(wl=wl, stc=stc, tokens=tokens, tokens_after=tokens_after, attn=attn, z_live=z_live,
+                ctx=ctx, st=st, pk=pk, sb=sb, keep=keep, n_live=n_live, logits=logits)
+
+
+def test_pack_full_size_bit_exact(full):
+    ref = O.pack_wavefronts(H.oracle_cfg(full["stc"]), H.oracle_state(full["stc"], full["tokens"]))
+    g = full["pk"].to_numpy()
+    assert int(g["n_live"][0]) == ref.n_live == full["n_live"]
+    for name in ("slot_req", "slot_s", "slot_pos0", "slot_kv_len", "slot_flags", "req_slot_begin", "qtok", "pos"):
+        np.testing.assert_array_equal(g[name], getattr(ref, name), err_msg=name)
+
+
+def test_attention_sampled_requests(full):
+    sp = H.sub_problem(full["stc"], full["tokens"], full["attn"], None, full["keep"])
+    opk = O.pack_wavefronts(sp["ocfg"], sp["ost"])
+    ref = O.wavefront_attn(sp["ocfg"], opk, sp["q"], sp["k_win"], sp["v_win"], sp["k_pool"], sp["v_pool"],
+                           sp["ost"].page_table)
+    n = len(sp["rows"])
+    got = full["sb"].out[torch.from_numpy(sp["rows"]).to(DEV)].float().cpu().numpy().astype(np.float64)
+    err = np.abs(got - ref[:n])
+    rel = np.linalg.norm(got - ref[:n]) / np.linalg.norm(ref[:n])
+    assert err.max() <= 1e-2 and rel <= 5e-3, (err.max(), rel)
+    assert n >= 6 * 32
+
+
+def test_attention_properties_all_rows(full):
+    """Every live output row is a convex combination of V rows drawn from
+    N(0,1): finite, and (softmax weights sum to one) bounded by the largest
+    |v|; padding rows are untouched."""
+    wl, sb, attn = full["wl"], full["sb"], full["attn"]
+    live = full["n_live"] * wl.block_len
+    out = sb.out[:live].float()
+    assert bool(torch.isfinite(out).all())
+    vmax = max(float(attn[2].float().abs().max()), float(attn[4].float().abs().max()))
+    assert float(out.abs().max()) <= vmax + 1e-2
+    assert bool((sb.out[live:].float() == 7.0).all())
+
+
+def test_t2t_sampled_requests_and_global_properties(full):
+    wl, stc, sb = full["wl"], full["stc"], full["sb"]
+    sp = H.sub_problem(stc, full["tokens"], None, full["z_live"], full["keep"])
+    opk = O.pack_wavefronts(sp["ocfg"], sp["ost"])
+    xhat, conf = O.t2t_rows(sp["ocfg"], opk, sp["logits"])
+    n = len(sp["rows"])
+    for thr in (np.float32(wl.tau_mask), np.float32(wl.tau_edit)):
+        assert np.abs(conf[:n] - float(thr)).min() >= 1e-3
+    action, stats = O.t2t_update(sp["ocfg"], opk, sp["ost"], xhat, conf)
+    rows = torch.from_numpy(sp["rows"]).to(DEV)
+    np.testing.assert_array_equal(sb.argmax[rows].cpu().numpy(), xhat[:n])
+    np.testing.assert_allclose(sb.conf[rows].cpu().numpy(), conf[:n], rtol=0, atol=2e-5)
+    np.testing.assert_array_equal(sb.action[rows].cpu().numpy(), action[:n])
+    for r in full["keep"]:
+        np.testing.assert_array_equal(full["tokens_after"][r], sp["ost"].tokens[r], err_msg=f"tokens of request {r}")
+    # properties over all live rows: the top-1 logit really is the row maximum,
+    # the first index attaining it; confidences are probabilities
+    live = full["n_live"] * wl.block_len
+    z = full["logits"][:live]
+    am = sb.argmax[:live].long()
+    top = z.gather(1, am[:, None])[:, 0]
+    assert bool((top == z.max(dim=1).values).all())
+    first = (z == top[:, None]).float().argmax(dim=1)
+    assert bool((first == am).all())
+    cf = sb.conf[:live]
+    assert bool(((cf > 0) & (cf <= 1.0)).all())
+    # slot statistics are consistent with the per-position action codes
+    act = sb.action[:live].view(full["n_live"], wl.block_len)
+    st = sb.slot_stats[:full["n_live"]]
+    assert bool(((act == 1).sum(1) == st[:, 2]).all()) and bool(((act == 2).sum(1) == st[:, 3]).all())
+    assert int(sb.slot_stats[full["n_live"]:].abs().sum()) == 0
+
+
+def test_gate_commit_sampled_requests(full):
+    stc, sb = full["stc"], full["sb"]
+    sp = H.sub_problem(stc, full["tokens"], full["attn"], full["z_live"], full["keep"])
+    opk = O.pack_wavefronts(sp["ocfg"], sp["ost"])
+    xhat, conf = O.t2t_rows(sp["ocfg"], opk, sp["logits"])
+    action, stats = O.t2t_update(sp["ocfg"], opk, sp["ost"], xhat, conf)
+    ncom, spawned, ctr = O.gate_commit(sp["ocfg"], opk, stats, sp["ost"], sp["k_win"], sp["v_win"],
+                                       sp["k_pool"], sp["v_pool"])
+    g = full["st"].to_numpy()
+    for r in full["keep"]:
+        assert int(sb.n_committed[r]) == int(ncom[r]) and int(sb.spawned[r]) == int(spawned[r])
+        for name in ("active", "prefix_len", "L", "R"):
+            assert int(g[name][r]) == int(getattr(sp["ost"], name)[r]), (name, r)
+        np.testing.assert_array_equal(g["pe_done"][r], sp["ost"].pe_done[r])
+        np.testing.assert_array_equal(g["tokens"][r], sp["ost"].tokens[r])
+    # counters add up over the whole batch
+    c = sb.step_counters.cpu().numpy()
+    assert c[O.CT_BLOCKS] == int(sb.n_committed.sum()) and c[O.CT_SPAWNED] == int(sb.spawned.sum())
+    assert c[O.CT_LIVE_SLOTS] == full["n_live"]
