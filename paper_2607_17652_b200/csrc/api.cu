@@ -93,9 +93,15 @@ int fb_create(const fb_config* cfg, fb_ctx** out) {
   ctx->tiles_per_slot = c.block_len * G / fb::kTileM;
   ctx->tokens_per_tile = fb::kTileM / G;
   ctx->target_items = fb::kDefaultTargetItems;
+  ctx->min_chunk_tiles = fb::kDefaultMinChunkTiles;
+  // tuning knobs of the split-KV work list (results do not depend on them)
   if (const char* e = getenv("FB_ATTN_TARGET_ITEMS")) {
     int v = atoi(e);
     if (v >= 1 && v <= (1 << 20)) ctx->target_items = v;
+  }
+  if (const char* e = getenv("FB_ATTN_MIN_CHUNK_TILES")) {
+    int v = atoi(e);
+    if (v >= 1 && v <= 4096) ctx->min_chunk_tiles = v;
   }
   ctx->sm_scale = c.sm_scale > 0.f ? c.sm_scale : 1.0f / sqrtf((float)c.head_dim);
   ctx->ws = make_layout(c, ctx->tiles_per_slot, ctx->target_items);

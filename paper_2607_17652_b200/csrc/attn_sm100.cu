@@ -590,39 +590,55 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem, 512); }
 }
 
-// Merge of the split-KV partials of one unit, chunks in index order.
+// Merge of the split-KV partials, chunks in index order.  Eight CTAs per unit,
+// 32 of its 256 rows each; a warp takes one row at a time and keeps the loads
+// of four chunks in flight.
+constexpr int kCombineSplit = 8;
 template <int D>
 __global__ void __launch_bounds__(256) attn_combine_kernel(const AttnParams p) {
-  const int u = blockIdx.x;
+  const int u = blockIdx.x / kCombineSplit;
   if (u >= p.hdr->n_units) return;
   const AttnUnit un = p.units[u];
   if (un.n_chunks <= 1) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr int PER = D / 32;
-  for (int rr = warp; rr < 2 * kTileM; rr += 8) {
+  const int row0 = (blockIdx.x % kCombineSplit) * (2 * kTileM / kCombineSplit);
+  for (int rr = row0 + warp; rr < row0 + 2 * kTileM / kCombineSplit; rr += 8) {
     const int X = rr / kTileM, row = rr % kTileM;
     const int slot = X == 0 ? un.slotA : un.slotB;
     if (slot < 0) continue;
     const int nvis = X == 0 ? un.nvisA : un.nvisB, t0 = X == 0 ? un.t0A : un.t0B;
+    int nc = 0;                               // chunks that hold keys visible to this tile
+    while (nc < un.n_chunks && (int)((long long)nc * un.n_tiles / un.n_chunks) < nvis) ++nc;
+    const size_t prow0 = ((size_t)un.part_base * 2 + X) * kTileM + row;   // chunk c: + c * 2 * kTileM
     float M = -INFINITY;
-    for (int c = 0; c < un.n_chunks; ++c) {
-      const int jb = (int)((long long)c * un.n_tiles / un.n_chunks);
-      if (jb >= nvis) break;
-      M = fmaxf(M, p.part_ml[(((size_t)(un.part_base + c) * 2 + X) * kTileM + row) * 2]);
-    }
+    for (int c = lane; c < nc; c += 32) M = fmaxf(M, p.part_ml[(prow0 + (size_t)c * 2 * kTileM) * 2]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
     float acc[PER];
 #pragma unroll
     for (int i = 0; i < PER; ++i) acc[i] = 0.f;
     float L = 0.f;
-    for (int c = 0; c < un.n_chunks; ++c) {
-      const int jb = (int)((long long)c * un.n_tiles / un.n_chunks);
-      if (jb >= nvis) break;
-      const size_t prow = ((size_t)(un.part_base + c) * 2 + X) * kTileM + row;
-      const float w = ex2_approx(p.part_ml[prow * 2] - M);
-      L += w * p.part_ml[prow * 2 + 1];
-      const float* src = p.part_o + prow * D + lane * PER;
+    for (int c0 = 0; c0 < nc; c0 += 4) {
+      float w[4], lv[4], v[4][PER];
 #pragma unroll
-      for (int i = 0; i < PER; ++i) acc[i] += w * src[i];
+      for (int k = 0; k < 4; ++k) {
+        const int c = min(c0 + k, nc - 1);
+        const size_t prow = prow0 + (size_t)c * 2 * kTileM;
+        w[k] = p.part_ml[prow * 2];
+        lv[k] = p.part_ml[prow * 2 + 1];
+        const float* src = p.part_o + prow * D + lane * PER;
+#pragma unroll
+        for (int i = 0; i < PER; ++i) v[k][i] = src[i];
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (c0 + k >= nc) break;
+        const float wk = ex2_approx(w[k] - M);
+        L += wk * lv[k];
+#pragma unroll
+        for (int i = 0; i < PER; ++i) acc[i] += wk * v[k][i];
+      }
     }
     const float inv = 1.0f / L;
     const int grow_ = slot * p.bl + t0 + row / p.group;
@@ -738,12 +754,12 @@ int launch_attn(fb_ctx* ctx, const fb_pack* pk, const void* q, const void* k_win
     wavefront_attn_kernel<64><<<grid, kAttnThreads, kSmem64, stream>>>(
         ctx->tm_q, ctx->tm_kwin, ctx->tm_vwin, ctx->tm_kpool, ctx->tm_vpool, p);
     if (int e = cuda_err(ctx, cudaGetLastError(), "wavefront_attn_kernel launch")) return e;
-    attn_combine_kernel<64><<<ctx->ws.max_units, 256, 0, stream>>>(p);
+    attn_combine_kernel<64><<<ctx->ws.max_units * kCombineSplit, 256, 0, stream>>>(p);
   } else {
     wavefront_attn_kernel<128><<<grid, kAttnThreads, kSmem128, stream>>>(
         ctx->tm_q, ctx->tm_kwin, ctx->tm_vwin, ctx->tm_kpool, ctx->tm_vpool, p);
     if (int e = cuda_err(ctx, cudaGetLastError(), "wavefront_attn_kernel launch")) return e;
-    attn_combine_kernel<128><<<ctx->ws.max_units, 256, 0, stream>>>(p);
+    attn_combine_kernel<128><<<ctx->ws.max_units * kCombineSplit, 256, 0, stream>>>(p);
   }
   return cuda_err(ctx, cudaGetLastError(), "attn_combine_kernel launch");
 }

@@ -14,8 +14,8 @@ namespace fb {
 constexpr int kTileM = 128;      // query rows per Q tile (tokens x group heads)
 constexpr int kTileN = 128;      // keys per K/V tile (two 64-token pages)
 constexpr int kPage = 64;
-constexpr int kMinChunkTiles = 8;
-constexpr int kDefaultTargetItems = 8 * 148;
+constexpr int kDefaultMinChunkTiles = 4;
+constexpr int kDefaultTargetItems = 2 * 148;   // about two work items per SM before key ranges are split
 
 // One unit = one (request, KV head, pair of Q tiles); split along the key
 // axis into n_chunks items.  16 ints each, read as four int4.
@@ -48,6 +48,7 @@ struct fb_ctx {
   int tiles_per_slot;   // bl * G / 128
   int tokens_per_tile;  // 128 / G
   int target_items;
+  int min_chunk_tiles;
   float sm_scale;
   fb::WsLayout ws;
   std::string err;

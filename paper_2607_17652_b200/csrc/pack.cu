@@ -20,7 +20,7 @@ struct PackParams {
   AttnItem* items;
   AttnUnit* units;
   int32_t max_requests, wmax, bl, max_slots, max_blocks, mask_id, n_kv_heads;
-  int32_t tiles_per_slot, tokens_per_tile, target_items, max_items, max_units, max_parts;
+  int32_t tiles_per_slot, tokens_per_tile, target_items, min_chunk_tiles, max_items, max_units, max_parts;
   int32_t n_gather_blocks;
 };
 
@@ -99,7 +99,7 @@ __device__ void build_sched(const PackParams& p) {
   __syncthreads();
   if (tid == 0) {
     long long ct = (sh_total + p.target_items - 1) / p.target_items;
-    sh_ct = (int)(ct < kMinChunkTiles ? kMinChunkTiles : (ct > (1 << 20) ? (1 << 20) : ct));
+    sh_ct = (int)(ct < p.min_chunk_tiles ? p.min_chunk_tiles : (ct > (1 << 20) ? (1 << 20) : ct));
   }
   __syncthreads();
   const int Ct = sh_ct;
@@ -258,6 +258,7 @@ int launch_pack(fb_ctx* ctx, const fb_state* st, const fb_pack* out, void* ws, i
   p.max_slots = c.max_requests * c.wmax; p.max_blocks = c.max_blocks; p.mask_id = c.mask_id;
   p.n_kv_heads = c.n_kv_heads; p.tiles_per_slot = ctx->tiles_per_slot;
   p.tokens_per_tile = ctx->tokens_per_tile; p.target_items = ctx->target_items;
+  p.min_chunk_tiles = ctx->min_chunk_tiles;
   p.max_items = ctx->ws.max_items; p.max_units = ctx->ws.max_units; p.max_parts = ctx->ws.max_parts;
   p.n_gather_blocks = (p.max_slots + kSlotsPerBlock - 1) / kSlotsPerBlock;
   pack_kernel<<<p.n_gather_blocks + 1, kPackThreads, 0, stream>>>(p);
