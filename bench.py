@@ -154,6 +154,20 @@ def build_inputs(wl, seed):
     return stc, tokens, n_live, z, attn
 
 
+def combine_ranks(times_ms, work, device, world):
+    """Whole-job figures from per-rank ones: every rank ran its own batch
+    (replicas, no data-path collective), so times combine as the MAX over
+    ranks and work as the SUM."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(times_ms, dtype=torch.float64, device=device)
+    w = torch.tensor(work, dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(w, op=dist.ReduceOp.SUM)
+    return [float(x) for x in t.cpu()], [float(x) for x in w.cpu()]
+
+
 # ---------------------------------------------------------------- our arm
 def run_ours(args):
     import torch
@@ -277,13 +291,8 @@ def run_ours(args):
     stc = stc0
     flops = flops_state
     ms_step = total_ms / args.steps
-    tms = torch.tensor([ms_step, e2e_ms], dtype=torch.float64, device=dev)
-    fl = torch.tensor([flops, t2t_bytes(stc, n_live)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
-        dist.all_reduce(fl, op=dist.ReduceOp.SUM)
-    ms_step_max, e2e_ms_max = (float(x) for x in tms.cpu())
-    flops_all, t2tb_all = (float(x) for x in fl.cpu())
+    (ms_step_max, e2e_ms_max), (flops_all, t2tb_all) = combine_ranks(
+        [ms_step, e2e_ms], [flops, t2t_bytes(stc, n_live)], dev, world)
 
     if rank == 0:
         peaks = load_peaks()
