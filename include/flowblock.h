@@ -160,6 +160,33 @@ int fb_wavefront_attn(fb_ctx* ctx, const fb_pack* pk, const void* q,
                       const int32_t* page_table, void* out, void* ws,
                       int32_t* status, void* stream);
 
+/* The paper has no counterpart to this call: it exists for callers that
+ * cannot allocate device memory (an engine that has given the whole device
+ * to its own pool, a plugin in a pre-partitioned process, a loop that must
+ * not take cudaMalloc's implicit synchronisation) and therefore cannot
+ * provide the workspace fb_wavefront_attn needs.  Same computation and same
+ * tensors as fb_pack_wavefronts followed by fb_wavefront_attn, but the
+ * scratch (the attention work list) lives in an 8 MiB __device__ array inside
+ * the library image; no cudaMalloc / cudaFree / allocating library routine is
+ * called.  The work list is rebuilt from `st` (the arrays of `pk` are
+ * rewritten with the same values fb_pack_wavefronts gives) and never splits
+ * the key axis, so results may differ from fb_wavefront_attn in the last
+ * rounding only.
+ *   - FB_ERR_WORKSPACE when the configuration's work list does not fit in
+ *     8 MiB (about 100,000 (request, KV head, Q-tile pair) units).
+ *   - The first call on each device looks up the array's device address and
+ *     sets kernel attributes; make that call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps the previous
+ *     call's contents (every call overwrites all it reads, nothing needs
+ *     clearing): two calls that overlap on the GPU, e.g. on two streams, race.
+ *   - Every GPU that loads the library holds the 8 MiB until the process
+ *     exits. */
+int fb_wavefront_attn_static(fb_ctx* ctx, const fb_state* st,
+                             const fb_pack* pk, const void* q,
+                             const void* k_win, const void* v_win,
+                             const void* k_pool, const void* v_pool, void* out,
+                             int32_t* status, void* stream);
+
 /* Sec. 2.1 Eq. 1 and the numerator / denominator of Eq. 2.
  *   logits     [max_slots*bl, vocab] bf16, slot order
  *   argmax     [max_slots*bl] int32  top-1 token (lowest index on ties)

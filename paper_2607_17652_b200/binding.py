@@ -26,7 +26,7 @@ FB_SLOT_STATS, FB_STEP_COUNTERS = 6, 8
 
 EXPORTS = ["fb_create", "fb_destroy", "fb_last_error", "fb_workspace_bytes",
            "fb_pack_wavefronts", "fb_wavefront_attn", "fb_t2t_step",
-           "fb_gate_commit", "fb_step_host"]
+           "fb_gate_commit", "fb_step_host", "fb_wavefront_attn_static"]
 
 
 class fb_config(C.Structure):
@@ -89,6 +89,8 @@ def lib() -> C.CDLL:
                                   C.POINTER(fb_state)] + [P] * 6
         l.fb_gate_commit.argtypes = [P, C.POINTER(fb_pack), P,
                                      C.POINTER(fb_state)] + [P] * 9
+        l.fb_wavefront_attn_static.argtypes = [P, C.POINTER(fb_state),
+                                               C.POINTER(fb_pack)] + [P] * 8
         l.fb_step_host.argtypes = [P, C.POINTER(fb_state), C.POINTER(fb_pack),
                                    C.POINTER(fb_device_bufs),
                                    C.POINTER(fb_host_io), P]
@@ -225,6 +227,17 @@ def fb_wavefront_attn(ctx: Context, pk: PackBuffers, q, k_win, v_win, k_pool,
         ctx.handle, C.byref(p), _ptr(q), _ptr(k_win), _ptr(v_win),
         _ptr(k_pool), _ptr(v_pool), _ptr(page_table), _ptr(out), _ptr(ws),
         _ptr(status), _stream(stream)))
+
+
+def fb_wavefront_attn_static(ctx: Context, st: DeviceState, pk: PackBuffers, q,
+                             k_win, v_win, k_pool, v_pool, out, status,
+                             stream=None):
+    """Attention for callers that cannot allocate: no workspace argument, the
+    scratch is an array inside the library (see the header for its limits)."""
+    s, p = st.c(), pk.c()
+    ctx.check(lib().fb_wavefront_attn_static(
+        ctx.handle, C.byref(s), C.byref(p), _ptr(q), _ptr(k_win), _ptr(v_win),
+        _ptr(k_pool), _ptr(v_pool), _ptr(out), _ptr(status), _stream(stream)))
 
 
 def fb_t2t_step(ctx: Context, pk: PackBuffers, logits, st: DeviceState, argmax,
