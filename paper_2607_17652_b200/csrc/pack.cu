@@ -156,17 +156,26 @@ __device__ void build_sched(const PackParams& p) {
     }
   }
   __syncthreads();
-  // descending exclusive offsets over the cost bins (single thread: 1024 adds)
-  if (tid == 0) {
-    int run = 0;
-    for (int k = kCostBins - 1; k >= 0; --k) { int c = bins[k]; bins[k] = run; run += c; }
-    p.hdr->n_items = min(run, p.max_items);
-    p.hdr->n_units = min(unit_run, p.max_units);
-    p.hdr->chunk_tiles = Ct;
-    p.hdr->n_parts = part_run;
-    p.hdr->total_tiles = (int)min(sh_total, (long long)0x7fffffff);
-    if (run > p.max_items || unit_run > p.max_units || part_run > p.max_parts)
-      atomicOr(p.status, FB_ST_BAD_STATE);
+  // descending exclusive offsets over the cost bins: thread t owns the four
+  // bins kCostBins-1-4t .. kCostBins-4-4t (largest cost first)
+  {
+    static_assert(kCostBins == 4 * kPackThreads, "four bins per thread");
+    int c[4], sum = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { c[j] = bins[kCostBins - 1 - (4 * tid + j)]; sum += c[j]; }
+    int total_items;
+    int base = block_excl_scan(sum, &total_items, sh_scan);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { bins[kCostBins - 1 - (4 * tid + j)] = base; base += c[j]; }
+    if (tid == 0) {
+      p.hdr->n_items = min(total_items, p.max_items);
+      p.hdr->n_units = min(unit_run, p.max_units);
+      p.hdr->chunk_tiles = Ct;
+      p.hdr->n_parts = part_run;
+      p.hdr->total_tiles = (int)min(sh_total, (long long)0x7fffffff);
+      if (total_items > p.max_items || unit_run > p.max_units || part_run > p.max_parts)
+        atomicOr(p.status, FB_ST_BAD_STATE);
+    }
   }
   __syncthreads();
   // phase 4: scatter items, longest first
