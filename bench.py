@@ -35,9 +35,12 @@ if ROOT not in sys.path:
 METRIC = "packed-wavefront attn TFLOP/s & T2T-step GB/s (fraction of B200 peak)"
 DEFAULT_WORKLOAD = 2
 KERNELS_PER_STEP = 6   # pack, attention, split-KV combine, T2T rows, T2T update, gate/commit
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures
-# summarised under profiles/ (None until captured for that kernel / workload)
-NCU_TRAFFIC = {}
+# dram__bytes_read.sum + dram__bytes_write.sum from the ncu captures summarised
+# under profiles/, as a ratio to the algorithmic bytes of the captured (smaller)
+# case of the same workload; a full launch's traffic is that ratio times its
+# algorithmic bytes (traffic grows in proportion to the requests processed).
+NCU_TRAFFIC_RATIO = {("attn", 2): (983.35 + 31.93) / 775.4,    # profiles/wavefront_attn_cfg2_32req.txt
+                     ("t2t", 2): (504.38 + 4.62) / 504.4}      # profiles/t2t_rows_cfg2_16req.txt
 
 
 def load_peaks():
@@ -302,14 +305,16 @@ def run_ours(args):
         roof_attn = {"kernel": "wavefront_attn_kernel(+combine)", "bound": "tensor",
                      "achieved": round(attn_tf, 2), "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                      "frac": round(attn_tf / peaks["bf16_tflops"], 4),
-                     "traffic": NCU_TRAFFIC.get(("attn", args.workload)),
+                     "traffic": (round(NCU_TRAFFIC_RATIO[("attn", args.workload)] * abytes_state)
+                                 if ("attn", args.workload) in NCU_TRAFFIC_RATIO and not args.requests else None),
                      "peak_source": peaks["source"] + " cuBLAS bf16 burst",
                      "hbm_floor_ms": round(abytes_state / peaks["hbm_gbs"] / 1e6, 4),
                      "tensor_floor_ms": round(flops / peaks["bf16_tflops"] / 1e9, 4),
                      "ms": round(attn_ms, 4)}
         roof_t2t = {"kernel": "t2t_rows_kernel(+update)", "bound": "hbm", "achieved": round(t2t_gbs, 1),
                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(t2t_gbs / peaks["hbm_gbs"], 4),
-                    "traffic": NCU_TRAFFIC.get(("t2t", args.workload)),
+                    "traffic": (round(NCU_TRAFFIC_RATIO[("t2t", args.workload)] * t2t_bytes(stc, n_live))
+                                if ("t2t", args.workload) in NCU_TRAFFIC_RATIO and not args.requests else None),
                     "peak_source": peaks["source"] + " copy bandwidth", "ms": round(t2t_ms, 4)}
         dominant = roof_attn if attn_ms >= t2t_ms else roof_t2t
         line = {
