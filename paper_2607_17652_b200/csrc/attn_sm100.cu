@@ -50,7 +50,7 @@ constexpr int kSmem128 = 6 * 32768 + 8192;
 #endif
 
 struct AttnParams {
-  const SchedHeader* hdr;
+  SchedHeader* hdr;
   const AttnItem* items;
   const AttnUnit* units;
   const int32_t* page_table;
@@ -150,14 +150,6 @@ __device__ __forceinline__ int tile_limit(const ItemGeom& g, int j, int winX) {
 }
 __device__ __forceinline__ int round16(int x) { return (x + 15) & ~15; }
 
-// static assignment of the longest-first item list: row k of width gridDim.x,
-// alternate rows reversed
-__device__ __forceinline__ int item_index(int k, int n_items) {
-  const int G = gridDim.x, c = blockIdx.x;
-  const int idx = k * G + ((k & 1) ? G - 1 - c : c);
-  return idx < n_items ? idx : -1;
-}
-
 template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKwin,
@@ -182,6 +174,9 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   uint64_t* p_full = bars + 12;   // [2]
   uint64_t* o_full = bars + 14;   // [2]
   uint64_t* p_half = bars + 16;   // [2] first 64 keys of P stored
+  uint64_t* item_full = bars + 20;   // [2] next work item published by the producer
+  uint64_t* item_empty = bars + 22;  // [2] ... and read by the MMA warp and the 8 softmax warps
+  volatile int* s_item = reinterpret_cast<volatile int*>(bars + 24);   // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
   volatile int* abortf = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -196,6 +191,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1);
       mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 128); mbar_init(&o_full[i], 1);
       mbar_init(&p_half[i], 128);
+      mbar_init(&item_full[i], 1); mbar_init(&item_empty[i], 9);
     }
     fence_mbar_init();
     tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmKwin); tma_prefetch_desc(&tmVwin);
@@ -207,6 +203,9 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const int n_items = p.hdr->n_items;
+#ifdef FB_TRACE
+  if (tid == 0) { unsigned long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); p.trace[4 * 8192 + 2 * blockIdx.x] = (long long)g; }
+#endif
 
   // The control warpgroup (warps 0-3) hands registers to the softmax
   // warpgroups.  All four warps of a warpgroup execute the same setmaxnreg
@@ -263,10 +262,23 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       FB_TR(0, isV ? 4 : 3);
       return true;
     };
-    for (int k = 0; ok && k * (int)gridDim.x < n_items; ++k) {
-      const int idx = item_index(k, n_items);
+    // Work items are handed out longest first through a global ticket; the
+    // producer draws the ticket and publishes the item to the other roles.
+    for (int k = 0; ok; ++k) {
+      if (k >= 2 && !warp_wait(&item_empty[k & 1], ((k >> 1) - 1) & 1, abortf, LIM)) { ok = false; break; }
+      int idx = 0;
+      if (lane == 0) idx = atomicAdd(&p.hdr->ticket, 1);
+      idx = uni(idx);
+      if (idx >= n_items) idx = -1;
+      if (lane == 0) { s_item[k & 1] = idx; mbar_arrive(&item_full[k & 1]); }
+      __syncwarp();
+      if (idx < 0) {
+        // the last CTA to run dry re-arms the ticket for the next launch
+        if (lane == 0 && atomicAdd(&p.hdr->done, 1) == (int)gridDim.x - 1) { p.hdr->ticket = 0; p.hdr->done = 0; }
+        break;
+      }
       ItemU g;
-      if (idx < 0 || !load_item_uniform(p, idx, g)) continue;
+      if (!load_item_uniform(p, idx, g)) continue;
       FB_TR(0, 10);
       if (q_uses > 0 && !warp_wait(q_empty, (q_uses - 1) & 1, abortf, LIM)) { ok = false; break; }
       FB_TR(0, 11);
@@ -329,10 +341,14 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       __syncwarp();
     };
     auto commit = [&](uint64_t* bar) { if (leader) umma_commit(bar); __syncwarp(); };
-    for (int k = 0; ok && k * (int)gridDim.x < n_items; ++k) {
-      const int idx = item_index(k, n_items);
+    for (int k = 0; ok; ++k) {
+      if (!warp_wait(&item_full[k & 1], (k >> 1) & 1, abortf, LIM)) { ok = false; break; }
+      const int idx = s_item[k & 1];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&item_empty[k & 1]);
+      if (idx < 0) break;
       ItemU g;
-      if (idx < 0 || !load_item_uniform(p, idx, g)) continue;
+      if (!load_item_uniform(p, idx, g)) continue;
       const int nA = g.nA, nB = g.nB, n = g.n;
       FB_TR(1, 10);
       if (!warp_wait(q_full, q_cnt & 1, abortf, LIM)) { ok = false; break; }
@@ -416,10 +432,14 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     int cntS = 0, cntO = 0;
     bool ok = true;
     int tr_n = (quad == 0 && lane == 0) ? 0 : 1 << 30; (void)tr_n;
-    for (int k = 0; ok && k * (int)gridDim.x < n_items; ++k) {
-      const int idx = item_index(k, n_items);
+    for (int k = 0; ok; ++k) {
+      if (!mbar_wait(&item_full[k & 1], (k >> 1) & 1, abortf, LIM)) { ok = false; break; }
+      const int idx = s_item[k & 1];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&item_empty[k & 1]);
+      if (idx < 0) break;
       ItemGeom g;
-      if (idx < 0 || !load_item(p, idx, g)) continue;
+      if (!load_item(p, idx, g)) continue;
       const int nMine = X == 0 ? g.nA : g.nB;
       if (nMine == 0) continue;
       const int winX = X == 0 ? g.un.winA : g.un.winB;
@@ -580,6 +600,9 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   // ---------------------------------------------------------------- teardown
   tc_fence_before();
   __syncthreads();
+#ifdef FB_TRACE
+  if (tid == 0) { unsigned long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); p.trace[4 * 8192 + 2 * blockIdx.x + 1] = (long long)g; }
+#endif
   if (*abortf) {
     if (tid == 0) atomicOr(p.status, FB_ST_DEV_TIMEOUT);
     // give copies that are still in flight time to land before the CTA's
@@ -654,7 +677,7 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const AttnParams p) {
 #ifdef FB_TRACE
 static long long* g_trace_ptr = nullptr;
 extern "C" int fb_debug_trace(long long* host_out) {
-  return (int)cudaMemcpy(host_out, g_trace_ptr, 4 * 8192 * sizeof(long long), cudaMemcpyDeviceToHost);
+  return (int)cudaMemcpy(host_out, g_trace_ptr, (4 * 8192 + 512) * sizeof(long long), cudaMemcpyDeviceToHost);
 }
 #endif
 static int ensure_device(fb_ctx* ctx) {
@@ -729,7 +752,7 @@ int launch_attn(fb_ctx* ctx, const fb_pack* pk, const void* q, const void* k_win
   }
   uint8_t* w = static_cast<uint8_t*>(ws);
   AttnParams p;
-  p.hdr = reinterpret_cast<const SchedHeader*>(w + ctx->ws.header);
+  p.hdr = reinterpret_cast<SchedHeader*>(w + ctx->ws.header);
   p.items = reinterpret_cast<const AttnItem*>(w + ctx->ws.items);
   p.units = reinterpret_cast<const AttnUnit*>(w + ctx->ws.units);
   p.page_table = page_table;
@@ -742,8 +765,8 @@ int launch_attn(fb_ctx* ctx, const fb_pack* pk, const void* q, const void* k_win
   p.scale_log2 = ctx->sm_scale * kLog2eF;
 #ifdef FB_TRACE
   static long long* g_trace = nullptr;
-  if (!g_trace) { cudaMalloc(&g_trace, 4 * 8192 * sizeof(long long)); }
-  cudaMemsetAsync(g_trace, 0, 4 * 8192 * sizeof(long long), stream);
+  if (!g_trace) { cudaMalloc(&g_trace, (4 * 8192 + 512) * sizeof(long long)); }
+  cudaMemsetAsync(g_trace, 0, (4 * 8192 + 512) * sizeof(long long), stream);
   p.trace = g_trace;
   g_trace_ptr = g_trace;
 #endif

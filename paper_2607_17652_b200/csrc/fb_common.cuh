@@ -32,7 +32,9 @@ struct __align__(16) AttnItem {
 
 struct SchedHeader {
   int32_t n_items, n_units, chunk_tiles, n_parts;
-  int32_t total_tiles, pad[11];
+  int32_t total_tiles;
+  int32_t ticket, done;                // dynamic item hand-out of the attention kernel
+  int32_t pad[9];
 };
 
 struct WsLayout {

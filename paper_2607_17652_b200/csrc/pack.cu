@@ -65,6 +65,13 @@ __device__ __forceinline__ int block_excl_scan(int v, int* total, int* sh /*[kPa
   return base + x - v;
 }
 
+// Sort key of a work item: its key-tile iterations; an iteration with two Q
+// tiles takes about 7/6 of one with a single tile (measured).
+__device__ __forceinline__ int item_cost(int nA, int nB) {
+  const int n = max(nA, nB), both = min(nA, nB);
+  return (6 * n + both + 1) >> 1;
+}
+
 struct ReqGeom {
   int w, ntq, npairs, P, npt, nt;
 };
@@ -149,7 +156,7 @@ __device__ void build_sched(const PackParams& p) {
           p.units[u] = un;
           for (int c = 0; c < un.n_chunks; ++c) {
             const int jb = (int)((long long)c * g.nt / nch), je = (int)((long long)(c + 1) * g.nt / nch);
-            int cost = max(0, min(je, un.nvisA) - jb) + max(0, min(je, un.nvisB) - jb);
+            int cost = item_cost(max(0, min(je, un.nvisA) - jb), max(0, min(je, un.nvisB) - jb));
             atomicAdd(&bins[min(cost, kCostBins - 1)], 1);
           }
         }
@@ -173,6 +180,7 @@ __device__ void build_sched(const PackParams& p) {
       p.hdr->chunk_tiles = Ct;
       p.hdr->n_parts = part_run;
       p.hdr->total_tiles = (int)min(sh_total, (long long)0x7fffffff);
+      p.hdr->ticket = 0; p.hdr->done = 0;
       if (total_items > p.max_items || unit_run > p.max_units || part_run > p.max_parts)
         atomicOr(p.status, FB_ST_BAD_STATE);
     }
@@ -184,7 +192,7 @@ __device__ void build_sched(const PackParams& p) {
     const int nch = un.n_chunks;
     for (int c = 0; c < nch; ++c) {
       const int jb = (int)((long long)c * un.n_tiles / nch), je = (int)((long long)(c + 1) * un.n_tiles / nch);
-      int cost = max(0, min(je, un.nvisA) - jb) + max(0, min(je, un.nvisB) - jb);
+      int cost = item_cost(max(0, min(je, un.nvisA) - jb), max(0, min(je, un.nvisB) - jb));
       const int at = atomicAdd(&bins[min(cost, kCostBins - 1)], 1);
       if (at < p.max_items) {
         AttnItem it; it.unit = u; it.chunk = c; it.jb = jb; it.je = je;
