@@ -365,6 +365,9 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         const int st = kt & 1, st1 = (kt + 1) & 1;
         FB_TR(1, 20);
         if (!warp_wait(&v_full[st], (kt >> 1) & 1, abortf, LIM)) { ok = false; break; }
+        // K(j+1) has normally landed by now: taking its barrier here keeps the wait
+        // off the P V -> next Q K^T stretch that the softmax warps are waiting for
+        if (j + 1 < n && !warp_wait(&k_full[st1], ((kt + 1) >> 1) & 1, abortf, LIM)) { ok = false; break; }
         FB_TR(1, 21);
         // tile A: O_A += P_A(j) V(j), then S_A(j+1) so that softmax A can go on
         if (j < nA) {
@@ -381,7 +384,6 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           FB_TR(1, 24);
         }
         if (j + 1 < nA) {
-          if (!warp_wait(&k_full[st1], ((kt + 1) >> 1) & 1, abortf, LIM)) { ok = false; break; }
           FB_TR(1, 25);
           tc_fence_after();
           issue_qk(0, st1, round16(g.limit(j + 1, g.winA)));
@@ -402,10 +404,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         }
         commit(&v_empty[st]);
         if (j + 1 < nB) {
-          if (!(j + 1 < nA)) {
-            if (!warp_wait(&k_full[st1], ((kt + 1) >> 1) & 1, abortf, LIM)) { ok = false; break; }
-            tc_fence_after();
-          }
+          tc_fence_after();
           issue_qk(1, st1, round16(g.limit(j + 1, g.winB)));
         }
         if (j + 1 < n) {
