@@ -263,7 +263,8 @@ def run_ours(args):
                     h_n_committed=torch.zeros(wl.n_requests, dtype=torch.int32).pin_memory(),
                     h_spawned=torch.zeros(wl.n_requests, dtype=torch.uint8).pin_memory(),
                     h_step_counters=torch.zeros(8, dtype=torch.int32).pin_memory(),
-                    h_status=torch.zeros(1, dtype=torch.int32).pin_memory())
+                    h_status=torch.zeros(1, dtype=torch.int32).pin_memory(),
+                    n_rows=synth.n_live_slots(stc1) * wl.block_len)
         devb = dict(q=q, k_win=kw, v_win=vw, out=sb.out, logits=logits, k_pool=kp, v_pool=vp,
                     argmax=sb.argmax, conf=sb.conf, action=sb.action, slot_stats=sb.slot_stats,
                     n_committed=sb.n_committed, spawned=sb.spawned, step_counters=sb.step_counters,
@@ -280,7 +281,7 @@ def run_ours(args):
         e1.record(stream)
         barrier()
         e2e_ms = e0.elapsed_time(e1) / e2e_steps
-        h2d = sum(t.numel() * t.element_size() for t in (hq, hkw, hvw, hz))
+        h2d = sum(host["n_rows"] * t[0].numel() * t.element_size() for t in (hq, hkw, hvw, hz))
         d2h = wl.n_requests * 4 + wl.n_requests + 8 * 4 + 4
     t2 = time.time()
     clocks = sampler.stop(t0, t2)

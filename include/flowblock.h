@@ -232,6 +232,9 @@ typedef struct {
   uint8_t* h_spawned;        /* [R_max]  */
   int32_t* h_step_counters;  /* [8]      */
   int32_t* h_status;         /* [1]      */
+  int64_t n_rows;            /* leading rows of q / k_win / v_win / logits
+                                the caller has filled (live slots * bl);
+                                0 or out of range: all max_slots*bl rows    */
 } fb_host_io;
 
 typedef struct {

@@ -52,7 +52,7 @@ class fb_pack(C.Structure):
 class fb_host_io(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in (
         "h_q", "h_k_win", "h_v_win", "h_logits", "h_n_committed", "h_spawned",
-        "h_step_counters", "h_status")]
+        "h_step_counters", "h_status")] + [("n_rows", C.c_int64)]
 
 
 class fb_device_bufs(C.Structure):
@@ -264,7 +264,8 @@ def fb_step_host(ctx: Context, st: DeviceState, pk: PackBuffers, dev: dict,
     """dev / host: dicts of tensors keyed by the C field names."""
     s, p = st.c(), pk.c()
     d = fb_device_bufs(*(_ptr(dev[n]) for n, _ in fb_device_bufs._fields_))
-    h = fb_host_io(*(_ptr(host[n]) for n, _ in fb_host_io._fields_))
+    h = fb_host_io(*(_ptr(host[n]) for n, _ in fb_host_io._fields_[:-1]),
+                   int(host.get("n_rows", 0)))
     ctx.check(lib().fb_step_host(ctx.handle, C.byref(s), C.byref(p),
                                  C.byref(d), C.byref(h), _stream(stream)))
 

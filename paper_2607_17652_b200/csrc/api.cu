@@ -184,7 +184,8 @@ int fb_step_host(fb_ctx* ctx, const fb_state* st, const fb_pack* pk, const fb_de
     return fail(ctx, FB_ERR_INVALID_ARG, "a device staging pointer is null");
   const fb_config& c = ctx->cfg;
   cudaStream_t s = (cudaStream_t)stream;
-  const size_t rows = (size_t)c.max_requests * c.wmax * c.block_len;
+  size_t rows = (size_t)c.max_requests * c.wmax * c.block_len;
+  if (io->n_rows > 0 && (size_t)io->n_rows < rows) rows = (size_t)io->n_rows;   // only the rows in use travel
   const size_t qb = rows * c.n_q_heads * c.head_dim * 2, kb = rows * c.n_kv_heads * c.head_dim * 2;
   const size_t lb = rows * (size_t)c.vocab * 2;
   int e;

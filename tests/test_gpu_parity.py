@@ -66,6 +66,17 @@ WORKLOADS = {
                                      prefix_hi=136, w_lo=1, w_hi=4),
     "tiny_noprefix": synth.tiny_workload(prefix_lo=0, prefix_hi=0, w_lo=1,
                                          w_hi=3, n_requests=4),
+    # block lengths 96 / 128 and W = 5 of the paper's robustness sweeps
+    # (Sec. 4.5, 4.6), group sizes 8 and 1
+    "tiny_b96": synth.tiny_workload(block_len=96, wmax=2, w_lo=1, w_hi=2,
+                                    n_q_heads=8, n_kv_heads=2, head_dim=128,
+                                    prefix_lo=0, prefix_hi=500, n_requests=4),
+    "tiny_b128_w5_mha": synth.tiny_workload(block_len=128, wmax=5, w_lo=1, w_hi=5,
+                                            n_q_heads=2, n_kv_heads=2, head_dim=64,
+                                            prefix_lo=3, prefix_hi=260, n_requests=4,
+                                            max_blocks=16),
+    "tiny_g8": synth.tiny_workload(n_q_heads=16, n_kv_heads=2, head_dim=128,
+                                   prefix_lo=60, prefix_hi=420, n_requests=4),
     "cfg0": synth.WORKLOADS[0],
     "cfg1": synth.WORKLOADS[1],
 }
@@ -297,12 +308,14 @@ def test_attention_isolation_from_invisible_memory():
 # --------------------------------------------------- multi-step state machine
 def test_multi_step_trajectory_matches_oracle():
     """Eight consecutive steps (pack -> attention -> T2T -> gate/commit) with
-    confidences rising by 0.05 per step: states, pools and attention outputs
-    are compared after every step, so commits and admissions of one step feed
-    the next one on both sides."""
+    confidences rising by 0.05 per step and two requests arriving at steps 2
+    and 4 (the serving-sweep pattern): states, pools and attention outputs are
+    compared after every step, so commits and admissions of one step feed the
+    next one on both sides."""
     wl = synth.tiny_workload(n_requests=5, wmax=3, w_lo=1, w_hi=2,
                              prefix_lo=40, prefix_hi=400, max_blocks=10)
-    stc = synth.make_structure(wl)
+    stc = synth.make_structure(wl, n_inactive=2)        # two requests arrive later
+    late = [int(r) for r in np.flatnonzero(stc.active == 0)]
     tokens = synth.make_tokens(stc)
     case = dict(wl=wl, stc=stc, tokens=tokens)
     ctx, st, pk, sb = gpu_objects(case, s_pe=1)
@@ -313,6 +326,10 @@ def test_multi_step_trajectory_matches_oracle():
     dkp, dvp = kp.to(DEV), vp.to(DEV)
     total_commits = 0
     for step in range(8):
+        if step in (2, 4):                  # staggered arrival: the caller writes the state row
+            r = late[step // 2 - 1]
+            ost.active[r] = 1
+            st.active[r] = 1
         # this step's synthetic model outputs, placed from the ORACLE's state
         cur = dataclasses.replace(stc)
         cur.active, cur.prefix_len, cur.L, cur.R = (ost.active.copy(), ost.prefix_len.copy(),
@@ -351,3 +368,47 @@ def test_multi_step_trajectory_matches_oracle():
         assert int(sb.status.item()) == 0
         total_commits += int(ncom.sum())
     assert total_commits >= 3, "the trajectory never committed a block"
+
+
+def test_step_host_equals_the_four_calls():
+    """fb_step_host (host buffers in, decisions out) against the four device
+    calls on a second, identical state."""
+    wl = synth.tiny_workload(n_requests=4, prefix_lo=30, prefix_hi=260)
+    case = make_case(wl, logits_kind="calibrated", conf_shift=0.25)
+    stc = case["stc"]
+    q, kw, vw, kp, vp = case["attn"]
+    z = case["logits"]
+    # device path
+    ctx, st, pk, sb = gpu_objects(case)
+    dq, dkw, dvw, dkp, dvp, dz = (t.to(DEV) for t in (q, kw, vw, kp, vp, z))
+    B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+    B.fb_wavefront_attn(ctx, pk, dq, dkw, dvw, dkp, dvp, st.page_table, sb.out, sb.ws, sb.status)
+    B.fb_t2t_step(ctx, pk, dz, st, sb.argmax, sb.conf, sb.action, sb.slot_stats, sb.status)
+    B.fb_gate_commit(ctx, pk, sb.slot_stats, st, dkw, dvw, dkp, dvp, sb.n_committed, sb.spawned,
+                     sb.step_counters, sb.status)
+    torch.cuda.synchronize()
+    # host path on fresh buffers
+    ctx2, st2, pk2, sb2 = gpu_objects(case)
+    n_rows = synth.n_live_slots(stc) * wl.block_len
+    hkp, hvp = kp.to(DEV), vp.to(DEV)
+    dev = dict(q=torch.zeros_like(dq), k_win=torch.zeros_like(dkw), v_win=torch.zeros_like(dvw), out=sb2.out,
+               logits=torch.zeros_like(dz), k_pool=hkp, v_pool=hvp, argmax=sb2.argmax, conf=sb2.conf,
+               action=sb2.action, slot_stats=sb2.slot_stats, n_committed=sb2.n_committed, spawned=sb2.spawned,
+               step_counters=sb2.step_counters, status=sb2.status, ws=sb2.ws)
+    host = dict(h_q=q.pin_memory(), h_k_win=kw.pin_memory(), h_v_win=vw.pin_memory(), h_logits=z.pin_memory(),
+                h_n_committed=torch.full((wl.n_requests,), -1, dtype=torch.int32).pin_memory(),
+                h_spawned=torch.full((wl.n_requests,), 7, dtype=torch.uint8).pin_memory(),
+                h_step_counters=torch.full((8,), -1, dtype=torch.int32).pin_memory(),
+                h_status=torch.full((1,), -1, dtype=torch.int32).pin_memory(), n_rows=n_rows)
+    B.fb_step_host(ctx2, st2, pk2, dev, host)
+    torch.cuda.synchronize()
+    assert int(host["h_status"][0]) == 0
+    np.testing.assert_array_equal(host["h_n_committed"].numpy(), sb.n_committed.cpu().numpy())
+    np.testing.assert_array_equal(host["h_spawned"].numpy(), sb.spawned.cpu().numpy())
+    np.testing.assert_array_equal(host["h_step_counters"].numpy(), sb.step_counters.cpu().numpy())
+    np.testing.assert_array_equal(sb2.out[:n_rows].float().cpu().numpy(), sb.out[:n_rows].float().cpu().numpy())
+    a, b2 = st.to_numpy(), st2.to_numpy()
+    for name in ("active", "prefix_len", "L", "R", "tokens", "pe_done"):
+        np.testing.assert_array_equal(a[name], b2[name], err_msg=name)
+    assert torch.equal(hkp, dkp) and torch.equal(hvp, dvp)
+    assert bool((dev["logits"][n_rows:] == 0).all())      # rows beyond n_rows were not copied
