@@ -89,24 +89,26 @@ __device__ __forceinline__ ReqGeom req_geom(const PackParams& p, int r, int32_t*
 __device__ void build_sched(const PackParams& p) {
   __shared__ int sh_scan[kPackThreads / 32 + 1];
   __shared__ int bins[kCostBins];
-  __shared__ long long sh_total;
+  __shared__ int sh_total;
   __shared__ int sh_ct;
   const int tid = threadIdx.x;
   // bad states are reported once, by the gather blocks (null status here)
   // phase 1: total key-tile work -> chunk length
-  long long mine = 0;
+  int mine = 0;
   for (int r = tid; r < p.max_requests; r += kPackThreads) {
     ReqGeom g = req_geom(p, r, nullptr);
-    mine += (long long)g.npairs * p.n_kv_heads * g.nt;
+    mine += g.npairs * p.n_kv_heads * g.nt;
   }
   if (tid == 0) sh_total = 0;
   for (int i = tid; i < kCostBins; i += kPackThreads) bins[i] = 0;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
   __syncthreads();
-  atomicAdd((unsigned long long*)&sh_total, (unsigned long long)mine);
+  if ((tid & 31) == 0) atomicAdd(&sh_total, mine);
   __syncthreads();
   if (tid == 0) {
-    long long ct = (sh_total + p.target_items - 1) / p.target_items;
-    sh_ct = (int)(ct < p.min_chunk_tiles ? p.min_chunk_tiles : (ct > (1 << 20) ? (1 << 20) : ct));
+    const int ct = (sh_total + p.target_items - 1) / p.target_items;
+    sh_ct = ct < p.min_chunk_tiles ? p.min_chunk_tiles : ct;
   }
   __syncthreads();
   const int Ct = sh_ct;
@@ -155,7 +157,7 @@ __device__ void build_sched(const PackParams& p) {
           un.prefix_len = g.P; un.npt = g.npt; un.win_row0 = first * p.bl;
           p.units[u] = un;
           for (int c = 0; c < un.n_chunks; ++c) {
-            const int jb = (int)((long long)c * g.nt / nch), je = (int)((long long)(c + 1) * g.nt / nch);
+            const int jb = c * g.nt / nch, je = (c + 1) * g.nt / nch;
             int cost = item_cost(max(0, min(je, un.nvisA) - jb), max(0, min(je, un.nvisB) - jb));
             atomicAdd(&bins[min(cost, kCostBins - 1)], 1);
           }
@@ -179,7 +181,7 @@ __device__ void build_sched(const PackParams& p) {
       p.hdr->n_units = min(unit_run, p.max_units);
       p.hdr->chunk_tiles = Ct;
       p.hdr->n_parts = part_run;
-      p.hdr->total_tiles = (int)min(sh_total, (long long)0x7fffffff);
+      p.hdr->total_tiles = sh_total;
       p.hdr->ticket = 0; p.hdr->done = 0;
       if (total_items > p.max_items || unit_run > p.max_units || part_run > p.max_parts)
         atomicOr(p.status, FB_ST_BAD_STATE);
@@ -191,7 +193,7 @@ __device__ void build_sched(const PackParams& p) {
     const AttnUnit un = p.units[u];
     const int nch = un.n_chunks;
     for (int c = 0; c < nch; ++c) {
-      const int jb = (int)((long long)c * un.n_tiles / nch), je = (int)((long long)(c + 1) * un.n_tiles / nch);
+      const int jb = c * un.n_tiles / nch, je = (c + 1) * un.n_tiles / nch;
       int cost = item_cost(max(0, min(je, un.nvisA) - jb), max(0, min(je, un.nvisB) - jb));
       const int at = atomicAdd(&bins[min(cost, kCostBins - 1)], 1);
       if (at < p.max_items) {
@@ -229,33 +231,30 @@ __global__ void __launch_bounds__(kPackThreads) pack_kernel(const PackParams p) 
   }
   if (blockIdx.x == 0 && tid == 0) { p.req_slot_begin[p.max_requests] = run; *p.n_live = run; }
   __syncthreads();
-  for (int k = 0; k < kSlotsPerBlock; ++k) {
+  // all slots of this block at once: one thread per (slot, token)
+  for (int i = tid; i < kSlotsPerBlock * p.bl; i += kPackThreads) {
+    const int k = i / p.bl, t = i % p.bl;
     const int slot = slot0 + k;
     if (slot >= p.max_slots) break;
     const int r = s_req[k];
     if (r < 0) {
-      if (tid == 0) {
+      if (t == 0) {
         p.slot_req[slot] = -1; p.slot_s[slot] = 0; p.slot_pos0[slot] = 0; p.slot_kv_len[slot] = 0;
         p.slot_flags[slot] = 0;
       }
-      for (int t = tid; t < p.bl; t += kPackThreads) {
-        p.qtok[slot * p.bl + t] = p.mask_id; p.pos[slot * p.bl + t] = 0;
-      }
+      p.qtok[slot * p.bl + t] = p.mask_id; p.pos[slot * p.bl + t] = 0;
       continue;
     }
     const int s = s_idx[k], w = s_w[k];
     const int P = p.prefix_len[r], g = p.L[r] + s;
     const int pos0 = P + s * p.bl;
-    if (tid == 0) {
+    if (t == 0) {
       p.slot_req[slot] = r; p.slot_s[slot] = s; p.slot_pos0[slot] = pos0;
       p.slot_kv_len[slot] = P + (s + 1) * p.bl;
       p.slot_flags[slot] = (s == 0 ? FB_FLAG_OLDEST : 0) | (s == w - 1 ? FB_FLAG_FRONTIER : 0);
     }
-    const int32_t* src = p.tokens + (size_t)r * p.max_blocks * p.bl + (size_t)g * p.bl;
-    for (int t = tid; t < p.bl; t += kPackThreads) {
-      p.qtok[slot * p.bl + t] = src[t];        // Eq. 4: qtok = x[b, o_b + ...]
-      p.pos[slot * p.bl + t] = pos0 + t;       //        pos  = o_b + ...
-    }
+    p.qtok[slot * p.bl + t] = p.tokens[(size_t)r * p.max_blocks * p.bl + (size_t)g * p.bl + t];  // Eq. 4: qtok = x[b, o_b + ...]
+    p.pos[slot * p.bl + t] = pos0 + t;                                                           //        pos  = o_b + ...
   }
 }
 
