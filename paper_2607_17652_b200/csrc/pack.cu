@@ -132,7 +132,9 @@ __device__ void build_sched(const PackParams& p) {
     if (r < p.max_requests && nunits) {
       for (int pr = 0; pr < g.npairs; ++pr)
         for (int h = 0; h < p.n_kv_heads; ++h) {
-          const int u = ubase + pr * p.n_kv_heads + h;
+          // the Q-tile pairs of one (request, KV head) get adjacent unit numbers: they stream the
+          // same K/V, are handed out back to back and so share it through L2
+          const int u = ubase + h * g.npairs + pr;
           if (u >= p.max_units) continue;
           const int qa = 2 * pr, qb = 2 * pr + 1;
           AttnUnit un;
@@ -152,7 +154,7 @@ __device__ void build_sched(const PackParams& p) {
             un.slotB = -1; un.t0B = 0; un.winB = 0; un.nvisB = 0;
           }
           un.n_tiles = g.nt; un.n_chunks = nch;
-          un.part_base = nch > 1 ? pbase + (pr * p.n_kv_heads + h) * nch : -1;
+          un.part_base = nch > 1 ? pbase + (h * g.npairs + pr) * nch : -1;
           if (nch > 1 && un.part_base + nch > p.max_parts) un.n_chunks = 0;  // cannot happen; see header
           un.prefix_len = g.P; un.npt = g.npt; un.win_row0 = first * p.bl;
           p.units[u] = un;
