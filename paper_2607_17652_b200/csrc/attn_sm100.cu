@@ -173,7 +173,6 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   uint64_t* s_full = bars + 10;   // [2] A, B
   uint64_t* p_full = bars + 12;   // [2]
   uint64_t* o_full = bars + 14;   // [2]
-  uint64_t* p_half = bars + 16;   // [2] first 64 keys of P stored
   uint64_t* item_full = bars + 20;   // [2] next work item published by the producer
   uint64_t* item_empty = bars + 22;  // [2] ... and read by the MMA warp and the 8 softmax warps
   volatile int* s_item = reinterpret_cast<volatile int*>(bars + 24);   // [2]
@@ -190,7 +189,6 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1);
       mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1);
       mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 128); mbar_init(&o_full[i], 1);
-      mbar_init(&p_half[i], 128);
       mbar_init(&item_full[i], 1); mbar_init(&item_empty[i], 9);
     }
     fence_mbar_init();
@@ -372,15 +370,11 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         // tile A: O_A += P_A(j) V(j), then S_A(j+1) so that softmax A can go on
         if (j < nA) {
           const int nks = round16(g.limit(j, g.winA)) >> 4;
-          if (!warp_wait(&p_half[0], cntPA & 1, abortf, LIM)) { ok = false; break; }
-          FB_TR(1, 22);
-          tc_fence_after();
-          issue_pv(0, st, 0, min(nks, 4), j > 0);
           if (!warp_wait(&p_full[0], cntPA & 1, abortf, LIM)) { ok = false; break; }
           FB_TR(1, 23);
           ++cntPA;
           tc_fence_after();
-          issue_pv(0, st, 4, nks, j > 0);
+          issue_pv(0, st, 0, nks, j > 0);
           FB_TR(1, 24);
         }
         if (j + 1 < nA) {
@@ -392,15 +386,11 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         // tile B
         if (j < nB) {
           const int nks = round16(g.limit(j, g.winB)) >> 4;
-          if (!warp_wait(&p_half[1], cntPB & 1, abortf, LIM)) { ok = false; break; }
-          FB_TR(1, 32);
-          tc_fence_after();
-          issue_pv(1, st, 0, min(nks, 4), j > 0);
           if (!warp_wait(&p_full[1], cntPB & 1, abortf, LIM)) { ok = false; break; }
           FB_TR(1, 33);
           ++cntPB;
           tc_fence_after();
-          issue_pv(1, st, 4, nks, j > 0);
+          issue_pv(1, st, 0, nks, j > 0);
         }
         commit(&v_empty[st]);
         if (j + 1 < nB) {
@@ -508,7 +498,8 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         FB_TR(2 + X, 43);
         // pass 2: P = 2^(s * scale - m) in 32-column chunks; a chunk's 16 packed
         // columns overwrite score columns that have already been consumed.  The
-        // MMA warp is told after keys 0-63 and again after keys 64-127.
+        // MMA warp is told once per tile: every extra barrier it has to take
+        // costs more than starting P V a little earlier gains.
         const float mb = m_ref * sl2;
         float2 acc2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
         const float2 sl2v = make_float2(sl2, sl2), nmb = make_float2(-mb, -mb);
@@ -541,11 +532,11 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           }
           FB_TR(2 + X, 70 + c);
           tmem_st16(tS + 16 * c, sr);
-          if (c == 1 || c == 3) {
+          if (c == 3) {
             tmem_st_wait();
-            FB_TR(2 + X, c == 1 ? 44 : 45);
+            FB_TR(2 + X, 45);
             tc_fence_before();
-            mbar_arrive(c == 1 ? &p_half[X] : &p_full[X]);
+            mbar_arrive(&p_full[X]);
           }
         }
         l += (acc2[0].x + acc2[0].y) + (acc2[1].x + acc2[1].y);
