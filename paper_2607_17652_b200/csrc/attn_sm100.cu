@@ -440,50 +440,80 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         ++cntS;
         tc_fence_after();
         const int limit = tile_limit(g, j, winX);
-        // pass 1: row max over the visible columns.  TMEM reads are cheap, so
-        // the scores are read again in pass 2 instead of living in registers.
-        float mx;
-        {
+        // The running reference m_ref is only re-based when a score exceeds it by
+        // more than 2^8 (lazy rescale), so the common tile needs no separate max
+        // pass: the exponentials are taken against the old reference while the
+        // largest exponent is tracked, P stays in registers, and only if the
+        // bound was broken is the tile redone against the new reference.  The
+        // first tile of an item has no reference yet and takes a max pass.
+        if (j == 0) {
           float m8[8];
 #pragma unroll
           for (int t = 0; t < 8; ++t) m8[t] = -INFINITY;
           uint32_t sa[64], sb[64];
           tmem_ld32(tS, sa); tmem_ld32(tS + 32, sa + 32);
           tmem_ld_wait();
-          FB_TR(2 + X, 47);
           tmem_ld32(tS + 64, sb); tmem_ld32(tS + 96, sb + 32);     // in flight during the first half
-          if (limit >= kTileN) {
 #pragma unroll
-            for (int i = 0; i < 64; i += 8)
+          for (int i = 0; i < 64; i += 8)
 #pragma unroll
-              for (int t = 0; t < 8; ++t) m8[t] = fmaxf(m8[t], __uint_as_float(sa[i + t]));
-            tmem_ld_wait();
+            for (int t = 0; t < 8; ++t) m8[t] = fmaxf(m8[t], i + t < limit ? __uint_as_float(sa[i + t]) : -INFINITY);
+          tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 64; i += 8)
+          for (int i = 0; i < 64; i += 8)
 #pragma unroll
-              for (int t = 0; t < 8; ++t) m8[t] = fmaxf(m8[t], __uint_as_float(sb[i + t]));
-          } else {
-#pragma unroll
-            for (int i = 0; i < 64; i += 8)
-#pragma unroll
-              for (int t = 0; t < 8; ++t) m8[t] = fmaxf(m8[t], i + t < limit ? __uint_as_float(sa[i + t]) : -INFINITY);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 64; i += 8)
-#pragma unroll
-              for (int t = 0; t < 8; ++t)
-                m8[t] = fmaxf(m8[t], 64 + i + t < limit ? __uint_as_float(sb[i + t]) : -INFINITY);
-          }
-          mx = fmaxf(fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3])), fmaxf(fmaxf(m8[4], m8[5]), fmaxf(m8[6], m8[7])));
+            for (int t = 0; t < 8; ++t)
+              m8[t] = fmaxf(m8[t], 64 + i + t < limit ? __uint_as_float(sb[i + t]) : -INFINITY);
+          m_ref = fmaxf(fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3])), fmaxf(fmaxf(m8[4], m8[5]), fmaxf(m8[6], m8[7])));
         }
         FB_TR(2 + X, 42);
-        // lazy rescale: keep the old reference unless the max grew by > 2^8
-        bool grow = false;
-        if (j == 0) m_ref = mx;
-        else grow = (mx - m_ref) * sl2 > kRescaleThreshold;
-        if (__any_sync(0xffffffffu, grow)) {
-          const float alpha = grow ? ex2_approx((m_ref - mx) * sl2) : 1.0f;
-          if (grow) { m_ref = mx; l *= alpha; }
+        uint32_t pk[64];                       // P of this tile, packed bf16 pairs
+        float tile_sum = 0.f;
+#pragma unroll 1
+        for (int attempt = 0; attempt < 2; ++attempt) {
+          const float mb = m_ref * sl2;
+          float2 acc2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+          float xm4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+          const float2 sl2v = make_float2(sl2, sl2), nmb = make_float2(-mb, -mb);
+          uint32_t sc[2][32];
+          tmem_ld32(tS, sc[0]);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint32_t* sr = sc[c & 1];
+            tmem_ld_wait();
+            if (c < 3) tmem_ld32(tS + 32 * (c + 1), sc[(c + 1) & 1]);   // next chunk in flight
+            if (limit >= 32 * c + 32) {
+#pragma unroll
+              for (int i = 0; i < 32; i += 2) {
+                const float2 x = __ffma2_rn(make_float2(__uint_as_float(sr[i]), __uint_as_float(sr[i + 1])), sl2v, nmb);
+                xm4[(i >> 1) & 3] = fmaxf(fmaxf(xm4[(i >> 1) & 3], x.x), x.y);
+                float2 pv;
+                if (((i >> 1) & 3) < FB_POLY_OF4) pv = exp2_poly2(x);
+                else pv = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+                acc2[(i >> 1) & 1] = __fadd2_rn(acc2[(i >> 1) & 1], pv);
+                pk[16 * c + (i >> 1)] = pack_bf16x2(pv.x, pv.y);
+              }
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; i += 2) {
+                const bool v0 = 32 * c + i < limit, v1 = 32 * c + i + 1 < limit;
+                const float x0 = fmaf(__uint_as_float(sr[i]), sl2, -mb), x1 = fmaf(__uint_as_float(sr[i + 1]), sl2, -mb);
+                if (v0) xm4[0] = fmaxf(xm4[0], x0);
+                if (v1) xm4[1] = fmaxf(xm4[1], x1);
+                const float p0 = v0 ? ex2_approx(x0) : 0.f, p1 = v1 ? ex2_approx(x1) : 0.f;
+                acc2[0].x += p0 + p1;
+                pk[16 * c + (i >> 1)] = pack_bf16x2(p0, p1);
+              }
+            }
+          }
+          tile_sum = (acc2[0].x + acc2[0].y) + (acc2[1].x + acc2[1].y);
+          const float xmax = fmaxf(fmaxf(xm4[0], xm4[1]), fmaxf(xm4[2], xm4[3]));
+          const bool grow = attempt == 0 && xmax > kRescaleThreshold;
+          if (!__any_sync(0xffffffffu, grow)) break;
+          // rare: re-base this row's reference, rescale what has been accumulated so far
+          // (O is quiescent: the commit behind this S also covered the previous P V)
+          const float alpha = grow ? ex2_approx(-xmax) : 1.0f;
+          if (grow) { m_ref += xmax / sl2; l *= alpha; }
 #pragma unroll
           for (int c = 0; c < D / 32; ++c) {
             uint32_t o[32];
@@ -495,51 +525,13 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           }
           tmem_st_wait();
         }
+        l += tile_sum;
         FB_TR(2 + X, 43);
-        // pass 2: P = 2^(s * scale - m) in 32-column chunks; a chunk's 16 packed
-        // columns overwrite score columns that have already been consumed.  The
-        // MMA warp is told once per tile: every extra barrier it has to take
-        // costs more than starting P V a little earlier gains.
-        const float mb = m_ref * sl2;
-        float2 acc2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-        const float2 sl2v = make_float2(sl2, sl2), nmb = make_float2(-mb, -mb);
-        uint32_t sc[2][32];
-        tmem_ld32(tS, sc[0]);
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t* sr = sc[c & 1];
-          tmem_ld_wait();
-          FB_TR(2 + X, 60 + c);
-          if (c < 3) tmem_ld32(tS + 32 * (c + 1), sc[(c + 1) & 1]);   // next chunk in flight
-          if (limit >= 32 * c + 32) {
-#pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-              const float2 x = __ffma2_rn(make_float2(__uint_as_float(sr[i]), __uint_as_float(sr[i + 1])), sl2v, nmb);
-              float2 pv;
-              if (((i >> 1) & 3) < FB_POLY_OF4) pv = exp2_poly2(x);
-              else pv = make_float2(ex2_approx(x.x), ex2_approx(x.y));
-              acc2[(i >> 1) & 1] = __fadd2_rn(acc2[(i >> 1) & 1], pv);
-              sr[i >> 1] = pack_bf16x2(pv.x, pv.y);
-            }
-          } else {
-#pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-              const float p0 = 32 * c + i < limit ? ex2_approx(fmaf(__uint_as_float(sr[i]), sl2, -mb)) : 0.f;
-              const float p1 = 32 * c + i + 1 < limit ? ex2_approx(fmaf(__uint_as_float(sr[i + 1]), sl2, -mb)) : 0.f;
-              acc2[0].x += p0 + p1;
-              sr[i >> 1] = pack_bf16x2(p0, p1);
-            }
-          }
-          FB_TR(2 + X, 70 + c);
-          tmem_st16(tS + 16 * c, sr);
-          if (c == 3) {
-            tmem_st_wait();
-            FB_TR(2 + X, 45);
-            tc_fence_before();
-            mbar_arrive(&p_full[X]);
-          }
-        }
-        l += (acc2[0].x + acc2[0].y) + (acc2[1].x + acc2[1].y);
+        tmem_st32(tS, pk); tmem_st32(tS + 32, pk + 32);
+        tmem_st_wait();
+        FB_TR(2 + X, 45);
+        tc_fence_before();
+        mbar_arrive(&p_full[X]);
         FB_TR(2 + X, 46);
       }
       if (!ok) break;
