@@ -2,12 +2,13 @@
 // wavefronts (Sec. 3.1 "W-shaped block-causal attention"; Sec. 3.2 Eq. 5).
 //
 // Persistent, warp-specialised tcgen05 kernel, one CTA per SM:
-//   warp 0      TMA producer: Q tiles, K/V tiles of the paged prefix (page-table
-//               lookups) and of the window tensors, 2-stage K and V rings
+//   warps 0, 2  TMA producers: Q tiles, K/V tiles of the paged prefix (page-table
+//               lookups) and of the window tensors, 2-stage K and V rings, one
+//               stage of each per warp
 //   warp 1      MMA issuer: S = Q K^T and O += P V with tcgen05.mma, S/P and O
 //               in TMEM, two Q tiles (A, B) ping-ponged so that the tensor pipe
 //               works on one tile while the other is in softmax
-//   warps 2-3   idle (they complete the control warpgroup, which gives its
+//   warp 3      idle (it completes the control warpgroup, which gives its
 //               registers to the softmax warpgroups with setmaxnreg)
 //   warps 4-7   softmax of tile A, one thread per query row: tcgen05.ld S (once
 //               for the row max, once more in 32-column chunks for the
@@ -43,7 +44,12 @@ constexpr int kSmem128 = 6 * 32768 + 8192;
 
 // Optional per-role timeline of CTA 0 (debug builds with -DFB_TRACE only).
 #ifdef FB_TRACE
-#define FB_TR(role, tag) do { if (blockIdx.x == 0 && tr_n < 4096) { p.trace[(role) * 8192 + 2 * tr_n] = (tag); \
+#if FB_TRACE == 2      // light: one event per key tile from the MMA warp only
+#define FB_TR_ON(role, tag) ((role) == 1 && (tag) == 20)
+#else
+#define FB_TR_ON(role, tag) true
+#endif
+#define FB_TR(role, tag) do { if (FB_TR_ON(role, tag) && blockIdx.x == 0 && tr_n < 4096) { p.trace[(role) * 8192 + 2 * tr_n] = (tag); \
     p.trace[(role) * 8192 + 2 * tr_n + 1] = clock64(); ++tr_n; } } while (0)
 #else
 #define FB_TR(role, tag) do { } while (0)
@@ -69,7 +75,7 @@ struct AttnParams {
 // Geometry of one work item, computed identically by every role.
 struct ItemGeom {
   AttnUnit un;
-  int jb, n, nA, nB, chunk;
+  int jb, n, nA, nB, chunk, kvhA, kvhB;
 };
 
 __device__ __forceinline__ bool load_item(const AttnParams& p, int idx, ItemGeom& g) {
@@ -77,6 +83,7 @@ __device__ __forceinline__ bool load_item(const AttnParams& p, int idx, ItemGeom
   const int4* up = reinterpret_cast<const int4*>(&p.units[it.x]);
   const int4 u0 = up[0], u1 = up[1], u2 = up[2], u3 = up[3];
   g.un.req = u0.x; g.un.kvh = u0.y; g.un.slotA = u0.z; g.un.slotB = u0.w;
+  g.kvhA = u0.y & 0xffff; g.kvhB = u0.y >> 16;
   g.un.t0A = u1.x; g.un.t0B = u1.y; g.un.n_tiles = u1.z; g.un.n_chunks = u1.w;
   g.un.nvisA = u2.x; g.un.nvisB = u2.y; g.un.part_base = u2.z; g.un.prefix_len = u2.w;
   g.un.npt = u3.x; g.un.win_row0 = u3.y; g.un.winA = u3.z; g.un.winB = u3.w;
@@ -117,7 +124,8 @@ __device__ __forceinline__ int uni(int x) { return __shfl_sync(0xffffffffu, x, 0
 // The subset of an item the control warps need, made warp-uniform (every lane
 // holds lane 0's copy) so that the compiler keeps it in uniform registers.
 struct ItemU {
-  int req, kvh, rowA, rowB, jb, n, nA, nB, npt, prefix_len, win_row0, winA, winB;
+  int req, kvhA, kvhB, rowA, rowB, jb, n, nA, nB, npt, prefix_len, win_row0, winA, winB;
+  __device__ __forceinline__ bool dual() const { return kvhA != kvhB; }   // two K/V streams
   __device__ __forceinline__ int limit(int j, int winX) const {
     const int gj = jb + j;
     const int lim = gj < npt ? prefix_len - gj * kTileN : winX - (gj - npt) * kTileN;
@@ -128,7 +136,7 @@ struct ItemU {
 __device__ __forceinline__ bool load_item_uniform(const AttnParams& p, int idx, ItemU& u) {
   ItemGeom g;
   load_item(p, idx, g);
-  u.req = uni(g.un.req); u.kvh = uni(g.un.kvh);
+  u.req = uni(g.un.req); u.kvhA = uni(g.kvhA); u.kvhB = uni(g.kvhB);
   u.rowA = uni(g.un.slotA * p.bl + g.un.t0A); u.rowB = uni(g.un.slotB * p.bl + g.un.t0B);
   u.jb = uni(g.jb); u.n = uni(g.n); u.nA = uni(g.nA); u.nB = uni(g.nB);
   u.npt = uni(g.un.npt); u.prefix_len = uni(g.un.prefix_len); u.win_row0 = uni(g.un.win_row0);
@@ -174,7 +182,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   uint64_t* p_full = bars + 12;   // [2]
   uint64_t* o_full = bars + 14;   // [2]
   uint64_t* item_full = bars + 20;   // [2] next work item published by the producer
-  uint64_t* item_empty = bars + 22;  // [2] ... and read by the MMA warp and the 8 softmax warps
+  uint64_t* item_empty = bars + 22;  // [2] ... and read by the second producer, the MMA warp and the 8 softmax warps
   volatile int* s_item = reinterpret_cast<volatile int*>(bars + 24);   // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
   volatile int* abortf = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -189,7 +197,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1);
       mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1);
       mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 128); mbar_init(&o_full[i], 1);
-      mbar_init(&item_full[i], 1); mbar_init(&item_empty[i], 9);
+      mbar_init(&item_full[i], 1); mbar_init(&item_empty[i], 10);
     }
     fence_mbar_init();
     tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmKwin); tma_prefetch_desc(&tmVwin);
@@ -208,43 +216,70 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   // The control warpgroup (warps 0-3) hands registers to the softmax
   // warpgroups.  All four warps of a warpgroup execute the same setmaxnreg
   // instruction, and each role's code is dominated by its warpgroup's one.
-  // Registers only move inside the CTA: what the four softmax warpgroups take
-  // (2 x 128 x (216 - 168)) must not exceed what the control warpgroup gives up
-  // (128 x (168 - 72)), or setmaxnreg.inc blocks for good.
+  // Registers only move inside the CTA: what the two softmax warpgroups take
+  // (2 x 128 x (208 - 168)) must not exceed what the control warpgroup gives up
+  // (128 x (168 - 88)), or setmaxnreg.inc blocks for good.
   if (warp < 4) {
-  asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
-  if (warp == 0) {
-    // ------------------------------------------------------------ producer
-    // The whole warp runs the loop converged and one elected lane issues the
-    // copies: operands of the TMA / MMA instructions then live in uniform
-    // registers (issuing from a single diverged lane costs ~200 cycles each).
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
+  if (warp == 0 || warp == 2) {
+    // ----------------------------------------------------------- producers
+    // Warp 0 owns K/V stage 0, warp 2 owns stage 1; warp 0 also draws the work
+    // items and loads Q.  A unit whose tiles share K/V takes the stages in turn
+    // (rr_k, rr_v), so each warp issues every other tile; a unit with two K/V
+    // streams gives stage X to tile X, so each warp feeds one stream.  The MMA
+    // warp follows the same rule.  The whole warp runs the loop converged and
+    // one elected lane issues the copies: operands of the TMA / MMA
+    // instructions then live in uniform registers (issuing from a single
+    // diverged lane costs ~200 cycles each).
     const bool leader = elect_one();
-    int q_uses = 0, kt_k = 0, kt_v = 0;
+    const int mine = warp >> 1;                    // the stage this warp fills
+    int q_uses = 0, kfill = 0, vfill = 0, rr_k = 0, rr_v = 0;
     bool ok = true;
-    int tr_n = leader ? 0 : 1 << 30; (void)tr_n;
-    auto load_kv = [&](const ItemU& g, int j, bool isV, int& kt) -> bool {
-      const int st = kt & 1, fill = kt >> 1;
-      uint64_t* full = isV ? &v_full[st] : &k_full[st];
-      uint64_t* empty = isV ? &v_empty[st] : &k_empty[st];
-      uint8_t* dst = (isV ? sV : sK) + st * TILE_BYTES;
-      if (fill > 0 && !warp_wait(empty, (fill - 1) & 1, abortf, LIM)) return false;
-      FB_TR(0, isV ? 2 : 1);
+    int tr_n = (leader && warp == 0) ? 0 : 1 << 30; (void)tr_n;
+    // Page ids of the current request: lane i of pc_cur holds entry 32 * pc_blk + i of its
+    // page-table row, pc_next the following 32 (loaded ahead), so a K/V tile costs two
+    // shuffles instead of two dependent global loads.
+    int pc_blk = 0, pc_cur = 0, pc_next = 0;
+    auto load_pages = [&](int req, int blk) -> int {
+      const int e = blk * 32 + lane;
+      return e < p.max_pages_per_req ? __ldg(&p.page_table[(size_t)req * p.max_pages_per_req + e]) : -1;
+    };
+    // key tile j of the item, K or V of KV head kvh, into this warp's stage
+    auto load_kv = [&](const ItemU& g, int kvh, int j, bool isV) -> bool {
+      const int fill = isV ? vfill : kfill;
+      uint64_t* full = isV ? &v_full[mine] : &k_full[mine];
+      uint64_t* empty = isV ? &v_empty[mine] : &k_empty[mine];
+      uint8_t* dst = (isV ? sV : sK) + mine * TILE_BYTES;
       const int gj = g.jb + j;
-      if (gj < g.npt) {
-        const int npg = (gj * kTileN + kPage < g.prefix_len) ? 2 : 1;
-        int page[2];
+      const bool paged = gj < g.npt;
+      const int npg = (gj * kTileN + kPage < g.prefix_len) ? 2 : 1;
+      int page[2] = {0, 0};
+      if (paged) {
+        // the window of 64 cached entries moves on once V has reached its second half
+        if (isV && ((gj * 2) >> 5) >= pc_blk + 1) {
+          pc_cur = pc_next; ++pc_blk;
+          pc_next = load_pages(g.req, pc_blk + 1);
+        }
 #pragma unroll
         for (int pg = 0; pg < 2; ++pg) {
-          const int pidx = gj * 2 + pg;
-          page[pg] = (pg < npg && pidx < p.max_pages_per_req)
-                         ? __ldg(&p.page_table[(size_t)g.req * p.max_pages_per_req + pidx]) : (pg < npg ? -1 : 0);
+          const int pidx = gj * 2 + pg, blk = pidx >> 5;
+          int v = __shfl_sync(0xffffffffu, blk == pc_blk ? pc_cur : pc_next, pidx & 31);
+          if (blk != pc_blk && blk != pc_blk + 1)                  // outside the window (not expected)
+            v = pidx < p.max_pages_per_req ? __ldg(&p.page_table[(size_t)g.req * p.max_pages_per_req + pidx]) : -1;
+          page[pg] = pg < npg ? v : 0;
+        }
+      }
+      if (fill > 0 && !warp_wait(empty, (fill - 1) & 1, abortf, LIM)) return false;
+      FB_TR(0, isV ? 2 : 1);
+      if (paged) {
+#pragma unroll
+        for (int pg = 0; pg < 2; ++pg) {
           if (page[pg] < 0 || page[pg] >= p.num_pages) { if (leader) atomicOr(p.status, FB_ST_BAD_PAGE); page[pg] = 0; }
-          page[pg] = uni(page[pg]);
         }
         if (leader) {
           mbar_arrive_expect_tx(full, npg * PAGE_BYTES);
           for (int pg = 0; pg < npg; ++pg) {
-            const int y = (page[pg] * p.n_kv_heads + g.kvh) * kPage;
+            const int y = (page[pg] * p.n_kv_heads + kvh) * kPage;
             for (int h = 0; h < NH; ++h)
               tma_load_2d(dst + h * 16384 + pg * 8192, isV ? &tmVpool : &tmKpool, full, h * 64, y);
           }
@@ -253,54 +288,77 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         mbar_arrive_expect_tx(full, TILE_BYTES);
         const int row0 = g.win_row0 + (gj - g.npt) * kTileN;
         for (int h = 0; h < NH; ++h)
-          tma_load_3d(dst + h * 16384, isV ? &tmVwin : &tmKwin, full, h * 64, g.kvh, row0);
+          tma_load_3d(dst + h * 16384, isV ? &tmVwin : &tmKwin, full, h * 64, kvh, row0);
       }
       __syncwarp();
-      ++kt;
+      if (isV) ++vfill; else ++kfill;
       FB_TR(0, isV ? 4 : 3);
       return true;
     };
-    // Work items are handed out longest first through a global ticket; the
-    // producer draws the ticket and publishes the item to the other roles.
+    // Work items are handed out longest first through a global ticket; warp 0
+    // draws the ticket and publishes the item to the other roles.
     for (int k = 0; ok; ++k) {
-      if (k >= 2 && !warp_wait(&item_empty[k & 1], ((k >> 1) - 1) & 1, abortf, LIM)) { ok = false; break; }
       int idx = 0;
-      if (lane == 0) idx = atomicAdd(&p.hdr->ticket, 1);
-      idx = uni(idx);
-      if (idx >= n_items) idx = -1;
-      if (lane == 0) { s_item[k & 1] = idx; mbar_arrive(&item_full[k & 1]); }
-      __syncwarp();
-      if (idx < 0) {
-        // the last CTA to run dry re-arms the ticket for the next launch
-        if (lane == 0 && atomicAdd(&p.hdr->done, 1) == (int)gridDim.x - 1) { p.hdr->ticket = 0; p.hdr->done = 0; }
-        break;
+      if (warp == 0) {
+        if (k >= 2 && !warp_wait(&item_empty[k & 1], ((k >> 1) - 1) & 1, abortf, LIM)) { ok = false; break; }
+        if (lane == 0) idx = atomicAdd(&p.hdr->ticket, 1);
+        idx = uni(idx);
+        if (idx >= n_items) idx = -1;
+        if (lane == 0) { s_item[k & 1] = idx; mbar_arrive(&item_full[k & 1]); }
+        __syncwarp();
+        if (idx < 0) {
+          // the last CTA to run dry re-arms the ticket for the next launch
+          if (lane == 0 && atomicAdd(&p.hdr->done, 1) == (int)gridDim.x - 1) { p.hdr->ticket = 0; p.hdr->done = 0; }
+          break;
+        }
+      } else {
+        if (!warp_wait(&item_full[k & 1], (k >> 1) & 1, abortf, LIM)) { ok = false; break; }
+        idx = s_item[k & 1];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&item_empty[k & 1]);
+        if (idx < 0) break;
       }
       ItemU g;
       if (!load_item_uniform(p, idx, g)) continue;
       FB_TR(0, 10);
-      if (q_uses > 0 && !warp_wait(q_empty, (q_uses - 1) & 1, abortf, LIM)) { ok = false; break; }
-      FB_TR(0, 11);
-      ++q_uses;
-      if (leader) {
-        mbar_arrive_expect_tx(q_full, ((g.nA > 0) + (g.nB > 0)) * TILE_BYTES);
-        if (g.nA > 0)
-          for (int h = 0; h < NH; ++h)
-            tma_load_3d(sQ + h * 16384, &tmQ, q_full, h * 64, g.kvh * p.group, g.rowA);
-        if (g.nB > 0)
-          for (int h = 0; h < NH; ++h)
-            tma_load_3d(sQ + TILE_BYTES + h * 16384, &tmQ, q_full, h * 64, g.kvh * p.group, g.rowB);
+      pc_blk = (g.jb * 2) >> 5;
+      pc_cur = load_pages(g.req, pc_blk);
+      pc_next = load_pages(g.req, pc_blk + 1);
+      if (warp == 0) {
+        if (q_uses > 0 && !warp_wait(q_empty, (q_uses - 1) & 1, abortf, LIM)) { ok = false; break; }
+        FB_TR(0, 11);
+        ++q_uses;
+        if (leader) {
+          mbar_arrive_expect_tx(q_full, ((g.nA > 0) + (g.nB > 0)) * TILE_BYTES);
+          if (g.nA > 0)
+            for (int h = 0; h < NH; ++h)
+              tma_load_3d(sQ + h * 16384, &tmQ, q_full, h * 64, g.kvhA * p.group, g.rowA);
+          if (g.nB > 0)
+            for (int h = 0; h < NH; ++h)
+              tma_load_3d(sQ + TILE_BYTES + h * 16384, &tmQ, q_full, h * 64, g.kvhB * p.group, g.rowB);
+        }
+        __syncwarp();
       }
-      __syncwarp();
-      if (!load_kv(g, 0, false, kt_k)) { ok = false; break; }
-      for (int j = 0; j < g.n; ++j) {
-        if (j + 1 < g.n && !load_kv(g, j + 1, false, kt_k)) { ok = false; break; }
-        if (!load_kv(g, j, true, kt_v)) { ok = false; break; }
+      if (!g.dual()) {
+        // K runs one tile ahead of V; this warp takes the tiles that fall on its stage
+        if ((rr_k++ & 1) == mine && !load_kv(g, g.kvhA, 0, false)) { ok = false; break; }
+        for (int j = 0; j < g.n; ++j) {
+          if (j + 1 < g.n && (rr_k++ & 1) == mine && !load_kv(g, g.kvhA, j + 1, false)) { ok = false; break; }
+          if ((rr_v++ & 1) == mine && !load_kv(g, g.kvhA, j, true)) { ok = false; break; }
+        }
+      } else {
+        const int kvh = mine ? g.kvhB : g.kvhA;
+        if (!load_kv(g, kvh, 0, false)) { ok = false; break; }
+        for (int j = 0; j < g.n; ++j) {
+          if (!load_kv(g, kvh, j, true)) { ok = false; break; }
+          if (j + 1 < g.n && !load_kv(g, kvh, j + 1, false)) { ok = false; break; }
+        }
       }
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------- MMA issuer
     const bool leader = elect_one();
-    int q_cnt = 0, kt = 0, cntPA = 0, cntPB = 0;
+    int q_cnt = 0, cntPA = 0, cntPB = 0;
     bool ok = true;
     int tr_n = leader ? 0 : 1 << 30; (void)tr_n;
     // All descriptors are built once; a k-step only adds a constant to the
@@ -339,6 +397,18 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       __syncwarp();
     };
     auto commit = [&](uint64_t* bar) { if (leader) umma_commit(bar); __syncwarp(); };
+    // fills consumed from each K / V stage (see the producer)
+    int kuse0 = 0, kuse1 = 0, vuse0 = 0, vuse1 = 0, rr_k = 0, rr_v = 0;
+    auto wait_k = [&](int st) -> bool {
+      const int use = st ? kuse1 : kuse0;
+      if (st) ++kuse1; else ++kuse0;
+      return warp_wait(&k_full[st], use & 1, abortf, LIM);
+    };
+    auto wait_v = [&](int st) -> bool {
+      const int use = st ? vuse1 : vuse0;
+      if (st) ++vuse1; else ++vuse0;
+      return warp_wait(&v_full[st], use & 1, abortf, LIM);
+    };
     for (int k = 0; ok; ++k) {
       if (!warp_wait(&item_full[k & 1], (k >> 1) & 1, abortf, LIM)) { ok = false; break; }
       const int idx = s_item[k & 1];
@@ -352,54 +422,109 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       if (!warp_wait(q_full, q_cnt & 1, abortf, LIM)) { ok = false; break; }
       ++q_cnt;
       FB_TR(1, 11);
-      if (!warp_wait(&k_full[kt & 1], (kt >> 1) & 1, abortf, LIM)) { ok = false; break; }
-      FB_TR(1, 12);
-      tc_fence_after();
-      if (nA > 0) issue_qk(0, kt & 1, round16(g.limit(0, g.winA)));
-      if (nB > 0) issue_qk(1, kt & 1, round16(g.limit(0, g.winB)));
-      commit(&k_empty[kt & 1]);
-      if (n == 1) commit(q_empty);               // Q is free once its last QK has run
-      for (int j = 0; j < n; ++j, ++kt) {
-        const int st = kt & 1, st1 = (kt + 1) & 1;
-        FB_TR(1, 20);
-        if (!warp_wait(&v_full[st], (kt >> 1) & 1, abortf, LIM)) { ok = false; break; }
-        // K(j+1) has normally landed by now: taking its barrier here keeps the wait
-        // off the P V -> next Q K^T stretch that the softmax warps are waiting for
-        if (j + 1 < n && !warp_wait(&k_full[st1], ((kt + 1) >> 1) & 1, abortf, LIM)) { ok = false; break; }
-        FB_TR(1, 21);
-        // tile A: O_A += P_A(j) V(j), then S_A(j+1) so that softmax A can go on
-        if (j < nA) {
-          const int nks = round16(g.limit(j, g.winA)) >> 4;
-          if (!warp_wait(&p_full[0], cntPA & 1, abortf, LIM)) { ok = false; break; }
-          FB_TR(1, 23);
-          ++cntPA;
-          tc_fence_after();
-          issue_pv(0, st, 0, nks, j > 0);
-          FB_TR(1, 24);
+      if (!g.dual()) {
+        // ---- tiles A and B share every K/V tile
+        int st = rr_k++ & 1;
+        if (!wait_k(st)) { ok = false; break; }
+        FB_TR(1, 12);
+        tc_fence_after();
+        if (nA > 0) issue_qk(0, st, round16(g.limit(0, g.winA)));
+        if (nB > 0) issue_qk(1, st, round16(g.limit(0, g.winB)));
+        commit(&k_empty[st]);
+        if (n == 1) commit(q_empty);               // Q is free once its last QK has run
+        for (int j = 0; j < n; ++j) {
+          const int sv = rr_v++ & 1;
+          const int st1 = rr_k & 1;                // stage of K(j+1), if there is one
+          FB_TR(1, 20);
+          if (!wait_v(sv)) { ok = false; break; }
+          // K(j+1) has normally landed by now: taking its barrier here keeps the wait
+          // off the P V -> next Q K^T stretch that the softmax warps are waiting for
+          if (j + 1 < n) { ++rr_k; if (!wait_k(st1)) { ok = false; break; } }
+          FB_TR(1, 21);
+          // tile A: O_A += P_A(j) V(j), then S_A(j+1) so that softmax A can go on
+          if (j < nA) {
+            const int nks = round16(g.limit(j, g.winA)) >> 4;
+            if (!warp_wait(&p_full[0], cntPA & 1, abortf, LIM)) { ok = false; break; }
+            FB_TR(1, 23);
+            ++cntPA;
+            tc_fence_after();
+            issue_pv(0, sv, 0, nks, j > 0);
+            FB_TR(1, 24);
+          }
+          if (j + 1 < nA) {
+            FB_TR(1, 25);
+            tc_fence_after();
+            issue_qk(0, st1, round16(g.limit(j + 1, g.winA)));
+            FB_TR(1, 26);
+          }
+          // tile B
+          if (j < nB) {
+            const int nks = round16(g.limit(j, g.winB)) >> 4;
+            if (!warp_wait(&p_full[1], cntPB & 1, abortf, LIM)) { ok = false; break; }
+            FB_TR(1, 33);
+            ++cntPB;
+            tc_fence_after();
+            issue_pv(1, sv, 0, nks, j > 0);
+          }
+          commit(&v_empty[sv]);
+          if (j + 1 < nB) {
+            tc_fence_after();
+            issue_qk(1, st1, round16(g.limit(j + 1, g.winB)));
+          }
+          if (j + 1 < n) {
+            commit(&k_empty[st1]);
+            if (j + 2 == n) commit(q_empty);
+          }
         }
-        if (j + 1 < nA) {
-          FB_TR(1, 25);
+      } else {
+        // ---- one Q tile under two KV heads: stream X owns K stage X and V stage X
+        // (nA == nB == n, and both tiles see the same keys)
+        if (!wait_k(0)) { ok = false; break; }
+        FB_TR(1, 12);
+        tc_fence_after();
+        issue_qk(0, 0, round16(g.limit(0, g.winA)));
+        commit(&k_empty[0]);
+        if (!wait_k(1)) { ok = false; break; }
+        tc_fence_after();
+        issue_qk(1, 1, round16(g.limit(0, g.winB)));
+        commit(&k_empty[1]);
+        if (n == 1) commit(q_empty);
+        // The streams do not depend on each other: serve whichever tile's P is ready.
+        int jA = 0, jB = 0, qk_left = 2 * (n - 1), spins = 0;
+        long long t0 = clock64();
+        while (jA < n || jB < n) {
+          int X = -1;
+          if (jA < n && __all_sync(0xffffffffu, mbar_test(&p_full[0], cntPA & 1))) X = 0;
+          else if (jB < n && __all_sync(0xffffffffu, mbar_test(&p_full[1], cntPB & 1))) X = 1;
+          if (X < 0) {
+            if ((++spins & 63) == 0) {
+              bool give_up = *abortf != 0;
+              if (!give_up && clock64() - t0 > LIM) { *abortf = 1; give_up = true; }
+              if (__any_sync(0xffffffffu, give_up)) { ok = false; break; }
+            }
+            continue;
+          }
+          const int j = X ? jB : jA;
+          if (X) { ++jB; ++cntPB; } else { ++jA; ++cntPA; }
+          FB_TR(1, X ? 33 : 23);
+          if (!wait_v(X)) { ok = false; break; }
+          FB_TR(1, 34);
           tc_fence_after();
-          issue_qk(0, st1, round16(g.limit(j + 1, g.winA)));
-          FB_TR(1, 26);
-        }
-        // tile B
-        if (j < nB) {
-          const int nks = round16(g.limit(j, g.winB)) >> 4;
-          if (!warp_wait(&p_full[1], cntPB & 1, abortf, LIM)) { ok = false; break; }
-          FB_TR(1, 33);
-          ++cntPB;
-          tc_fence_after();
-          issue_pv(1, st, 0, nks, j > 0);
-        }
-        commit(&v_empty[st]);
-        if (j + 1 < nB) {
-          tc_fence_after();
-          issue_qk(1, st1, round16(g.limit(j + 1, g.winB)));
-        }
-        if (j + 1 < n) {
-          commit(&k_empty[st1]);
-          if (j + 2 == n) commit(q_empty);
+          issue_pv(X, X, 0, round16(g.limit(j, g.winA)) >> 4, j > 0);
+          commit(&v_empty[X]);
+          FB_TR(1, 35);
+          if (j + 1 < n) {
+            // this stream's next K tile could only be requested when its last Q K^T had
+            // finished, one softmax ago: give it the time of the P V as well
+            if (!wait_k(X)) { ok = false; break; }
+            FB_TR(1, 36);
+            tc_fence_after();
+            issue_qk(X, X, round16(g.limit(j + 1, g.winA)));
+            commit(&k_empty[X]);
+            if (--qk_left == 0) commit(q_empty);
+          }
+          FB_TR(1, 20);
+          t0 = clock64();
         }
       }
       if (!ok) break;
@@ -410,7 +535,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   } else {
     // ------------------------------------------------- softmax + epilogue
     // Four warps per Q tile, one thread per query row (its TMEM lane).
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
     const int X = (warp - 4) >> 2;                 // 0: tile A, 1: tile B
     const int quad = warp & 3;                     // TMEM lane quadrant of this warp
     const int row = quad * 32 + lane;              // query row of the tile
@@ -543,7 +668,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       if (g.un.n_chunks <= 1) {
         const int slot = X == 0 ? g.un.slotA : g.un.slotB, t0 = X == 0 ? g.un.t0A : g.un.t0B;
         const int grow_ = slot * p.bl + t0 + row / p.group;
-        const int head = g.un.kvh * p.group + row % p.group;
+        const int head = (X == 0 ? g.kvhA : g.kvhB) * p.group + row % p.group;
         uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)grow_ * p.n_q_heads + head) * D);
         const float inv = 1.0f / l;
 #pragma unroll
@@ -647,7 +772,7 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const AttnParams p) {
     }
     const float inv = 1.0f / L;
     const int grow_ = slot * p.bl + t0 + row / p.group;
-    const int head = un.kvh * p.group + row % p.group;
+    const int head = (X == 0 ? (un.kvh & 0xffff) : (un.kvh >> 16)) * p.group + row % p.group;
     __nv_bfloat16* dst = p.out + ((size_t)grow_ * p.n_q_heads + head) * D + lane * PER;
 #pragma unroll
     for (int i = 0; i < PER; i += 2)

@@ -17,10 +17,13 @@ constexpr int kPage = 64;
 constexpr int kDefaultMinChunkTiles = 4;
 constexpr int kDefaultTargetItems = 2 * 148;   // about two work items per SM before key ranges are split
 
-// One unit = one (request, KV head, pair of Q tiles); split along the key
+// One unit = two Q tiles of one request that run side by side in a CTA: either
+// two different tiles under one KV head (they share every K/V tile), or one
+// tile under two adjacent KV heads (two K/V streams).  Split along the key
 // axis into n_chunks items.  16 ints each, read as four int4.
 struct __align__(16) AttnUnit {
-  int32_t req, kvh, slotA, slotB;      // slotB = -1: single tile
+  int32_t req, kvh, slotA, slotB;      // kvh: KV head of tile A | KV head of tile B << 16
+                                       // slotB = -1: single tile
   int32_t t0A, t0B, n_tiles, n_chunks; // n_tiles: key tiles of the request
   int32_t nvisA, nvisB, part_base, prefix_len;
   int32_t npt, win_row0, winA, winB;   // npt prefix tiles; winX = window keys

@@ -72,14 +72,22 @@ __device__ __forceinline__ int item_cost(int nA, int nB) {
   return (6 * n + both + 1) >> 1;
 }
 
+// A request's Q tiles are paired two by two (a pair shares every K/V tile).
+// An odd tile left over is paired with itself across two adjacent KV heads
+// instead: the two halves stream different K/V but keep both tile slots of a
+// CTA busy, which a lone tile cannot.  nunits counts both kinds.
 struct ReqGeom {
   int w, ntq, npairs, P, npt, nt;
+  int nfull, odd, nunits;   // full pairs per KV head; leftover tile; units of the request
 };
 __device__ __forceinline__ ReqGeom req_geom(const PackParams& p, int r, int32_t* status) {
   ReqGeom g;
   g.w = live_blocks(p, r, status);
   g.ntq = g.w * p.tiles_per_slot;
   g.npairs = (g.ntq + 1) >> 1;
+  g.nfull = g.ntq >> 1;
+  g.odd = g.ntq & 1;
+  g.nunits = g.nfull * p.n_kv_heads + g.odd * ((p.n_kv_heads + 1) >> 1);
   g.P = g.w ? max(p.prefix_len[r], 0) : 0;
   g.npt = (g.P + kTileN - 1) / kTileN;
   g.nt = g.w ? g.npt + (g.w * p.bl + kTileN - 1) / kTileN : 0;
@@ -97,7 +105,7 @@ __device__ void build_sched(const PackParams& p) {
   int mine = 0;
   for (int r = tid; r < p.max_requests; r += kPackThreads) {
     ReqGeom g = req_geom(p, r, nullptr);
-    mine += g.npairs * p.n_kv_heads * g.nt;
+    mine += g.nunits * g.nt;
   }
   if (tid == 0) sh_total = 0;
   for (int i = tid; i < kCostBins; i += kPackThreads) bins[i] = 0;
@@ -121,7 +129,7 @@ __device__ void build_sched(const PackParams& p) {
     if (r < p.max_requests) {
       g = req_geom(p, r, nullptr);
       nch = g.nt ? (g.nt + Ct - 1) / Ct : 0;
-      nunits = g.npairs * p.n_kv_heads;
+      nunits = g.nunits;
     }
     int tu, tp, ti, ts;
     const int ubase = unit_run + block_excl_scan(nunits, &tu, sh_scan);
@@ -130,40 +138,48 @@ __device__ void build_sched(const PackParams& p) {
     const int first = slot_run + block_excl_scan(g.w, &ts, sh_scan);  // first slot of the request
     unit_run += tu; part_run += tp; item_run += ti; slot_run += ts;
     if (r < p.max_requests && nunits) {
-      for (int pr = 0; pr < g.npairs; ++pr)
-        for (int h = 0; h < p.n_kv_heads; ++h) {
-          // the Q-tile pairs of one (request, KV head) get adjacent unit numbers: they stream the
-          // same K/V, are handed out back to back and so share it through L2
-          const int u = ubase + h * g.npairs + pr;
-          if (u >= p.max_units) continue;
-          const int qa = 2 * pr, qb = 2 * pr + 1;
-          AttnUnit un;
-          un.req = r; un.kvh = h;
-          const int sA = qa / p.tiles_per_slot;
-          un.slotA = first + sA;
-          un.t0A = (qa % p.tiles_per_slot) * p.tokens_per_tile;
-          un.winA = (sA + 1) * p.bl;
-          un.nvisA = g.npt + (un.winA + kTileN - 1) / kTileN;
-          if (qb < g.ntq) {
-            const int sB = qb / p.tiles_per_slot;
-            un.slotB = first + sB;
-            un.t0B = (qb % p.tiles_per_slot) * p.tokens_per_tile;
-            un.winB = (sB + 1) * p.bl;
-            un.nvisB = g.npt + (un.winB + kTileN - 1) / kTileN;
-          } else {
-            un.slotB = -1; un.t0B = 0; un.winB = 0; un.nvisB = 0;
-          }
-          un.n_tiles = g.nt; un.n_chunks = nch;
-          un.part_base = nch > 1 ? pbase + (h * g.npairs + pr) * nch : -1;
-          if (nch > 1 && un.part_base + nch > p.max_parts) un.n_chunks = 0;  // cannot happen; see header
-          un.prefix_len = g.P; un.npt = g.npt; un.win_row0 = first * p.bl;
-          p.units[u] = un;
-          for (int c = 0; c < un.n_chunks; ++c) {
-            const int jb = c * g.nt / nch, je = (c + 1) * g.nt / nch;
-            int cost = item_cost(max(0, min(je, un.nvisA) - jb), max(0, min(je, un.nvisB) - jb));
-            atomicAdd(&bins[min(cost, kCostBins - 1)], 1);
-          }
+      for (int ul = 0; ul < g.nunits; ++ul) {
+        // Full pairs first, numbered h * nfull + pr: the pairs of one (request, KV head) are
+        // adjacent, are handed out back to back and so share their K/V through L2.  Then the
+        // leftover tile, one unit per two KV heads.
+        const int u = ubase + ul;
+        if (u >= p.max_units) continue;
+        const bool full = ul < g.nfull * p.n_kv_heads;
+        const int h = full ? ul / g.nfull : 2 * (ul - g.nfull * p.n_kv_heads);
+        const int qa = full ? 2 * (ul % g.nfull) : g.ntq - 1;
+        AttnUnit un;
+        un.req = r;
+        const int sA = qa / p.tiles_per_slot;
+        un.slotA = first + sA;
+        un.t0A = (qa % p.tiles_per_slot) * p.tokens_per_tile;
+        un.winA = (sA + 1) * p.bl;
+        un.nvisA = g.npt + (un.winA + kTileN - 1) / kTileN;
+        if (full) {
+          const int qb = qa + 1;
+          const int sB = qb / p.tiles_per_slot;
+          un.kvh = h | (h << 16);
+          un.slotB = first + sB;
+          un.t0B = (qb % p.tiles_per_slot) * p.tokens_per_tile;
+          un.winB = (sB + 1) * p.bl;
+          un.nvisB = g.npt + (un.winB + kTileN - 1) / kTileN;
+        } else if (h + 1 < p.n_kv_heads) {
+          un.kvh = h | ((h + 1) << 16);
+          un.slotB = un.slotA; un.t0B = un.t0A; un.winB = un.winA; un.nvisB = un.nvisA;
+        } else {
+          un.kvh = h | (h << 16);
+          un.slotB = -1; un.t0B = 0; un.winB = 0; un.nvisB = 0;
         }
+        un.n_tiles = g.nt; un.n_chunks = nch;
+        un.part_base = nch > 1 ? pbase + ul * nch : -1;
+        if (nch > 1 && un.part_base + nch > p.max_parts) un.n_chunks = 0;  // cannot happen; see header
+        un.prefix_len = g.P; un.npt = g.npt; un.win_row0 = first * p.bl;
+        p.units[u] = un;
+        for (int c = 0; c < un.n_chunks; ++c) {
+          const int jb = c * g.nt / nch, je = (c + 1) * g.nt / nch;
+          int cost = item_cost(max(0, min(je, un.nvisA) - jb), max(0, min(je, un.nvisB) - jb));
+          atomicAdd(&bins[min(cost, kCostBins - 1)], 1);
+        }
+      }
     }
   }
   __syncthreads();
