@@ -720,19 +720,22 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem, 512); }
 }
 
-// Merge of the split-KV partials, chunks in index order.  Eight CTAs per unit,
-// 32 of its 256 rows each; a warp takes one row at a time and keeps the loads
-// of four chunks in flight.
+// Merge of the split-KV partials, chunks in index order.  A unit is cut into
+// eight pieces of 32 of its 256 rows; the CTAs of a fixed-size grid loop over
+// the pieces (nothing to do, and an immediate return, when no unit was split).
+// A warp takes one row at a time and keeps the loads of four chunks in flight.
 constexpr int kCombineSplit = 8;
+constexpr int kCombineCtasPerSm = 4;
 template <int D>
 __global__ void __launch_bounds__(256) attn_combine_kernel(const AttnParams p) {
-  const int u = blockIdx.x / kCombineSplit;
-  if (u >= p.hdr->n_units) return;
-  const AttnUnit un = p.units[u];
-  if (un.n_chunks <= 1) return;
+  if (p.hdr->n_parts == 0) return;
+  const int n_pieces = p.hdr->n_units * kCombineSplit;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr int PER = D / 32;
-  const int row0 = (blockIdx.x % kCombineSplit) * (2 * kTileM / kCombineSplit);
+  for (int piece = blockIdx.x; piece < n_pieces; piece += gridDim.x) {
+  const AttnUnit un = p.units[piece / kCombineSplit];
+  if (un.n_chunks <= 1) continue;
+  const int row0 = (piece % kCombineSplit) * (2 * kTileM / kCombineSplit);
   for (int rr = row0 + warp; rr < row0 + 2 * kTileM / kCombineSplit; rr += 8) {
     const int X = rr / kTileM, row = rr % kTileM;
     const int slot = X == 0 ? un.slotA : un.slotB;
@@ -777,6 +780,7 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const AttnParams p) {
 #pragma unroll
     for (int i = 0; i < PER; i += 2)
       *reinterpret_cast<uint32_t*>(dst + i) = pack_bf16x2(acc[i] * inv, acc[i + 1] * inv);
+  }
   }
 }
 
@@ -880,16 +884,17 @@ int launch_attn(fb_ctx* ctx, const fb_pack* pk, const void* q, const void* k_win
   p.wait_cycles = 2000000000LL;
   if (const char* e = getenv("FB_WAIT_CYCLES")) { long long v = atoll(e); if (v > 0) p.wait_cycles = v; }
   const int grid = ctx->num_sms;
+  const int combine_grid = min(ctx->ws.max_units * kCombineSplit, kCombineCtasPerSm * ctx->num_sms);
   if (c.head_dim == 64) {
     wavefront_attn_kernel<64><<<grid, kAttnThreads, kSmem64, stream>>>(
         ctx->tm_q, ctx->tm_kwin, ctx->tm_vwin, ctx->tm_kpool, ctx->tm_vpool, p);
     if (int e = cuda_err(ctx, cudaGetLastError(), "wavefront_attn_kernel launch")) return e;
-    attn_combine_kernel<64><<<ctx->ws.max_units * kCombineSplit, 256, 0, stream>>>(p);
+    attn_combine_kernel<64><<<combine_grid, 256, 0, stream>>>(p);
   } else {
     wavefront_attn_kernel<128><<<grid, kAttnThreads, kSmem128, stream>>>(
         ctx->tm_q, ctx->tm_kwin, ctx->tm_vwin, ctx->tm_kpool, ctx->tm_vpool, p);
     if (int e = cuda_err(ctx, cudaGetLastError(), "wavefront_attn_kernel launch")) return e;
-    attn_combine_kernel<128><<<ctx->ws.max_units * kCombineSplit, 256, 0, stream>>>(p);
+    attn_combine_kernel<128><<<combine_grid, 256, 0, stream>>>(p);
   }
   return cuda_err(ctx, cudaGetLastError(), "attn_combine_kernel launch");
 }
