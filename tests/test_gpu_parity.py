@@ -305,6 +305,63 @@ def test_attention_isolation_from_invisible_memory():
     assert again == base
 
 
+def _amplify_keys(case, where, factor):
+    """Returns attention inputs in which the keys of one stretch of every
+    request's context are `factor` times larger, so that the running softmax
+    reference has to move there: by a few powers of two (factor 6) or by far
+    more than fp32's exponent range could absorb without re-basing (factor 40).
+    V is halved so that near-one-hot outputs round to bf16 within the tolerance."""
+    stc = case["stc"]
+    wl = stc.wl
+    b = wl.block_len
+    q, kw, vw, kp, vp = (t.clone() for t in case["attn"])
+    vw = (vw.float() * 0.5).to(torch.bfloat16)
+    vp = (vp.float() * 0.5).to(torch.bfloat16)
+    pk = O.pack_wavefronts(H.oracle_cfg(stc), H.oracle_state(stc, case["tokens"]))
+    for r in range(wl.n_requests):
+        if stc.active[r] != 1:
+            continue
+        P = int(stc.prefix_len[r])
+        if where == "first_tile":
+            lo, hi = 0, min(P, 100)
+        elif where == "second_tile":
+            lo, hi = min(P, 130), min(P, 250)
+        elif where == "prefix_tail":
+            lo, hi = max(P - 37, 0), P
+        else:
+            lo = hi = 0
+        for pos in range(lo, hi):
+            pg = int(stc.page_table[r, pos // 64])
+            kp[pg, :, pos % 64] = (kp[pg, :, pos % 64].float() * factor).to(torch.bfloat16)
+        if where == "window_last_block":
+            s_last = int(pk.req_slot_begin[r + 1]) - 1
+            rows = slice(s_last * b, (s_last + 1) * b)
+            kw[rows] = (kw[rows].float() * factor).to(torch.bfloat16)
+        if where == "window_first_block":
+            s0 = int(pk.req_slot_begin[r])
+            rows = slice(s0 * b, (s0 + 1) * b)
+            kw[rows] = (kw[rows].float() * factor).to(torch.bfloat16)
+    return q, kw, vw, kp, vp
+
+
+@pytest.mark.parametrize("factor", [6.0, 40.0])
+@pytest.mark.parametrize("where", ["first_tile", "second_tile", "prefix_tail",
+                                   "window_first_block", "window_last_block"])
+@pytest.mark.parametrize("target", [296, 100000])
+def test_attention_when_the_softmax_reference_moves(where, factor, target, monkeypatch):
+    """Scores that jump far above (or start far above and fall far below) what
+    earlier key tiles held: the lazily re-based reference, the rescaling of the
+    accumulated output and the redo of the tile must agree with the plain
+    softmax of the oracle, with and without a key-axis split."""
+    monkeypatch.setenv("FB_ATTN_TARGET_ITEMS", str(target))
+    wl = synth.tiny_workload(prefix_lo=300, prefix_hi=900, n_requests=5, wmax=4,
+                             w_lo=1, w_hi=4, head_dim=128, n_q_heads=8, n_kv_heads=2,
+                             max_blocks=16)
+    case = make_case(wl, with_logits=False)
+    case = dict(case, attn=_amplify_keys(case, where, factor))
+    run_attention(case)
+
+
 # --------------------------------------------------- multi-step state machine
 def test_multi_step_trajectory_matches_oracle():
     """Eight consecutive steps (pack -> attention -> T2T -> gate/commit) with
