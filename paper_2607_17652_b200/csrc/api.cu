@@ -23,8 +23,9 @@ fb::WsLayout make_layout(const fb_config& c, int tiles_per_slot, int target_item
   fb::WsLayout w{};
   const long long qtiles = (long long)c.max_requests * c.wmax * tiles_per_slot;
   w.max_units = (int)((qtiles + c.max_requests + 1) / 2) * c.n_kv_heads;
-  w.max_items = w.max_units + target_items + 8;
-  w.max_parts = 2 * target_items + 8;
+  // split units: at most 2 x target pieces from the coarse split, 1.2 x target more from the filler
+  w.max_items = w.max_units + 3 * target_items + 8;
+  w.max_parts = 4 * target_items + 8;
   size_t off = 0;
   w.header = off;  off = align_up(off + sizeof(fb::SchedHeader), 256);
   w.items = off;   off = align_up(off + (size_t)w.max_items * sizeof(fb::AttnItem), 256);

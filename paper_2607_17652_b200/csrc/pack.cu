@@ -76,6 +76,14 @@ __device__ __forceinline__ int item_cost(int nA, int nB) {
 // An odd tile left over is paired with itself across two adjacent KV heads
 // instead: the two halves stream different K/V but keep both tile slots of a
 // CTA busy, which a lone tile cannot.  nunits counts both kinds.
+#ifndef FB_FILL_PCT
+#define FB_FILL_PCT 15
+#endif
+#ifndef FB_FILL_DIV
+#define FB_FILL_DIV 8
+#endif
+constexpr int kFillerPercent = FB_FILL_PCT;   // share of the key-tile work cut into filler pieces
+constexpr int kFillerDiv = FB_FILL_DIV;       // a filler piece is 1/kFillerDiv of a CTA's share
 struct ReqGeom {
   int w, ntq, npairs, P, npt, nt;
   int nfull, odd, nunits;   // full pairs per KV head; leftover tile; units of the request
@@ -97,41 +105,56 @@ __device__ __forceinline__ ReqGeom req_geom(const PackParams& p, int r, int32_t*
 __device__ void build_sched(const PackParams& p) {
   __shared__ int sh_scan[kPackThreads / 32 + 1];
   __shared__ int bins[kCostBins];
-  __shared__ int sh_total;
-  __shared__ int sh_ct;
+  __shared__ int sh_total, sh_units;
+  __shared__ int sh_ct, sh_fine_ct, sh_fine_from;
   const int tid = threadIdx.x;
   // bad states are reported once, by the gather blocks (null status here)
   // phase 1: total key-tile work -> chunk length
-  int mine = 0;
+  int mine = 0, mine_units = 0;
   for (int r = tid; r < p.max_requests; r += kPackThreads) {
     ReqGeom g = req_geom(p, r, nullptr);
     mine += g.nunits * g.nt;
+    mine_units += g.nt ? g.nunits : 0;
   }
-  if (tid == 0) sh_total = 0;
+  if (tid == 0) { sh_total = 0; sh_units = 0; }
   for (int i = tid; i < kCostBins; i += kPackThreads) bins[i] = 0;
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
+  for (int o = 16; o > 0; o >>= 1) {
+    mine += __shfl_xor_sync(0xffffffffu, mine, o);
+    mine_units += __shfl_xor_sync(0xffffffffu, mine_units, o);
+  }
   __syncthreads();
-  if ((tid & 31) == 0) atomicAdd(&sh_total, mine);
+  if ((tid & 31) == 0) { atomicAdd(&sh_total, mine); atomicAdd(&sh_units, mine_units); }
   __syncthreads();
   if (tid == 0) {
     const int ct = (sh_total + p.target_items - 1) / p.target_items;
     sh_ct = ct < p.min_chunk_tiles ? p.min_chunk_tiles : ct;
+    // Filler: items are handed out longest first, so the CTAs run dry within one shortest
+    // item of each other.  When even the short items are long (few, long requests), the
+    // units of the last requests -- about 15 % of the work -- are cut into pieces of 1/8 of
+    // a CTA's share (target_items = two items per CTA), which level that tail.
+    const int share = (int)(2ll * sh_total / p.target_items);
+    const int fine = max(p.min_chunk_tiles, share / kFillerDiv);
+    const bool on = sh_units > 0 && sh_total / sh_units > 2 * fine && fine < sh_ct;
+    sh_fine_ct = fine;
+    sh_fine_from = on ? sh_total - (int)((long long)kFillerPercent * sh_total / 100) : 0x7fffffff;
   }
   __syncthreads();
-  const int Ct = sh_ct;
+  const int Ct = sh_ct, fineCt = sh_fine_ct, fineFrom = sh_fine_from;
   // phase 2 + 3: per-request bases (chunked scan), units, cost histogram
-  int unit_run = 0, part_run = 0, item_run = 0, slot_run = 0;
+  int unit_run = 0, part_run = 0, item_run = 0, slot_run = 0, work_run = 0;
   for (int r0 = 0; r0 < p.max_requests; r0 += kPackThreads) {
     const int r = r0 + tid;
     ReqGeom g{};
     int nch = 0, nunits = 0;
     if (r < p.max_requests) {
       g = req_geom(p, r, nullptr);
-      nch = g.nt ? (g.nt + Ct - 1) / Ct : 0;
       nunits = g.nunits;
     }
-    int tu, tp, ti, ts;
+    int tu, tp, ti, ts, tw;
+    const int wbase = work_run + block_excl_scan(nunits * g.nt, &tw, sh_scan);
+    work_run += tw;
+    if (g.nt) nch = (g.nt + (wbase + nunits * g.nt > fineFrom ? fineCt : Ct) - 1) / (wbase + nunits * g.nt > fineFrom ? fineCt : Ct);
     const int ubase = unit_run + block_excl_scan(nunits, &tu, sh_scan);
     const int pbase = part_run + block_excl_scan(nch > 1 ? nunits * nch : 0, &tp, sh_scan);
     block_excl_scan(nunits * nch, &ti, sh_scan);
