@@ -354,6 +354,97 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------ serving sweep
+def run_sweep(args):
+    """`--sweep`: the serving workload as a sequence -- requests arrive over the
+    first 24 steps, confidences rise by 0.05 per step, blocks reveal, commit and
+    spawn (48 steps by default).  One untimed pass, then the timed one; every
+    step's four calls are bracketed by CUDA events, logits patching (it stands
+    in for the LM head) stays outside.  Reports steps/s and committed tokens/s
+    beside the usual fields; the rows that are live come from the device state
+    read back before each step."""
+    import dataclasses
+    import torch
+    from paper_2607_17652_b200 import binding as B, sweep, synth
+    B.lib()                                     # fails loudly when the CUDA library is missing
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    wl = synth.WORKLOADS[args.workload]
+    if args.requests:
+        wl = dataclasses.replace(wl, n_requests=args.requests)
+    n_steps = args.steps if args.steps != 20 else 48
+    inp = sweep.SweepInputs(wl, n_steps=n_steps)
+    run = sweep.SweepRunner(inp, dev)
+
+    def one_pass(timed):
+        seg, flops, live, committed = [], [], [], 0
+        for step in range(n_steps):
+            for r in inp.arrivals(step):
+                run.arrive(r)
+            active, plen, L, R = run.host_state()
+            rows, cols, vals, _ = inp.begin_step(step, active, L, R)
+            inp.apply(run.z, rows, cols, vals)
+            cur = dataclasses.replace(inp.stc)
+            cur.active, cur.prefix_len, cur.L, cur.R = active, plen, L, R
+            t = run.step()
+            if timed:
+                seg.append(t)
+                flops.append(attn_flops(cur))
+                live.append(len(rows) // wl.block_len)
+                committed += int(run.sb.n_committed.sum().item()) * wl.block_len
+        return np.array(seg), np.array(flops), np.array(live), committed
+
+    one_pass(False)
+    run.reset()
+    uuid = str(torch.cuda.get_device_properties(0).uuid)
+    sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+    sampler.start()
+    time.sleep(0.2)
+    t0 = time.time()
+    seg, flops, live, committed = one_pass(True)
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    clocks["window"] = "the timed pass of the sweep (device time is a fraction of it: inputs are patched between steps)"
+    status = int(run.sb.status.item())
+    total_ms = float(seg.sum())
+    peaks = load_peaks()
+    attn_ms, t2t_ms = float(seg[:, 1].sum()), float(seg[:, 2].sum())
+    attn_tf = float(flops.sum()) / attn_ms / 1e9
+    t2t_b = float(sum(l * wl.block_len * (2.0 * wl.vocab + 13) + l * 24 for l in live))
+    t2t_gbs = t2t_b / t2t_ms / 1e6
+    line = {
+        "metric": METRIC, "value": round(float(flops.sum()) / total_ms / 1e9, 3),
+        "unit": "TFLOP/s (attention FLOPs / whole-step time)",
+        "n_gpus": 1, "steps": n_steps, "warmup": n_steps, "ms_per_step": round(total_ms / n_steps, 4),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": wl.name + " (sweep)", "requests": wl.n_requests, "block_len": wl.block_len,
+                   "wmax": wl.wmax, "slots": wl.max_slots, "live_slots": float(live.mean()),
+                   "q_heads": wl.n_q_heads, "kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim,
+                   "vocab": wl.vocab, "prefix_range": [wl.prefix_lo, wl.prefix_hi],
+                   "logits": "noise bank, one winner per live row patched per step", "parallelism": "replicas x1",
+                   "l2": "inputs larger than L2 (logits + KV pools >> 126 MB); no flush"},
+        "sweep": {"steps_per_s": round(n_steps / total_ms * 1e3, 1),
+                  "committed_tokens_per_s": round(committed / total_ms * 1e3, 1),
+                  "committed_tokens": committed, "live_slots_first_last": [int(live[0]), int(live[-1])],
+                  "device_ms_total": round(total_ms, 3)},
+        "clocks": clocks,
+        "e2e": {"value": None, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+                "note": "the sweep is timed with resident inputs only; see the default run for host buffers"},
+        "gpu_launches": KERNELS_PER_STEP * n_steps,
+        "kernels": {"pack_ms": round(float(seg[:, 0].mean()), 4), "attn_ms": round(attn_ms / n_steps, 4),
+                    "t2t_ms": round(t2t_ms / n_steps, 4), "gate_commit_ms": round(float(seg[:, 3].mean()), 4),
+                    "attn_tflops": round(attn_tf, 2), "t2t_gbs": round(t2t_gbs, 1)},
+        "roofline": {"bound": "tensor", "achieved": round(attn_tf, 2), "peak": peaks["bf16_tflops"],
+                     "unit": "TFLOP/s", "frac": round(attn_tf / peaks["bf16_tflops"], 4), "traffic": None,
+                     "kernel": "wavefront_attn_kernel(+combine)",
+                     "peak_source": peaks["source"] + " cuBLAS bf16 burst"},
+        "roofline_t2t": {"bound": "hbm", "achieved": round(t2t_gbs, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": round(t2t_gbs / peaks["hbm_gbs"], 4), "traffic": None},
+        "device_status": status,
+    }
+    print(json.dumps(line), flush=True)
+
+
 # ------------------------------------------------------- the oracle, timed
 def oracle_sample_step(wl, stc, tokens, z_live, attn, n_req):
     """One oracle step (pack, attention, T2T, gate/commit) on the first n_req
@@ -447,10 +538,14 @@ def main():
                     help="time one call only (profiler captures); the JSON line then has no step metric")
     ap.add_argument("--cpu-budget", type=float, default=12.0)
     ap.add_argument("--ref-requests", type=int, default=2)
+    ap.add_argument("--sweep", action="store_true",
+                    help="run the serving workload as a 48-step sequence with arrivals (use with --workload 4)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.sweep:
+        run_sweep(args)
     else:
         run_ours(args)
 

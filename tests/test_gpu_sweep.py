@@ -1,0 +1,102 @@
+"""Serving sweep on the GPU against the oracle, state by state: 128 requests
+arriving over 24 steps, 48 steps in all, confidences rising by 0.05 per step
+(the serving workload's structure: 512 slots, 64 blocks per request, prefixes of
+512-4096 tokens; the vocabulary is cut to 4096 so that the oracle's own row
+pass over every live row stays affordable).  After every step the tokens, the
+window bounds, the prefix lengths, the per-step outputs and the frozen K/V of
+the blocks that retired are compared; commits and admissions of one step feed
+the next one on both sides."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import flowblock_oracle as O
+from paper_2607_17652_b200 import sweep, synth
+from tests import harness as H
+
+pytestmark = pytest.mark.gpu
+CONF_TOL = 2e-5
+
+
+def _frozen_kv_matches(run, opk, ost_before, ncom, b):
+    """Pool rows [P_old, P_old + c*bl) of every request that retired c blocks
+    equal the window K/V rows of those blocks, byte for byte (Eq. 6)."""
+    kp, vp, kw, vw = run.kp, run.vp, run.kw, run.vw
+    pt = ost_before.page_table
+    for r in np.flatnonzero(ncom > 0):
+        P0 = int(ost_before.prefix_len[r])
+        slot0 = int(opk.req_slot_begin[r])
+        n = int(ncom[r]) * b
+        pos = np.arange(P0, P0 + n)
+        pages = torch.from_numpy(pt[r, pos // 64].astype(np.int64)).to(kp.device)
+        offs = torch.from_numpy((pos % 64).astype(np.int64)).to(kp.device)
+        rows = torch.arange(slot0 * b, slot0 * b + n, device=kp.device)
+        if not (torch.equal(kp[pages, :, offs], kw[rows]) and torch.equal(vp[pages, :, offs], vw[rows])):
+            return False
+    return True
+
+
+def test_serving_sweep_states_match_oracle_every_step():
+    wl = dataclasses.replace(synth.WORKLOADS[4], vocab=4096)
+    n_steps = 48
+    # EOS winners from the third block on, so that some requests terminate within the 48 steps
+    inp = sweep.SweepInputs(wl, n_steps=n_steps, eos_min_block=2)
+    run = sweep.SweepRunner(inp)
+    stc = inp.stc
+    b = wl.block_len
+    ocfg = H.oracle_cfg(stc)
+    ost = H.oracle_state(stc, inp.tokens0())
+    n_rows = wl.max_slots * b
+    commits = spawns = edits = 0
+    for step in range(n_steps):
+        for r in inp.arrivals(step):                      # the caller writes the state row
+            ost.active[r] = 1
+            run.arrive(r)
+        rows, cols, vals, conf = inp.begin_step(step, ost.active, ost.L, ost.R)
+        inp.apply(run.z, rows, cols, vals)
+        run.step()
+        sb = run.sb
+        assert int(sb.status.item()) == 0
+        opk = O.pack_wavefronts(ocfg, ost)
+        g = run.pk.to_numpy()
+        assert int(g["n_live"][0]) == opk.n_live == len(rows) // b
+        for name in ("slot_req", "slot_s", "slot_pos0", "slot_kv_len", "slot_flags", "req_slot_begin",
+                     "qtok", "pos"):
+            np.testing.assert_array_equal(g[name], getattr(opk, name), err_msg=f"{name}@{step}")
+        if step in (0, 7, 23, 47):
+            # the plain row pass of the oracle on the patched logits pins the declared
+            # winners and confidences
+            z64 = H.f64(run.z[:len(rows)].cpu())
+            full = np.zeros((n_rows, wl.vocab))
+            full[:len(rows)] = z64
+            xo, co = O.t2t_rows(ocfg, opk, full)
+            np.testing.assert_array_equal(xo[:len(rows)], cols)
+            assert np.abs(co[:len(rows)] - conf).max() < 1e-12
+        xhat = np.full(n_rows, -1, np.int32)
+        cf = np.zeros(n_rows)
+        xhat[rows] = cols
+        cf[rows] = conf
+        before = dataclasses.replace(ost, prefix_len=ost.prefix_len.copy())
+        action, stats = O.t2t_update(ocfg, opk, ost, xhat, cf)
+        ncom, spawned, ctr = O.gate_commit(ocfg, opk, stats, ost)
+        live = slice(0, len(rows))
+        np.testing.assert_array_equal(sb.argmax.cpu().numpy()[live], xhat[live])
+        assert np.abs(sb.conf.cpu().numpy()[live].astype(np.float64) - cf[live]).max() <= CONF_TOL
+        np.testing.assert_array_equal(sb.action.cpu().numpy(), action)
+        np.testing.assert_array_equal(sb.slot_stats.cpu().numpy()[:opk.n_live], stats[:opk.n_live])
+        np.testing.assert_array_equal(sb.n_committed.cpu().numpy(), ncom)
+        np.testing.assert_array_equal(sb.spawned.cpu().numpy(), spawned)
+        np.testing.assert_array_equal(sb.step_counters.cpu().numpy(), ctr)
+        gs = run.st.to_numpy()
+        for name in ("active", "prefix_len", "L", "R", "tokens", "pe_done"):
+            np.testing.assert_array_equal(gs[name], getattr(ost, name), err_msg=f"{name}@{step}")
+        assert _frozen_kv_matches(run, opk, before, ncom, b), f"frozen K/V @ {step}"
+        commits += int(ncom.sum())
+        spawns += int(spawned.sum())
+        edits += int((action == O.ACT_T2T).sum())
+    assert (ost.active != 0).all(), "every request has arrived"
+    assert commits >= 2 * wl.n_requests and spawns >= commits
+    assert edits > 0, "the re-drawn winners never produced a T2T edit"
+    assert (ost.active == 2).any(), "no request reached a committed EOS"
