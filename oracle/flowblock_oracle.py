@@ -27,6 +27,12 @@ Pins (tests/test_oracle_*.py, all CPU):
   gate_commit            hand-worked Alg. 1 cases; window of one block equals
                          an independently written serial block-wise decoder;
                          packed run equals per-request runs
+  scatter_window_kv      brute-force placement (every live window position, no
+                         other pool element); attention over the page-resident
+                         window equals attention over the slot-order window;
+                         pointer-bump commit equals copy-at-commit
+  rope_rotate            textbook special cases (position 0, d = 2 rotation,
+                         norm, relative-offset invariance of q.k)
 Nothing in this file is "parity unpinned".
 
 Readings of the paper taken where it is silent or ambiguous are the named
@@ -181,16 +187,18 @@ def visible_keys(cfg: Config, pk: Pack, slot: int, k_win, k_pool, page_table):
     the request's committed prefix [0, o_r) read through its page table, then
     window blocks L..g of the same request (g = the slot's own block), every
     token of each -- bidirectional inside a block, nothing to the right.
+    With ``k_win`` None the window is resident in the pages as well (it was
+    scattered there, Eq. 6) and every key is read through the page table.
     Returns [kv_len, Hkv, d]."""
     b, ps = cfg.block_len, cfg.page_size
     r, s = int(pk.slot_req[slot]), int(pk.slot_s[slot])
     first = int(pk.req_slot_begin[r])
     P = int(pk.slot_pos0[slot]) - s * b
     rows = []
-    for j in range(P):
+    for j in range(P if k_win is not None else P + (s + 1) * b):
         page = int(page_table[r, j // ps])
         rows.append(k_pool[page, :, j % ps, :])
-    for s2 in range(s + 1):
+    for s2 in range(s + 1 if k_win is not None else 0):
         for t in range(b):
             rows.append(k_win[(first + s2) * b + t])
     return np.stack(rows, axis=0)
@@ -262,6 +270,49 @@ def dense_mask_attn_bruteforce(cfg: Config, st_prefix_len, st_wlive, q_req,
             Pm = Pm / Pm.sum(axis=1, keepdims=True)
             out[bi, :, h, :] = Pm @ v_phys[bi, :, h // G, :]
     return out
+
+
+# --------------------------------------------------------------------------
+# next: Eq. 6 as data movement -- the window resident in the pages
+# --------------------------------------------------------------------------
+def rope_rotate(x, pos, base: float):
+    """Rotary position embedding of one vector (last axis = head dim d) at
+    absolute position ``pos``: pair (x_i, x_{i+d/2}), i < d/2, is rotated by the
+    angle pos * base^(-2i/d).
+
+    READING: the paper only says that the gathered window carries "absolute
+    position ids for RoPE" (Sec. 3.2); the pairing (rotate-half) and the base
+    are the model's, taken here as parameters."""
+    d = x.shape[-1]
+    i = np.arange(d // 2, dtype=np.float64)
+    ang = float(pos) * np.power(float(base), -2.0 * i / d)
+    c, s = np.cos(ang), np.sin(ang)
+    lo, hi = x[..., :d // 2], x[..., d // 2:]
+    return np.concatenate([lo * c - hi * s, hi * c + lo * s], axis=-1)
+
+
+def scatter_window_kv(cfg: Config, pk: Pack, k_new, v_new, k_pool, v_pool,
+                      page_table, rope_base: float = 0.0):
+    """Eq. 6 as data movement: the fresh K/V of every live window position go
+    to the request's pages at their absolute positions, cache[r, o_r + s*bl +
+    t] = k_new[slot, t], every step; in place on the pools.
+
+    k_new, v_new [S*bl, Hkv, d] in slot order.  With ``rope_base`` > 0 the keys
+    are rotated by their absolute position first (rope_rotate); V never is.
+    The frozen prefix [0, o_r) and every position right of the window are not
+    touched.  Retirement then needs no copy: advancing o_r freezes what is
+    already in place."""
+    b, ps = cfg.block_len, cfg.page_size
+    for slot in range(pk.n_live):
+        r = int(pk.slot_req[slot])
+        for t in range(b):
+            pos = int(pk.slot_pos0[slot]) + t
+            page = int(page_table[r, pos // ps])
+            k = k_new[slot * b + t]
+            if rope_base > 0.0:
+                k = rope_rotate(k, pos, rope_base)
+            k_pool[page, :, pos % ps, :] = k
+            v_pool[page, :, pos % ps, :] = v_new[slot * b + t]
 
 
 # --------------------------------------------------------------------------
