@@ -92,6 +92,12 @@ typedef struct {
   float tau_edit;            /* must be >= tau_mask                         */
   float theta_spawn;
   float sm_scale;            /* 0 -> 1/sqrt(head_dim)                       */
+  int32_t window_in_pages;   /* 0: this step's window K/V are passed to the
+                                attention and copied to the pages when a block
+                                retires.  1: they are scattered to the pages
+                                every step (fb_scatter_window_kv, Eq. 6), the
+                                attention reads every key through the page
+                                table and retirement copies nothing          */
 } fb_config;
 
 /* Per-request wavefront state (Sec. 3.2: (L_b, R_b), in-order commit
@@ -153,12 +159,34 @@ int fb_pack_wavefronts(fb_ctx* ctx, const fb_state* st, const fb_pack* out,
  *   page_table    [R_max, max_pages_per_req] int32
  * bf16 inputs, fp32 accumulation, bf16 output.  Rows of padding slots are
  * not written.  `pk` and `ws` must come from fb_pack_wavefronts of this
- * step. */
+ * step.  In a context with window_in_pages = 1 the window blocks are read
+ * from the pages too (positions [o_r, o_r + (s+1) bl), written there by
+ * fb_scatter_window_kv); k_win and v_win must then be NULL. */
 int fb_wavefront_attn(fb_ctx* ctx, const fb_pack* pk, const void* q,
                       const void* k_win, const void* v_win,
                       const void* k_pool, const void* v_pool,
                       const int32_t* page_table, void* out, void* ws,
                       int32_t* status, void* stream);
+
+/* Sec. 3.2 Eq. 6 as data movement (contexts with window_in_pages = 1): the
+ * fresh K/V of every live window position go to the request's pages at their
+ * absolute positions, cache[r, o_r + s*bl + t] = k_new[slot, t], for all KV
+ * heads; the frozen prefix [0, o_r) and positions right of the window are
+ * not touched.  Retirement then freezes what is already in place.
+ *   k_new, v_new  [max_slots*bl, n_kv_heads, head_dim] bf16, slot order
+ *   rope_base     0: keys are stored as given.  > 0: each key is first
+ *                 rotated by its absolute position (pairs (x_i, x_{i+d/2})
+ *                 turned by pos * rope_base^(-2i/d); the paper only says the
+ *                 window carries absolute position ids for RoPE, the pairing
+ *                 and the base are the model's), fp32 arithmetic with the
+ *                 angle formed in fp64, result rounded to bf16
+ * `pk` must come from fb_pack_wavefronts of this step; rows of padding slots
+ * are not read.  A page id outside the pool sets FB_ST_BAD_PAGE and that row
+ * is skipped. */
+int fb_scatter_window_kv(fb_ctx* ctx, const fb_pack* pk,
+                         const int32_t* page_table, const void* k_new,
+                         const void* v_new, void* k_pool, void* v_pool,
+                         float rope_base, int32_t* status, void* stream);
 
 /* The paper has no counterpart to this call: it exists for callers that
  * cannot allocate device memory (an engine that has given the whole device
@@ -172,6 +200,7 @@ int fb_wavefront_attn(fb_ctx* ctx, const fb_pack* pk, const void* q,
  * rewritten with the same values fb_pack_wavefronts gives) and never splits
  * the key axis, so results may differ from fb_wavefront_attn in the last
  * rounding only.
+ *   - FB_ERR_UNSUPPORTED for contexts with window_in_pages = 1.
  *   - FB_ERR_WORKSPACE when the configuration's work list does not fit in
  *     8 MiB (about 100,000 (request, KV head, Q-tile pair) units).
  *   - The first call on each device looks up the array's device address and
@@ -211,7 +240,9 @@ int fb_t2t_step(fb_ctx* ctx, const fb_pack* pk, const void* logits,
  *   spawned       [R_max] uint8
  *   step_counters [8] int32 (FB_CT_*), overwritten
  * Mutates st->{active, prefix_len, L, R, tokens (new block), pe_done} and the
- * pool pages of committed blocks; frozen positions are never rewritten. */
+ * pool pages of committed blocks; frozen positions are never rewritten.
+ * With window_in_pages = 1 nothing is copied (k_win, v_win, k_pool, v_pool
+ * may be NULL): advancing prefix_len freezes what the scatter put in place. */
 int fb_gate_commit(fb_ctx* ctx, const fb_pack* pk, const int32_t* slot_stats,
                    const fb_state* st, const void* k_win, const void* v_win,
                    void* k_pool, void* v_pool, int32_t* n_committed,

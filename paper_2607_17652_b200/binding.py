@@ -26,7 +26,8 @@ FB_SLOT_STATS, FB_STEP_COUNTERS = 6, 8
 
 EXPORTS = ["fb_create", "fb_destroy", "fb_last_error", "fb_workspace_bytes",
            "fb_pack_wavefronts", "fb_wavefront_attn", "fb_t2t_step",
-           "fb_gate_commit", "fb_step_host", "fb_wavefront_attn_static"]
+           "fb_gate_commit", "fb_step_host", "fb_wavefront_attn_static",
+           "fb_scatter_window_kv"]
 
 
 class fb_config(C.Structure):
@@ -35,7 +36,8 @@ class fb_config(C.Structure):
         "head_dim", "page_size", "num_pages", "max_pages_per_req", "vocab",
         "mask_id", "eos_id", "max_blocks", "s_pe")] + \
         [(n, C.c_float) for n in ("tau_mask", "tau_edit", "theta_spawn",
-                                  "sm_scale")]
+                                  "sm_scale")] + \
+        [("window_in_pages", C.c_int32)]
 
 
 class fb_state(C.Structure):
@@ -91,6 +93,8 @@ def lib() -> C.CDLL:
                                      C.POINTER(fb_state)] + [P] * 9
         l.fb_wavefront_attn_static.argtypes = [P, C.POINTER(fb_state),
                                                C.POINTER(fb_pack)] + [P] * 8
+        l.fb_scatter_window_kv.argtypes = [P, C.POINTER(fb_pack)] + [P] * 5 + \
+            [C.c_float, P, P]
         l.fb_step_host.argtypes = [P, C.POINTER(fb_state), C.POINTER(fb_pack),
                                    C.POINTER(fb_device_bufs),
                                    C.POINTER(fb_host_io), P]
@@ -227,6 +231,17 @@ def fb_wavefront_attn(ctx: Context, pk: PackBuffers, q, k_win, v_win, k_pool,
         ctx.handle, C.byref(p), _ptr(q), _ptr(k_win), _ptr(v_win),
         _ptr(k_pool), _ptr(v_pool), _ptr(page_table), _ptr(out), _ptr(ws),
         _ptr(status), _stream(stream)))
+
+
+def fb_scatter_window_kv(ctx: Context, pk: PackBuffers, page_table, k_new, v_new,
+                         k_pool, v_pool, status, rope_base: float = 0.0,
+                         stream=None):
+    """Eq. 6 as data movement (contexts with window_in_pages=1)."""
+    p = pk.c()
+    ctx.check(lib().fb_scatter_window_kv(
+        ctx.handle, C.byref(p), _ptr(page_table), _ptr(k_new), _ptr(v_new),
+        _ptr(k_pool), _ptr(v_pool), C.c_float(rope_base), _ptr(status),
+        _stream(stream)))
 
 
 def fb_wavefront_attn_static(ctx: Context, st: DeviceState, pk: PackBuffers, q,

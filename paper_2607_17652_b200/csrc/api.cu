@@ -85,6 +85,8 @@ int fb_create(const fb_config* cfg, fb_ctx** out) {
   if (c.s_pe > 255) return fail(nullptr, FB_ERR_UNSUPPORTED, "s_pe must be at most 255");
   if (c.tau_edit < c.tau_mask)
     return fail(nullptr, FB_ERR_UNSUPPORTED, "tau_edit < tau_mask is not supported");
+  if (c.window_in_pages != 0 && c.window_in_pages != 1)
+    return fail(nullptr, FB_ERR_INVALID_ARG, "window_in_pages must be 0 or 1");
   if ((long long)c.max_requests * c.wmax * c.block_len > (1ll << 24))
     return fail(nullptr, FB_ERR_UNSUPPORTED, "max_requests * wmax * block_len is too large");
   fb_ctx* ctx = new (std::nothrow) fb_ctx();
@@ -136,8 +138,12 @@ int fb_wavefront_attn(fb_ctx* ctx, const fb_pack* pk, const void* q, const void*
                       int32_t* status, void* stream) {
   if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");
   if (int e = check_pack(ctx, pk)) return e;
-  if (!q || !k_win || !v_win || !k_pool || !v_pool || !page_table || !out)
+  const bool resident = ctx->cfg.window_in_pages != 0;
+  if (!q || !k_pool || !v_pool || !page_table || !out)
     return fail(ctx, FB_ERR_INVALID_ARG, "a tensor pointer is null");
+  if (resident && (k_win || v_win))
+    return fail(ctx, FB_ERR_INVALID_ARG, "window_in_pages = 1: k_win and v_win must be null (the window is read from the pages)");
+  if (!resident && (!k_win || !v_win)) return fail(ctx, FB_ERR_INVALID_ARG, "a tensor pointer is null");
   if (!ws) return fail(ctx, FB_ERR_WORKSPACE, "workspace is null");
   if (!status) return fail(ctx, FB_ERR_INVALID_ARG, "status is null");
   if (!aligned16(q) || !aligned16(k_win) || !aligned16(v_win) || !aligned16(k_pool) || !aligned16(v_pool) ||
@@ -146,6 +152,20 @@ int fb_wavefront_attn(fb_ctx* ctx, const fb_pack* pk, const void* q, const void*
   if (reinterpret_cast<uintptr_t>(ws) & 255u) return fail(ctx, FB_ERR_ALIGNMENT, "workspace must be 256-byte aligned");
   return fb::launch_attn(ctx, pk, q, k_win, v_win, k_pool, v_pool, page_table, out, ws, status,
                          (cudaStream_t)stream);
+}
+
+int fb_scatter_window_kv(fb_ctx* ctx, const fb_pack* pk, const int32_t* page_table, const void* k_new,
+                         const void* v_new, void* k_pool, void* v_pool, float rope_base, int32_t* status,
+                         void* stream) {
+  if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");
+  if (int e = check_pack(ctx, pk)) return e;
+  if (!page_table || !k_new || !v_new || !k_pool || !v_pool || !status)
+    return fail(ctx, FB_ERR_INVALID_ARG, "a tensor pointer is null");
+  if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_pool) || !aligned16(v_pool))
+    return fail(ctx, FB_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  if (!(rope_base == rope_base) || rope_base < 0.f) return fail(ctx, FB_ERR_INVALID_ARG, "rope_base is NaN or negative");
+  return fb::launch_scatter(ctx, pk, page_table, k_new, v_new, k_pool, v_pool, rope_base, status,
+                            (cudaStream_t)stream);
 }
 
 int fb_t2t_step(fb_ctx* ctx, const fb_pack* pk, const void* logits, const fb_state* st, int32_t* argmax,
@@ -165,8 +185,9 @@ int fb_gate_commit(fb_ctx* ctx, const fb_pack* pk, const int32_t* slot_stats, co
   if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");
   if (int e = check_pack(ctx, pk)) return e;
   if (int e = check_state(ctx, st)) return e;
-  if (!slot_stats || !k_win || !v_win || !k_pool || !v_pool || !n_committed || !spawned || !step_counters ||
-      !status)
+  if (ctx->cfg.window_in_pages) k_win = v_win = nullptr;      // nothing to copy: the window already lives in the pages
+  else if (!k_win || !v_win || !k_pool || !v_pool) return fail(ctx, FB_ERR_INVALID_ARG, "a tensor pointer is null");
+  if (!slot_stats || !n_committed || !spawned || !step_counters || !status)
     return fail(ctx, FB_ERR_INVALID_ARG, "a tensor pointer is null");
   if (!aligned16(k_win) || !aligned16(v_win) || !aligned16(k_pool) || !aligned16(v_pool))
     return fail(ctx, FB_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
@@ -195,8 +216,12 @@ int fb_step_host(fb_ctx* ctx, const fb_state* st, const fb_pack* pk, const fb_de
   if ((e = fb::cuda_err(ctx, cudaMemcpyAsync(dev->v_win, io->h_v_win, kb, cudaMemcpyHostToDevice, s), "copy v_win"))) return e;
   if ((e = fb::cuda_err(ctx, cudaMemcpyAsync(dev->logits, io->h_logits, lb, cudaMemcpyHostToDevice, s), "copy logits"))) return e;
   if ((e = fb_pack_wavefronts(ctx, st, pk, dev->ws, dev->status, stream))) return e;
-  if ((e = fb_wavefront_attn(ctx, pk, dev->q, dev->k_win, dev->v_win, dev->k_pool, dev->v_pool, st->page_table,
-                             dev->out, dev->ws, dev->status, stream))) return e;
+  const bool resident = c.window_in_pages != 0;
+  if (resident && (e = fb_scatter_window_kv(ctx, pk, st->page_table, dev->k_win, dev->v_win, dev->k_pool,
+                                            dev->v_pool, 0.f, dev->status, stream))) return e;
+  if ((e = fb_wavefront_attn(ctx, pk, dev->q, resident ? nullptr : dev->k_win, resident ? nullptr : dev->v_win,
+                             dev->k_pool, dev->v_pool, st->page_table, dev->out, dev->ws, dev->status, stream)))
+    return e;
   if ((e = fb_t2t_step(ctx, pk, dev->logits, st, dev->argmax, dev->conf, dev->action, dev->slot_stats,
                        dev->status, stream))) return e;
   if ((e = fb_gate_commit(ctx, pk, dev->slot_stats, st, dev->k_win, dev->v_win, dev->k_pool, dev->v_pool,

@@ -65,6 +65,7 @@ struct AttnParams {
   float* part_o;
   int32_t* status;
   int32_t bl, n_q_heads, n_kv_heads, group, max_pages_per_req, num_pages;
+  int32_t resident;     // 1: the window is read from the pages (every key tile is a paged one)
   float scale_log2;
   long long wait_cycles;
 #ifdef FB_TRACE
@@ -126,9 +127,11 @@ __device__ __forceinline__ int uni(int x) { return __shfl_sync(0xffffffffu, x, 0
 struct ItemU {
   int req, kvhA, kvhB, rowA, rowB, jb, n, nA, nB, npt, prefix_len, win_row0, winA, winB;
   __device__ __forceinline__ bool dual() const { return kvhA != kvhB; }   // two K/V streams
-  __device__ __forceinline__ int limit(int j, int winX) const {
+  // keys of local tile j that a tile with window reach winX may see; `resident`: the
+  // window follows the prefix in the pages, one run of keys [0, prefix_len + winX)
+  __device__ __forceinline__ int limit(int j, int winX, int resident) const {
     const int gj = jb + j;
-    const int lim = gj < npt ? prefix_len - gj * kTileN : winX - (gj - npt) * kTileN;
+    const int lim = gj < npt ? prefix_len + (resident ? winX : 0) - gj * kTileN : winX - (gj - npt) * kTileN;
     return min(lim, kTileN);
   }
 };
@@ -151,9 +154,10 @@ __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volati
 }
 
 // number of keys of local tile j that tile X (window reach winX) may see
-__device__ __forceinline__ int tile_limit(const ItemGeom& g, int j, int winX) {
+__device__ __forceinline__ int tile_limit(const ItemGeom& g, int j, int winX, int resident) {
   const int gj = g.jb + j;
-  const int lim = gj < g.un.npt ? g.un.prefix_len - gj * kTileN : winX - (gj - g.un.npt) * kTileN;
+  const int lim = gj < g.un.npt ? g.un.prefix_len + (resident ? winX : 0) - gj * kTileN
+                                : winX - (gj - g.un.npt) * kTileN;
   return min(lim, kTileN);
 }
 __device__ __forceinline__ int round16(int x) { return (x + 15) & ~15; }
@@ -252,7 +256,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       uint8_t* dst = (isV ? sV : sK) + mine * TILE_BYTES;
       const int gj = g.jb + j;
       const bool paged = gj < g.npt;
-      const int npg = (gj * kTileN + kPage < g.prefix_len) ? 2 : 1;
+      const int npg = (gj * kTileN + kPage < g.prefix_len + (p.resident ? max(g.winA, g.winB) : 0)) ? 2 : 1;
       int page[2] = {0, 0};
       if (paged) {
         // the window of 64 cached entries moves on once V has reached its second half
@@ -428,8 +432,8 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         if (!wait_k(st)) { ok = false; break; }
         FB_TR(1, 12);
         tc_fence_after();
-        if (nA > 0) issue_qk(0, st, round16(g.limit(0, g.winA)));
-        if (nB > 0) issue_qk(1, st, round16(g.limit(0, g.winB)));
+        if (nA > 0) issue_qk(0, st, round16(g.limit(0, g.winA, p.resident)));
+        if (nB > 0) issue_qk(1, st, round16(g.limit(0, g.winB, p.resident)));
         commit(&k_empty[st]);
         if (n == 1) commit(q_empty);               // Q is free once its last QK has run
         for (int j = 0; j < n; ++j) {
@@ -443,7 +447,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           FB_TR(1, 21);
           // tile A: O_A += P_A(j) V(j), then S_A(j+1) so that softmax A can go on
           if (j < nA) {
-            const int nks = round16(g.limit(j, g.winA)) >> 4;
+            const int nks = round16(g.limit(j, g.winA, p.resident)) >> 4;
             if (!warp_wait(&p_full[0], cntPA & 1, abortf, LIM)) { ok = false; break; }
             FB_TR(1, 23);
             ++cntPA;
@@ -454,12 +458,12 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           if (j + 1 < nA) {
             FB_TR(1, 25);
             tc_fence_after();
-            issue_qk(0, st1, round16(g.limit(j + 1, g.winA)));
+            issue_qk(0, st1, round16(g.limit(j + 1, g.winA, p.resident)));
             FB_TR(1, 26);
           }
           // tile B
           if (j < nB) {
-            const int nks = round16(g.limit(j, g.winB)) >> 4;
+            const int nks = round16(g.limit(j, g.winB, p.resident)) >> 4;
             if (!warp_wait(&p_full[1], cntPB & 1, abortf, LIM)) { ok = false; break; }
             FB_TR(1, 33);
             ++cntPB;
@@ -469,7 +473,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           commit(&v_empty[sv]);
           if (j + 1 < nB) {
             tc_fence_after();
-            issue_qk(1, st1, round16(g.limit(j + 1, g.winB)));
+            issue_qk(1, st1, round16(g.limit(j + 1, g.winB, p.resident)));
           }
           if (j + 1 < n) {
             commit(&k_empty[st1]);
@@ -482,11 +486,11 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         if (!wait_k(0)) { ok = false; break; }
         FB_TR(1, 12);
         tc_fence_after();
-        issue_qk(0, 0, round16(g.limit(0, g.winA)));
+        issue_qk(0, 0, round16(g.limit(0, g.winA, p.resident)));
         commit(&k_empty[0]);
         if (!wait_k(1)) { ok = false; break; }
         tc_fence_after();
-        issue_qk(1, 1, round16(g.limit(0, g.winB)));
+        issue_qk(1, 1, round16(g.limit(0, g.winB, p.resident)));
         commit(&k_empty[1]);
         if (n == 1) commit(q_empty);
         // The streams do not depend on each other: serve whichever tile's P is ready.
@@ -510,7 +514,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           if (!wait_v(X)) { ok = false; break; }
           FB_TR(1, 34);
           tc_fence_after();
-          issue_pv(X, X, 0, round16(g.limit(j, g.winA)) >> 4, j > 0);
+          issue_pv(X, X, 0, round16(g.limit(j, g.winA, p.resident)) >> 4, j > 0);
           commit(&v_empty[X]);
           FB_TR(1, 35);
           if (j + 1 < n) {
@@ -519,7 +523,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             if (!wait_k(X)) { ok = false; break; }
             FB_TR(1, 36);
             tc_fence_after();
-            issue_qk(X, X, round16(g.limit(j + 1, g.winA)));
+            issue_qk(X, X, round16(g.limit(j + 1, g.winA, p.resident)));
             commit(&k_empty[X]);
             if (--qk_left == 0) commit(q_empty);
           }
@@ -564,7 +568,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         FB_TR(2 + X, 41);
         ++cntS;
         tc_fence_after();
-        const int limit = tile_limit(g, j, winX);
+        const int limit = tile_limit(g, j, winX, p.resident);
         // The running reference m_ref is only re-based when a score exceeds it by
         // more than 2^8 (lazy rescale), so the common tile needs no separate max
         // pass: the exponentials are taken against the old reference while the
@@ -849,8 +853,9 @@ int launch_attn(fb_ctx* ctx, const fb_pack* pk, const void* q, const void* k_win
       cuuint64_t dims[3] = {D, (cuuint64_t)c.n_kv_heads, rows};
       cuuint64_t str[2] = {D * 2, (cuuint64_t)c.n_kv_heads * D * 2};
       cuuint32_t box[3] = {64, 1, 128};
-      if (int e = encode(ctx, &ctx->tm_kwin, k_win, 3, dims, str, box)) return e;
-      if (int e = encode(ctx, &ctx->tm_vwin, v_win, 3, dims, str, box)) return e;
+      // window resident in the pages: no window tensors; the two maps are never used then
+      if (int e = encode(ctx, &ctx->tm_kwin, k_win ? k_win : k_pool, 3, dims, str, box)) return e;
+      if (int e = encode(ctx, &ctx->tm_vwin, v_win ? v_win : v_pool, 3, dims, str, box)) return e;
     }
     {
       cuuint64_t dims[2] = {D, (cuuint64_t)c.num_pages * c.n_kv_heads * kPage};
@@ -873,6 +878,7 @@ int launch_attn(fb_ctx* ctx, const fb_pack* pk, const void* q, const void* k_win
   p.status = status;
   p.bl = c.block_len; p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.group = ctx->group;
   p.max_pages_per_req = c.max_pages_per_req; p.num_pages = c.num_pages;
+  p.resident = c.window_in_pages;
   p.scale_log2 = ctx->sm_scale * kLog2eF;
 #ifdef FB_TRACE
   static long long* g_trace = nullptr;

@@ -60,6 +60,8 @@ extern "C" int fb_wavefront_attn_static(fb_ctx* ctx, const fb_state* st, const f
   if (!ctx) return FB_ERR_INVALID_ARG;
   if (!st || !pk || !q || !k_win || !v_win || !k_pool || !v_pool || !out || !status || !st->page_table)
     return fb::set_err(ctx, FB_ERR_INVALID_ARG, "fb_wavefront_attn_static: a pointer is null");
+  if (ctx->cfg.window_in_pages)
+    return fb::set_err(ctx, FB_ERR_UNSUPPORTED, "fb_wavefront_attn_static: contexts with window_in_pages = 1 are not supported");
   const void* ps[] = {q, k_win, v_win, k_pool, v_pool, out};
   for (const void* p : ps)
     if (reinterpret_cast<uintptr_t>(p) & 15u)

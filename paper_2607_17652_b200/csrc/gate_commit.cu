@@ -104,7 +104,8 @@ __global__ void __launch_bounds__(kGateThreads) gate_commit_kernel(const GatePar
   const int c = s_c, first = s_first, P = s_P;
   const int vec_per_head = p.head_dim / 8;                 // uint4 per (token, head)
   const int vec_per_tok = p.n_kv_heads * vec_per_head;
-  const int total = c * p.bl * vec_per_tok;
+  // (window resident in the pages: nothing to copy, the prefix pointer has moved over it)
+  const int total = p.k_win ? c * p.bl * vec_per_tok : 0;
   for (int i = tid; i < total; i += kGateThreads) {
     const int tok = i / vec_per_tok, rem = i % vec_per_tok;
     const int h = rem / vec_per_head, v = rem % vec_per_head;

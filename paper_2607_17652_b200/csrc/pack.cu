@@ -21,6 +21,7 @@ struct PackParams {
   AttnUnit* units;
   int32_t max_requests, wmax, bl, max_slots, max_blocks, mask_id, n_kv_heads;
   int32_t tiles_per_slot, tokens_per_tile, target_items, min_chunk_tiles, max_items, max_units, max_parts;
+  int32_t resident;   // window K/V live in the pages: key tiles follow absolute positions
   int32_t n_gather_blocks;
 };
 
@@ -99,6 +100,10 @@ __device__ __forceinline__ ReqGeom req_geom(const PackParams& p, int r, int32_t*
   g.P = g.w ? max(p.prefix_len[r], 0) : 0;
   g.npt = (g.P + kTileN - 1) / kTileN;
   g.nt = g.w ? g.npt + (g.w * p.bl + kTileN - 1) / kTileN : 0;
+  if (p.resident) {       // one run of keys [0, P + w*bl), all of it paged
+    g.nt = g.w ? (g.P + g.w * p.bl + kTileN - 1) / kTileN : 0;
+    g.npt = g.nt;
+  }
   return g;
 }
 
@@ -176,7 +181,7 @@ __device__ void build_sched(const PackParams& p) {
         un.slotA = first + sA;
         un.t0A = (qa % p.tiles_per_slot) * p.tokens_per_tile;
         un.winA = (sA + 1) * p.bl;
-        un.nvisA = g.npt + (un.winA + kTileN - 1) / kTileN;
+        un.nvisA = p.resident ? (g.P + un.winA + kTileN - 1) / kTileN : g.npt + (un.winA + kTileN - 1) / kTileN;
         if (full) {
           const int qb = qa + 1;
           const int sB = qb / p.tiles_per_slot;
@@ -184,7 +189,7 @@ __device__ void build_sched(const PackParams& p) {
           un.slotB = first + sB;
           un.t0B = (qb % p.tiles_per_slot) * p.tokens_per_tile;
           un.winB = (sB + 1) * p.bl;
-          un.nvisB = g.npt + (un.winB + kTileN - 1) / kTileN;
+          un.nvisB = p.resident ? (g.P + un.winB + kTileN - 1) / kTileN : g.npt + (un.winB + kTileN - 1) / kTileN;
         } else if (h + 1 < p.n_kv_heads) {
           un.kvh = h | ((h + 1) << 16);
           un.slotB = un.slotA; un.t0B = un.t0A; un.winB = un.winA; un.nvisB = un.nvisA;
@@ -316,6 +321,7 @@ int launch_pack(fb_ctx* ctx, const fb_state* st, const fb_pack* out, void* ws, i
   p.n_kv_heads = c.n_kv_heads; p.tiles_per_slot = ctx->tiles_per_slot;
   p.tokens_per_tile = ctx->tokens_per_tile; p.target_items = ctx->target_items;
   p.min_chunk_tiles = ctx->min_chunk_tiles;
+  p.resident = ctx->cfg.window_in_pages;
   p.max_items = ctx->ws.max_items; p.max_units = ctx->ws.max_units; p.max_parts = ctx->ws.max_parts;
   p.n_gather_blocks = (p.max_slots + kSlotsPerBlock - 1) / kSlotsPerBlock;
   pack_kernel<<<p.n_gather_blocks + 1, kPackThreads, 0, stream>>>(p);

@@ -31,6 +31,9 @@ def test_header_symbols_are_exported():
     for name in declared:
         assert hasattr(lib, name), name
     assert set(B.EXPORTS) >= declared - {"fb_no_such"}
+    # every call is bound with explicit argument types (a bare Python int would be cut to 32 bits)
+    for name in B.EXPORTS:
+        assert getattr(lib, name).argtypes is not None, name
 
 
 def test_struct_layouts_match_header_order():
@@ -48,12 +51,33 @@ def test_create_validates_configuration():
     bad = [dict(head_dim=96), dict(page_size=32), dict(block_len=24),
            dict(n_kv_heads=3), dict(wmax=0), dict(vocab=1001), dict(wmax=9),
            dict(tau_edit=0.5), dict(s_pe=300), dict(max_requests=-1),
-           dict(tau_mask=float("nan"))]
+           dict(tau_mask=float("nan")), dict(window_in_pages=2)]
     for delta in bad:
         with pytest.raises(B.FlowBlockError):
             B.Context(**dict(GOOD, **delta))
     assert B.lib().fb_create(None, None) == B.FB_ERR_INVALID_ARG
     assert b"null" in B.lib().fb_last_error(None)
+
+
+def test_window_in_pages_argument_rules():
+    lib = B.lib()
+    pk = B.fb_pack(*([0x1000] * 9))
+    res = B.Context(**dict(GOOD, window_in_pages=1))
+    a = [0x1000] * 12
+    # page-resident window: window tensors must be null for the attention
+    assert lib.fb_wavefront_attn(res.handle, C.byref(pk), 0x1000, 0x1000, 0x1000, 0x1000, 0x1000, 0x1000,
+                                 0x1000, 0x1000, 0x1000, None) == B.FB_ERR_INVALID_ARG
+    assert b"must be null" in lib.fb_last_error(res.handle)
+    assert lib.fb_scatter_window_kv(res.handle, C.byref(pk), 0x1000, None, 0x1000, 0x1000, 0x1000, 0.0,
+                                    0x1000, None) == B.FB_ERR_INVALID_ARG
+    assert lib.fb_scatter_window_kv(res.handle, C.byref(pk), 0x1000, 0x1008, 0x1000, 0x1000, 0x1000, 0.0,
+                                    0x1000, None) == B.FB_ERR_ALIGNMENT
+    assert lib.fb_scatter_window_kv(res.handle, C.byref(pk), 0x1000, 0x1000, 0x1000, 0x1000, 0x1000, -1.0,
+                                    0x1000, None) == B.FB_ERR_INVALID_ARG
+    # slot-order window: window tensors are required
+    ctx = B.Context(**GOOD)
+    assert lib.fb_wavefront_attn(ctx.handle, C.byref(pk), 0x1000, None, None, 0x1000, 0x1000, 0x1000,
+                                 0x1000, 0x1000, 0x1000, None) == B.FB_ERR_INVALID_ARG
 
 
 def test_null_and_misaligned_arguments_are_rejected_on_the_host():

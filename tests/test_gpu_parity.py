@@ -469,3 +469,65 @@ def test_step_host_equals_the_four_calls():
         np.testing.assert_array_equal(a[name], b2[name], err_msg=name)
     assert torch.equal(hkp, dkp) and torch.equal(hvp, dvp)
     assert bool((dev["logits"][n_rows:] == 0).all())      # rows beyond n_rows were not copied
+
+
+# ------------------------------------- Eq. 6 as data movement (window in pages)
+RESIDENT = ["tiny", "tiny_d128_b64", "tiny_wide", "tiny_noprefix", "tiny_b96", "tiny_g8", "cfg1"]
+
+
+@pytest.mark.parametrize("name", RESIDENT)
+@pytest.mark.parametrize("rope_base", [0.0, 10000.0])
+def test_scatter_window_kv_and_resident_attention(name, rope_base):
+    """fb_scatter_window_kv puts the fresh window K/V at their absolute
+    positions (bit-exact without the rotary embedding, within bf16 rounding of
+    the fp64 rotation with it) and touches nothing else; attention over the
+    page-resident window matches the oracle; retirement then copies nothing."""
+    case = make_case(WORKLOADS[name], with_logits=False)
+    stc = case["stc"]
+    wl = stc.wl
+    b = wl.block_len
+    ctx, st, pk, sb = gpu_objects(case, window_in_pages=1)
+    q, kw, vw, kp, vp = case["attn"]
+    dq, dkw, dvw, dkp, dvp = (t.to(DEV) for t in (q, kw, vw, kp, vp))
+    B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+    B.fb_scatter_window_kv(ctx, pk, st.page_table, dkw, dvw, dkp, dvp, sb.status, rope_base=rope_base)
+    sb.out.fill_(7.0)
+    B.fb_wavefront_attn(ctx, pk, dq, None, None, dkp, dvp, st.page_table, sb.out, sb.ws, sb.status)
+    torch.cuda.synchronize()
+    assert int(sb.status.item()) == 0
+    ocfg = H.oracle_cfg(stc)
+    ost = H.oracle_state(stc, case["tokens"])
+    opk = O.pack_wavefronts(ocfg, ost)
+    check_pack(pk, opk)
+    okp, ovp = H.f64(kp), H.f64(vp)
+    O.scatter_window_kv(ocfg, opk, H.f64(kw), H.f64(vw), okp, ovp, stc.page_table, rope_base=rope_base)
+    gk, gv = H.f64(dkp.cpu()), H.f64(dvp.cpu())
+    np.testing.assert_array_equal(gv, ovp)
+    if rope_base == 0.0:
+        np.testing.assert_array_equal(gk, okp)
+    else:
+        # fp32 rotation of bf16 inputs, rounded to bf16: half an ulp of the result
+        # (2^-9 relative) plus the fp32 arithmetic
+        assert np.all(np.abs(gk - okp) <= 2.0 ** -8 * np.abs(okp) + 1e-6)
+        untouched = okp == H.f64(kp)
+        np.testing.assert_array_equal(gk[untouched], okp[untouched])
+    # attention over what the GPU scattered (its own bf16 keys), against the oracle on the same pools
+    ref = O.wavefront_attn(ocfg, opk, H.f64(q), None, None, gk, gv, stc.page_table)
+    max_abs, rel = H.attn_errors(sb.out, ref, H.live_rows(opk, b))
+    assert max_abs <= ATTN_MAX_ABS and rel <= ATTN_REL_L2, (max_abs, rel)
+    assert bool((sb.out[opk.n_live * b:].float() == 7.0).all())
+    # pointer-bump retirement: every block finished, pools stay as they are
+    stats = torch.zeros_like(sb.slot_stats)
+    toks = st.tokens.clone()
+    toks[toks == stc.mask_id] = 1
+    st.tokens.copy_(toks)
+    ost.tokens[ost.tokens == stc.mask_id] = 1
+    B.fb_gate_commit(ctx, pk, stats, st, None, None, None, None, sb.n_committed, sb.spawned,
+                     sb.step_counters, sb.status)
+    torch.cuda.synchronize()
+    ncom, spawned, ctr = O.gate_commit(ocfg, opk, np.zeros((ocfg.max_slots, 6), np.int32), ost)
+    np.testing.assert_array_equal(sb.n_committed.cpu().numpy(), ncom)
+    g = st.to_numpy()
+    for nm in ("active", "prefix_len", "L", "R"):
+        np.testing.assert_array_equal(g[nm], getattr(ost, nm), err_msg=nm)
+    assert torch.equal(dkp.cpu().view(torch.int16), torch.from_numpy(synth.to_bits(torch.from_numpy(gk).to(torch.bfloat16)).view(np.int16)).view(dkp.shape))
