@@ -252,6 +252,33 @@ def run_ours(args):
     counters = sb.step_counters.cpu().numpy().tolist()
     stc1 = device_structure()
 
+    # ---------------------- next row: Eq. 6 as data movement (window in pages)
+    nxt = None
+    if only == "all" and world == 1:
+        ctx2 = B.Context(**synth.config_dict(stc, window_in_pages=1))
+        pk2 = B.PackBuffers.alloc(ctx2, dev)
+        ws2 = B.alloc_workspace(ctx2, dev)
+        n2 = max(3, min(args.steps, 10))
+        ev2 = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n2)]
+        for k in range(3 + n2):
+            B.fb_pack_wavefronts(ctx2, st, pk2, ws2, sb.status, stream)
+            e = ev2[k - 3] if k >= 3 else None
+            if e: e[0].record(stream)
+            B.fb_scatter_window_kv(ctx2, pk2, st.page_table, kw, vw, kp, vp, sb.status, 10000.0, stream)
+            if e: e[1].record(stream)
+            B.fb_wavefront_attn(ctx2, pk2, q, None, None, kp, vp, st.page_table, sb.out, ws2, sb.status, stream)
+            if e: e[2].record(stream)
+        barrier()
+        sc_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in ev2]))
+        ra_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in ev2]))
+        live_now = synth.n_live_slots(device_structure())
+        sc_bytes = 2.0 * 2 * live_now * wl.block_len * wl.n_kv_heads * wl.head_dim * 2      # K and V, read + write
+        nxt = {"scatter_window_kv": {"ms": round(sc_ms, 4), "bytes": sc_bytes, "rope": True,
+                                     "gbs": round(sc_bytes / sc_ms / 1e6, 1)},
+               "attn_window_in_pages": {"ms": round(ra_ms, 4),
+                                        "tflops": round(attn_flops(device_structure()) / ra_ms / 1e9, 2)}}
+        del ctx2, pk2, ws2
+
     # ------------------------------------------------------------ end to end
     e2e_ms, h2d, d2h = float("nan"), 0, 0
     if not args.no_e2e and only == "all":
@@ -347,6 +374,9 @@ def run_ours(args):
             "roofline_attn": roof_attn, "roofline_t2t": roof_t2t,
             "device_status": status, "step_counters": counters,
         }
+        if nxt:
+            nxt["scatter_window_kv"]["frac_of_measured_hbm"] = round(nxt["scatter_window_kv"]["gbs"] / peaks["hbm_gbs"], 4)
+            line["next_rows"] = nxt
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(wl, stc_init, tokens, z_live, attn, budget_s=args.cpu_budget)
         print(json.dumps(line), flush=True)

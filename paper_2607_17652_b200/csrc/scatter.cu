@@ -3,10 +3,11 @@
 // (all KV heads), optionally with the rotary embedding applied to the keys.
 // HBM-bound: 2 x rows x Hkv x d x 2 bytes read and as many written.
 //
-// One CTA per slot.  For a (token, head) the head_dim elements are contiguous
+// One to four CTAs per slot (the KV heads are dealt among them).  For a (token, head) the head_dim elements are contiguous
 // in the source (slot-order rows) and in the destination (pool row of that
 // position), so a thread moves 16-byte pieces: with the rotary embedding a
-// thread owns the two pieces that hold elements i and i + d/2 of eight pairs.
+// thread owns the two pieces that hold elements i and i + d/2 of eight pairs,
+// and the rotation angles come from a per-slot table in shared memory.
 #include "fb_common.cuh"
 
 namespace fb {
@@ -30,19 +31,6 @@ __device__ __forceinline__ uint32_t to_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// cos / sin of pos * base^(-2i/d) for the eight pairs a thread owns; the angle is
-// formed and reduced in fp64 (positions reach tens of thousands of radians)
-__device__ __forceinline__ void rope_angles(int pos, int i0, int d, float base, float (&c)[8], float (&s)[8]) {
-  const double l2b = log2((double)base);
-#pragma unroll
-  for (int k = 0; k < 8; ++k) {
-    const double ang = (double)pos * exp2(-2.0 * (double)(i0 + k) / (double)d * l2b);
-    double sd, cd;
-    sincos(ang, &sd, &cd);
-    c[k] = (float)cd; s[k] = (float)sd;
-  }
-}
-
 __global__ void __launch_bounds__(kScatterThreads) scatter_window_kv_kernel(const ScatterParams p) {
   const int slot = blockIdx.x;
   if (slot >= *p.n_live) return;
@@ -50,13 +38,40 @@ __global__ void __launch_bounds__(kScatterThreads) scatter_window_kv_kernel(cons
   const int vph = p.head_dim / 8;                    // 16-byte pieces per (token, head)
   const int vpt = p.n_kv_heads * vph;                // ... per token
   const bool rope = p.rope_base > 0.f;
+  // cos / sin of pos * base^(-2i/d), once per (token, pair) and shared by all KV heads, for
+  // 32 tokens of the slot at a time; the angle is formed and reduced in fp64 (positions
+  // reach tens of thousands of radians)
+  constexpr int kTokBatch = 32;
+  __shared__ float2 cs[kTokBatch * 64];              // [token of the batch][pair] (cos, sin), d/2 <= 64
+  const int half = p.head_dim / 2;
+  __shared__ double inv_freq[64];                    // base^(-2k/d)
+  if (rope && threadIdx.x < half)
+    inv_freq[threadIdx.x] = exp2(-2.0 * (double)threadIdx.x / (double)p.head_dim * log2((double)p.rope_base));
   // work item = (token, head, piece); with the rotary embedding only the lower half of the
   // pieces is enumerated and each item also handles its partner piece + d/16
   const int per_head = rope ? vph / 2 : vph;
-  const int total = p.bl * p.n_kv_heads * per_head;
+  for (int t0 = 0; t0 < p.bl; t0 += kTokBatch) {
+  const int nt = min(kTokBatch, p.bl - t0);
+  if (rope) {
+    __syncthreads();                                 // the previous batch has been read
+    for (int i = threadIdx.x; i < nt * half; i += kScatterThreads) {
+      const int t = i / half, k = i % half;
+      // angle in fp64, reduced to [-pi, pi] there; sine and cosine of the remainder in fp32
+      const double ang = (double)(pos0 + t0 + t) * inv_freq[k];
+      const double red = fma(-rint(ang * 0.15915494309189535), 6.283185307179586, ang);
+      float sf, cf;
+      sincosf((float)red, &sf, &cf);
+      cs[i] = make_float2(cf, sf);
+    }
+    __syncthreads();
+  }
+  // the KV heads are dealt to the gridDim.y CTAs of the slot
+  const int nh = (p.n_kv_heads - (int)blockIdx.y + (int)gridDim.y - 1) / (int)gridDim.y;
+  const int total = nt * nh * per_head;
   for (int i = threadIdx.x; i < total; i += kScatterThreads) {
-    const int t = i / (p.n_kv_heads * per_head), rem = i % (p.n_kv_heads * per_head);
-    const int h = rem / per_head, v = rem % per_head;
+    const int tb = i / (nh * per_head), rem = i % (nh * per_head);
+    const int t = t0 + tb;
+    const int h = (rem / per_head) * gridDim.y + blockIdx.y, v = rem % per_head;
     const int pos = pos0 + t, pidx = pos / kPage;
     if (pidx >= p.max_pages_per_req) { atomicOr(p.status, FB_ST_BAD_PAGE); continue; }
     const int page = p.page_table[(size_t)r * p.max_pages_per_req + pidx];
@@ -70,7 +85,11 @@ __global__ void __launch_bounds__(kScatterThreads) scatter_window_kv_kernel(cons
     }
     const uint4 a = p.k_new[src], b = p.k_new[src + vph / 2];      // elements i0.. and i0 + d/2..
     float c[8], s[8];
-    rope_angles(pos, v * 8, p.head_dim, p.rope_base, c, s);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const float2 a2 = cs[tb * half + v * 8 + k];
+      c[k] = a2.x; s[k] = a2.y;
+    }
     const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
     uint32_t lo[4], hi[4];
 #pragma unroll
@@ -83,6 +102,7 @@ __global__ void __launch_bounds__(kScatterThreads) scatter_window_kv_kernel(cons
     p.k_pool[dst + vph / 2] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
     p.v_pool[dst] = p.v_new[src];
     p.v_pool[dst + vph / 2] = p.v_new[src + vph / 2];
+  }
   }
 }
 
@@ -99,7 +119,8 @@ int launch_scatter(fb_ctx* ctx, const fb_pack* pk, const int32_t* page_table, co
   p.bl = c.block_len; p.n_kv_heads = c.n_kv_heads; p.head_dim = c.head_dim;
   p.max_pages_per_req = c.max_pages_per_req; p.num_pages = c.num_pages;
   p.rope_base = rope_base;
-  scatter_window_kv_kernel<<<c.max_requests * c.wmax, kScatterThreads, 0, stream>>>(p);
+  const dim3 grid(c.max_requests * c.wmax, c.n_kv_heads >= 4 ? 4 : 1);
+  scatter_window_kv_kernel<<<grid, kScatterThreads, 0, stream>>>(p);
   return cuda_err(ctx, cudaGetLastError(), "scatter_window_kv_kernel launch");
 }
 
