@@ -531,3 +531,73 @@ def test_scatter_window_kv_and_resident_attention(name, rope_base):
     for nm in ("active", "prefix_len", "L", "R"):
         np.testing.assert_array_equal(g[nm], getattr(ost, nm), err_msg=nm)
     assert torch.equal(dkp.cpu().view(torch.int16), torch.from_numpy(synth.to_bits(torch.from_numpy(gk).to(torch.bfloat16)).view(np.int16)).view(dkp.shape))
+
+
+# ------------------------------------------------ degenerate and faulty inputs
+def test_whole_step_on_an_empty_batch_touches_nothing():
+    """No decoding request: every call is a no-op that leaves the outputs of
+    padding rows, the state and the pools as they were."""
+    wl = WORKLOADS["tiny"]
+    case = make_case(wl)
+    case["stc"].active[:] = 0
+    stc = case["stc"]
+    ctx, st, pk, sb = gpu_objects(case)
+    q, kw, vw, kp, vp = (t.to(DEV) for t in case["attn"])
+    kp0, vp0 = kp.clone(), vp.clone()
+    z = case["logits"].to(DEV)
+    before = st.to_numpy()
+    sb.out.fill_(7.0)
+    B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+    B.fb_wavefront_attn(ctx, pk, q, kw, vw, kp, vp, st.page_table, sb.out, sb.ws, sb.status)
+    B.fb_t2t_step(ctx, pk, z, st, sb.argmax, sb.conf, sb.action, sb.slot_stats, sb.status)
+    B.fb_gate_commit(ctx, pk, sb.slot_stats, st, kw, vw, kp, vp, sb.n_committed, sb.spawned,
+                     sb.step_counters, sb.status)
+    torch.cuda.synchronize()
+    assert int(sb.status.item()) == 0 and int(pk.n_live.item()) == 0
+    assert bool((sb.out.float() == 7.0).all())
+    assert bool((sb.argmax == -1).all()) and bool((sb.conf == 0).all()) and bool((sb.action == 0).all())
+    assert int(sb.slot_stats.abs().sum()) == 0 and int(sb.n_committed.abs().sum()) == 0
+    assert int(sb.spawned.sum()) == 0
+    after = st.to_numpy()
+    for name in before:
+        np.testing.assert_array_equal(after[name], before[name], err_msg=name)
+    assert torch.equal(kp, kp0) and torch.equal(vp, vp0)
+
+
+def test_faulty_inputs_set_status_bits_and_nothing_traps():
+    """A page id outside the pool and a NaN logit are reported in the status
+    word; the calls complete and the rows that are fine keep their parity."""
+    wl = WORKLOADS["tiny"]
+    case = make_case(wl)
+    stc = case["stc"]
+    r_bad = int(np.flatnonzero(stc.active == 1)[0])
+    pt = stc.page_table.copy()
+    pt[r_bad, 0] = stc.num_pages + 5                      # the first prefix page of one request
+    ctx, st, pk, sb = gpu_objects(case)
+    st.page_table.copy_(torch.from_numpy(pt))
+    q, kw, vw, kp, vp = (t.to(DEV) for t in case["attn"])
+    B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+    B.fb_wavefront_attn(ctx, pk, q, kw, vw, kp, vp, st.page_table, sb.out, sb.ws, sb.status)
+    torch.cuda.synchronize()
+    assert int(sb.status.item()) & B.FB_ST_BAD_PAGE
+    # requests with intact page tables are unaffected
+    ocfg = H.oracle_cfg(stc)
+    opk = O.pack_wavefronts(ocfg, H.oracle_state(stc, case["tokens"]))
+    good = [s for s in range(opk.n_live) if int(opk.slot_req[s]) != r_bad]
+    ref = O.wavefront_attn(ocfg, opk, *(H.f64(t) for t in case["attn"]), stc.page_table, only_slots=good)
+    max_abs, rel = H.attn_errors(sb.out, ref, H.live_rows(opk, wl.block_len, good))
+    assert max_abs <= ATTN_MAX_ABS and rel <= ATTN_REL_L2
+    # NaN logit in one live row
+    sb.status.zero_()
+    z = case["logits"].clone()
+    z[3, 17] = float("nan")
+    st2 = gpu_objects(case)[1]
+    B.fb_t2t_step(ctx, pk, z.to(DEV), st2, sb.argmax, sb.conf, sb.action, sb.slot_stats, sb.status)
+    torch.cuda.synchronize()
+    assert int(sb.status.item()) & B.FB_ST_NAN_LOGIT
+    assert float(sb.conf[3]) == 0.0 and int(sb.action[3]) == 0
+    xhat, conf = O.t2t_rows(ocfg, opk, H.f64(case["logits"]))
+    live = opk.n_live * wl.block_len
+    keep = np.array([i for i in range(live) if i != 3])
+    np.testing.assert_array_equal(sb.argmax.cpu().numpy()[keep], xhat[keep])
+    np.testing.assert_allclose(sb.conf.cpu().numpy()[keep], conf[keep], rtol=0, atol=CONF_TOL)
