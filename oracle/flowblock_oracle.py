@@ -31,6 +31,7 @@ Pins (tests/test_oracle_*.py, all CPU):
                          other pool element); attention over the page-resident
                          window equals attention over the slot-order window;
                          pointer-bump commit equals copy-at-commit
+  embed_gather           brute force over (request, block, token)
   rope_rotate            textbook special cases (position 0, d = 2 rotation,
                          norm, relative-offset invariance of q.k)
 Nothing in this file is "parity unpinned".
@@ -313,6 +314,18 @@ def scatter_window_kv(cfg: Config, pk: Pack, k_new, v_new, k_pool, v_pool,
                 k = rope_rotate(k, pos, rope_base)
             k_pool[page, :, pos % ps, :] = k
             v_pool[page, :, pos % ps, :] = v_new[slot * b + t]
+
+
+def embed_gather(cfg: Config, pk: Pack, table):
+    """Input embeddings of the packed window: row i of the result is the
+    embedding-table row of the gathered token qtok[i] (Eq. 4 feeding the
+    model's first layer), for the rows of live slots; rows of padding slots
+    stay zero.  table [rows >= every token id in use, hidden]."""
+    n = pk.n_live * cfg.block_len
+    out = np.zeros((cfg.max_slots * cfg.block_len, table.shape[1]), table.dtype)
+    for i in range(n):
+        out[i] = table[int(pk.qtok[i])]
+    return out
 
 
 # --------------------------------------------------------------------------

@@ -110,3 +110,20 @@ def test_scatter_with_rope_rotates_keys_only():
             page, off = int(st.page_table[r, pos // ps]), pos % ps
             np.testing.assert_allclose(kp[page, :, off], O.rope_rotate(kw[slot * b + t], pos, 10000.0), atol=0)
             np.testing.assert_array_equal(vp[page, :, off], vw[slot * b + t])
+
+
+def test_embed_gather_brute_force():
+    wl, stc, cfg, st, pk, q, kw, vw, kp, vp = _case(seed=21)
+    rg = np.random.default_rng(3)
+    table = rg.normal(size=(wl.vocab, 12))
+    x = O.embed_gather(cfg, pk, table)
+    b = wl.block_len
+    slot = 0
+    for r in range(wl.n_requests):
+        if st.active[r] != 1:
+            continue
+        for g in range(int(st.L[r]), int(st.R[r])):
+            for t in range(b):
+                np.testing.assert_array_equal(x[slot * b + t], table[st.tokens[r, g * b + t]])
+            slot += 1
+    assert slot == pk.n_live and not x[slot * b:].any()
