@@ -52,7 +52,7 @@ typedef enum {
 
 typedef enum {
   FB_ST_BAD_PAGE = 1,     /* page id outside [0, num_pages): tile skipped */
-  FB_ST_BAD_TOKEN = 2,    /* reserved                                     */
+  FB_ST_BAD_TOKEN = 2,    /* fb_embed_gather: token id outside the table  */
   FB_ST_BAD_STATE = 4,    /* R-L outside [0, wmax] or L,R outside [0, n]  */
   FB_ST_NAN_LOGIT = 8,    /* a row's softmax sum was not finite           */
   FB_ST_DEV_TIMEOUT = 16  /* a bounded device-side wait gave up           */
@@ -187,6 +187,18 @@ int fb_scatter_window_kv(fb_ctx* ctx, const fb_pack* pk,
                          const int32_t* page_table, const void* k_new,
                          const void* v_new, void* k_pool, void* v_pool,
                          float rope_base, int32_t* status, void* stream);
+
+/* Sec. 3.2 Eq. 4 feeding the model: input embeddings of the packed window,
+ * x[i, :] = table[qtok[i], :] for the rows of live slots (rows of padding
+ * slots are not written).
+ *   table  [table_rows, hidden] bf16 (hidden a multiple of 8; table_rows must
+ *          exceed every token id in use, mask_id included)
+ *   x      [max_slots*bl, hidden] bf16
+ * A token id outside [0, table_rows) sets FB_ST_BAD_TOKEN and leaves its row
+ * unwritten. */
+int fb_embed_gather(fb_ctx* ctx, const fb_pack* pk, const void* table,
+                    int32_t table_rows, int32_t hidden, void* x,
+                    int32_t* status, void* stream);
 
 /* The paper has no counterpart to this call: it exists for callers that
  * cannot allocate device memory (an engine that has given the whole device

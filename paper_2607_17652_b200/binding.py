@@ -27,7 +27,7 @@ FB_SLOT_STATS, FB_STEP_COUNTERS = 6, 8
 EXPORTS = ["fb_create", "fb_destroy", "fb_last_error", "fb_workspace_bytes",
            "fb_pack_wavefronts", "fb_wavefront_attn", "fb_t2t_step",
            "fb_gate_commit", "fb_step_host", "fb_wavefront_attn_static",
-           "fb_scatter_window_kv"]
+           "fb_scatter_window_kv", "fb_embed_gather"]
 
 
 class fb_config(C.Structure):
@@ -95,6 +95,8 @@ def lib() -> C.CDLL:
                                                C.POINTER(fb_pack)] + [P] * 8
         l.fb_scatter_window_kv.argtypes = [P, C.POINTER(fb_pack)] + [P] * 5 + \
             [C.c_float, P, P]
+        l.fb_embed_gather.argtypes = [P, C.POINTER(fb_pack), P, C.c_int32,
+                                      C.c_int32, P, P, P]
         l.fb_step_host.argtypes = [P, C.POINTER(fb_state), C.POINTER(fb_pack),
                                    C.POINTER(fb_device_bufs),
                                    C.POINTER(fb_host_io), P]
@@ -242,6 +244,14 @@ def fb_scatter_window_kv(ctx: Context, pk: PackBuffers, page_table, k_new, v_new
         ctx.handle, C.byref(p), _ptr(page_table), _ptr(k_new), _ptr(v_new),
         _ptr(k_pool), _ptr(v_pool), C.c_float(rope_base), _ptr(status),
         _stream(stream)))
+
+
+def fb_embed_gather(ctx: Context, pk: PackBuffers, table, x, status, stream=None):
+    """x[i] = table[qtok[i]] for the rows of live slots (Eq. 4 feeding the model)."""
+    p = pk.c()
+    ctx.check(lib().fb_embed_gather(
+        ctx.handle, C.byref(p), _ptr(table), int(table.shape[0]),
+        int(table.shape[1]), _ptr(x), _ptr(status), _stream(stream)))
 
 
 def fb_wavefront_attn_static(ctx: Context, st: DeviceState, pk: PackBuffers, q,

@@ -168,6 +168,17 @@ int fb_scatter_window_kv(fb_ctx* ctx, const fb_pack* pk, const int32_t* page_tab
                             (cudaStream_t)stream);
 }
 
+int fb_embed_gather(fb_ctx* ctx, const fb_pack* pk, const void* table, int32_t table_rows, int32_t hidden,
+                    void* x, int32_t* status, void* stream) {
+  if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");
+  if (int e = check_pack(ctx, pk)) return e;
+  if (!table || !x || !status) return fail(ctx, FB_ERR_INVALID_ARG, "a tensor pointer is null");
+  if (table_rows < 1 || hidden < 8 || hidden % 8 != 0)
+    return fail(ctx, FB_ERR_SHAPE, "table_rows must be positive and hidden a positive multiple of 8");
+  if (!aligned16(table) || !aligned16(x)) return fail(ctx, FB_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  return fb::launch_embed(ctx, pk, table, table_rows, hidden, x, status, (cudaStream_t)stream);
+}
+
 int fb_t2t_step(fb_ctx* ctx, const fb_pack* pk, const void* logits, const fb_state* st, int32_t* argmax,
                 float* conf, uint8_t* action, int32_t* slot_stats, int32_t* status, void* stream) {
   if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");

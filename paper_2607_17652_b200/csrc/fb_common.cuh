@@ -74,6 +74,8 @@ int launch_attn(fb_ctx*, const fb_pack*, const void* q, const void* k_win, const
                 void* ws, int32_t* status, cudaStream_t);
 int launch_scatter(fb_ctx*, const fb_pack*, const int32_t* page_table, const void* k_new, const void* v_new,
                    void* k_pool, void* v_pool, float rope_base, int32_t* status, cudaStream_t);
+int launch_embed(fb_ctx*, const fb_pack*, const void* table, int table_rows, int hidden, void* x,
+                 int32_t* status, cudaStream_t);
 int launch_t2t(fb_ctx*, const fb_pack*, const void* logits, const fb_state*, int32_t* argmax,
                float* conf, uint8_t* action, int32_t* slot_stats, int32_t* status, cudaStream_t);
 int launch_gate(fb_ctx*, const fb_pack*, const int32_t* slot_stats, const fb_state*,

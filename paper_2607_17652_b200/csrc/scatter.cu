@@ -1,3 +1,5 @@
+// Data movement either side of the packed forward: fb_embed_gather (at the end of this
+// file) and
 // fb_scatter_window_kv: Eq. 6 as data movement.  The fresh K/V rows of every
 // live window position go to the request's pages at their absolute positions
 // (all KV heads), optionally with the rotary embedding applied to the keys.
@@ -122,6 +124,29 @@ int launch_scatter(fb_ctx* ctx, const fb_pack* pk, const int32_t* page_table, co
   const dim3 grid(c.max_requests * c.wmax, c.n_kv_heads >= 4 ? 4 : 1);
   scatter_window_kv_kernel<<<grid, kScatterThreads, 0, stream>>>(p);
   return cuda_err(ctx, cudaGetLastError(), "scatter_window_kv_kernel launch");
+}
+
+// fb_embed_gather: x[i, :] = table[qtok[i], :] for live rows; one warp per row, 16-byte pieces.
+__global__ void __launch_bounds__(256) embed_gather_kernel(const int32_t* n_live, const int32_t* qtok,
+                                                           const uint4* table, int table_rows, int vec_per_row,
+                                                           uint4* x, int bl, int32_t* status) {
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= *n_live * bl) return;
+  const int tok = qtok[row];
+  if (tok < 0 || tok >= table_rows) { if (lane == 0) atomicOr(status, FB_ST_BAD_TOKEN); return; }
+  const uint4* src = table + (size_t)tok * vec_per_row;
+  uint4* dst = x + (size_t)row * vec_per_row;
+  for (int v = lane; v < vec_per_row; v += 32) dst[v] = src[v];
+}
+
+int launch_embed(fb_ctx* ctx, const fb_pack* pk, const void* table, int table_rows, int hidden, void* x,
+                 int32_t* status, cudaStream_t stream) {
+  const fb_config& c = ctx->cfg;
+  const int rows = c.max_requests * c.wmax * c.block_len;
+  embed_gather_kernel<<<(rows + 7) / 8, 256, 0, stream>>>(pk->n_live, pk->qtok, static_cast<const uint4*>(table),
+                                                        table_rows, hidden / 8, static_cast<uint4*>(x),
+                                                        c.block_len, status);
+  return cuda_err(ctx, cudaGetLastError(), "embed_gather_kernel launch");
 }
 
 }  // namespace fb

@@ -601,3 +601,29 @@ def test_faulty_inputs_set_status_bits_and_nothing_traps():
     keep = np.array([i for i in range(live) if i != 3])
     np.testing.assert_array_equal(sb.argmax.cpu().numpy()[keep], xhat[keep])
     np.testing.assert_allclose(sb.conf.cpu().numpy()[keep], conf[keep], rtol=0, atol=CONF_TOL)
+
+
+@pytest.mark.parametrize("name", ["tiny", "tiny_wide", "cfg1"])
+def test_embed_gather_bit_exact(name):
+    case = make_case(WORKLOADS[name], with_attn=False, with_logits=False)
+    stc = case["stc"]
+    wl = stc.wl
+    ctx, st, pk, sb = gpu_objects(case)
+    hidden = 256
+    table = synth.randn_bf16((wl.vocab, hidden), stc.seed, 12)
+    x = torch.full((ctx.max_slots * wl.block_len, hidden), 7.0, dtype=torch.bfloat16, device=DEV)
+    B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+    B.fb_embed_gather(ctx, pk, table.to(DEV), x, sb.status)
+    torch.cuda.synchronize()
+    assert int(sb.status.item()) == 0
+    ocfg = H.oracle_cfg(stc)
+    opk = O.pack_wavefronts(ocfg, H.oracle_state(stc, case["tokens"]))
+    ref = O.embed_gather(ocfg, opk, H.f64(table))
+    live = opk.n_live * wl.block_len
+    np.testing.assert_array_equal(H.f64(x[:live].cpu()), ref[:live])
+    assert bool((x[live:].float() == 7.0).all())
+    # a table too short for the mask token is reported, nothing is read out of range
+    B.fb_embed_gather(ctx, pk, table[:wl.vocab - 1].contiguous().to(DEV), x, sb.status)
+    torch.cuda.synchronize()
+    has_mask = bool((opk.qtok[:live] == stc.mask_id).any())
+    assert bool(int(sb.status.item()) & B.FB_ST_BAD_TOKEN) == has_mask
