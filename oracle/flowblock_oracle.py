@@ -32,6 +32,9 @@ Pins (tests/test_oracle_*.py, all CPU):
                          window equals attention over the slot-order window;
                          pointer-bump commit equals copy-at-commit
   embed_gather           brute force over (request, block, token)
+  lm_head_rows           one-hot hidden states read the closed-form rows of
+                         t2t_rows back out of the weights; scaling x scales
+                         the logits; permuting the vocabulary permutes argmax
   rope_rotate            textbook special cases (position 0, d = 2 rotation,
                          norm, relative-offset invariance of q.k)
 Nothing in this file is "parity unpinned".
@@ -346,6 +349,19 @@ def t2t_rows(cfg: Config, pk: Pack, logits):
         xhat[i] = int(np.argmax(z))          # numpy returns first occurrence
         conf[i] = 1.0 / np.exp(z - m).sum()
     return xhat, conf
+
+
+def lm_head_rows(cfg: Config, pk: Pack, x, w):
+    """The row pass with the LM head in front of it: logits z = x W^T of the
+    live rows (hidden states x [S*bl, hidden], head weights w [V, hidden], both
+    float64), never rounded to a storage type, then exactly t2t_rows: top-1
+    token (lowest index on ties) and its softmax confidence.  Sec. 3.1 notes
+    that the readiness statistics come "from the current-step logits" at no
+    extra cost; this is that pass taken straight from the head's output."""
+    n = pk.n_live * cfg.block_len
+    logits = np.zeros((cfg.max_slots * cfg.block_len, w.shape[0]), np.float64)
+    logits[:n] = x[:n] @ w.T
+    return t2t_rows(cfg, pk, logits)
 
 
 # --------------------------------------------------------------------------

@@ -127,3 +127,33 @@ def test_embed_gather_brute_force():
                 np.testing.assert_array_equal(x[slot * b + t], table[st.tokens[r, g * b + t]])
             slot += 1
     assert slot == pk.n_live and not x[slot * b:].any()
+
+
+def test_lm_head_rows_closed_forms():
+    wl, stc, cfg, st, pk, q, kw, vw, kp, vp = _case(seed=4)
+    n = pk.n_live * wl.block_len
+    rows, V, hid = cfg.max_slots * wl.block_len, wl.vocab, 16
+    rg = np.random.default_rng(8)
+    # hidden state = unit vector e_0, so the logits of a row are column 0 of the weights:
+    # one entry a, the others 0  ->  p = e^a / (e^a + V - 1)
+    for a in (0.0, 2.0, 5.0):
+        w = np.zeros((V, hid)); w[:, 1:] = rg.normal(size=(V, hid - 1))
+        w[7, 0] = a
+        x = np.zeros((rows, hid)); x[:, 0] = 1.0
+        xhat, conf = O.lm_head_rows(cfg, pk, x, w)
+        want = np.exp(a) / (np.exp(a) + V - 1)
+        np.testing.assert_allclose(conf[:n], want, rtol=1e-12)
+        assert (xhat[:n] == (7 if a > 0 else 0)).all()          # a = 0: V-way tie -> index 0
+        assert (xhat[n:] == -1).all() and not conf[n:].any()
+    # generic inputs: a permutation of the vocabulary permutes the winners, keeps the confidences
+    w = rg.normal(size=(V, hid)) / 4.0
+    x = rg.normal(size=(rows, hid))
+    xhat, conf = O.lm_head_rows(cfg, pk, x, w)
+    perm = rg.permutation(V)
+    xhat2, conf2 = O.lm_head_rows(cfg, pk, x, w[perm])
+    np.testing.assert_array_equal(perm[xhat2[:n]], xhat[:n])
+    np.testing.assert_allclose(conf2[:n], conf[:n], rtol=1e-12)
+    # confidence of the winner against a direct evaluation of one row
+    z = w @ x[3]
+    np.testing.assert_allclose(conf[3], 1.0 / np.exp(z - z.max()).sum(), rtol=1e-12)
+    assert xhat[3] == int(np.argmax(z))
