@@ -241,6 +241,26 @@ int fb_t2t_step(fb_ctx* ctx, const fb_pack* pk, const void* logits,
                 uint8_t* action, int32_t* slot_stats, int32_t* status,
                 void* stream);
 
+/* fb_t2t_step with the LM head in front of it (Sec. 3.1: the readiness
+ * statistics come "from the current-step logits"): the logits z = x W^T are
+ * formed on the tensor cores (bf16 inputs, fp32 accumulation, no rounding to
+ * a storage type) and reduced to top-1 token and confidence tile by tile, so
+ * the [rows, vocab] logits are never written or read back; then Eq. 1 and the
+ * block counts exactly as in fb_t2t_step.
+ *   x       [max_slots*bl, hidden] bf16 hidden states, slot order
+ *   w       [vocab, hidden] bf16 head weights
+ *   hidden  multiple of 64
+ *   ws      fb_lm_head_workspace_bytes(ctx) bytes of device scratch, 16-byte
+ *           aligned (per row and 256-token slice of the vocabulary: max, sum
+ *           of exponentials, first index of the max)
+ * Outputs and state update as in fb_t2t_step. */
+size_t fb_lm_head_workspace_bytes(const fb_ctx* ctx);
+int fb_lm_head_t2t(fb_ctx* ctx, const fb_pack* pk, const void* x,
+                   const void* w, int32_t hidden, const fb_state* st,
+                   int32_t* argmax, float* conf, uint8_t* action,
+                   int32_t* slot_stats, void* ws, int32_t* status,
+                   void* stream);
+
 /* Alg. 1 lines 7-12, Eq. 2-3, Eq. 6 for the committing block: per decoding
  * request retire the maximal locally-finished prefix of its window in order
  * (stopping after a block that holds EOS), copy those blocks' window K/V to

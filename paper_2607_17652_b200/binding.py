@@ -27,7 +27,8 @@ FB_SLOT_STATS, FB_STEP_COUNTERS = 6, 8
 EXPORTS = ["fb_create", "fb_destroy", "fb_last_error", "fb_workspace_bytes",
            "fb_pack_wavefronts", "fb_wavefront_attn", "fb_t2t_step",
            "fb_gate_commit", "fb_step_host", "fb_wavefront_attn_static",
-           "fb_scatter_window_kv", "fb_embed_gather"]
+           "fb_scatter_window_kv", "fb_embed_gather", "fb_lm_head_t2t",
+           "fb_lm_head_workspace_bytes"]
 
 
 class fb_config(C.Structure):
@@ -97,11 +98,16 @@ def lib() -> C.CDLL:
             [C.c_float, P, P]
         l.fb_embed_gather.argtypes = [P, C.POINTER(fb_pack), P, C.c_int32,
                                       C.c_int32, P, P, P]
+        l.fb_lm_head_workspace_bytes.argtypes = [P]
+        l.fb_lm_head_workspace_bytes.restype = C.c_size_t
+        l.fb_lm_head_t2t.argtypes = [P, C.POINTER(fb_pack), P, P, C.c_int32,
+                                     C.POINTER(fb_state)] + [P] * 7
         l.fb_step_host.argtypes = [P, C.POINTER(fb_state), C.POINTER(fb_pack),
                                    C.POINTER(fb_device_bufs),
                                    C.POINTER(fb_host_io), P]
         for n in EXPORTS:
-            if n not in ("fb_last_error", "fb_workspace_bytes"):
+            if n not in ("fb_last_error", "fb_workspace_bytes",
+                         "fb_lm_head_workspace_bytes"):
                 getattr(l, n).restype = I
         _lib = l
     return _lib
@@ -272,6 +278,16 @@ def fb_t2t_step(ctx: Context, pk: PackBuffers, logits, st: DeviceState, argmax,
         ctx.handle, C.byref(p), _ptr(logits), C.byref(s), _ptr(argmax),
         _ptr(conf), _ptr(action), _ptr(slot_stats), _ptr(status),
         _stream(stream)))
+
+
+def fb_lm_head_t2t(ctx: Context, pk: PackBuffers, x, w, st: DeviceState, argmax,
+                   conf, action, slot_stats, ws, status, stream=None):
+    """fb_t2t_step with the LM head fused in front (logits never written)."""
+    s, p = st.c(), pk.c()
+    ctx.check(lib().fb_lm_head_t2t(
+        ctx.handle, C.byref(p), _ptr(x), _ptr(w), int(x.shape[1]), C.byref(s),
+        _ptr(argmax), _ptr(conf), _ptr(action), _ptr(slot_stats), _ptr(ws),
+        _ptr(status), _stream(stream)))
 
 
 def fb_gate_commit(ctx: Context, pk: PackBuffers, slot_stats, st: DeviceState,

@@ -14,7 +14,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 ROOT = os.path.dirname(HERE)
 LIB = os.path.join(HERE, "libflowblock.so")
-SOURCES = ["api.cu", "pack.cu", "t2t.cu", "gate_commit.cu", "attn_sm100.cu", "scatter.cu",
+SOURCES = ["api.cu", "pack.cu", "t2t.cu", "gate_commit.cu", "attn_sm100.cu", "scatter.cu", "lm_head.cu",
            "attn_static.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo",
               "-std=c++17", "-Xcompiler", "-fPIC", "-Xptxas", "-v"]

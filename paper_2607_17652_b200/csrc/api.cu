@@ -190,6 +190,24 @@ int fb_t2t_step(fb_ctx* ctx, const fb_pack* pk, const void* logits, const fb_sta
   return fb::launch_t2t(ctx, pk, logits, st, argmax, conf, action, slot_stats, status, (cudaStream_t)stream);
 }
 
+size_t fb_lm_head_workspace_bytes(const fb_ctx* ctx) { return ctx ? fb::lm_head_workspace_bytes(ctx) : 0; }
+
+int fb_lm_head_t2t(fb_ctx* ctx, const fb_pack* pk, const void* x, const void* w, int32_t hidden,
+                   const fb_state* st, int32_t* argmax, float* conf, uint8_t* action, int32_t* slot_stats,
+                   void* ws, int32_t* status, void* stream) {
+  if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");
+  if (int e = check_pack(ctx, pk)) return e;
+  if (int e = check_state(ctx, st)) return e;
+  if (!x || !w || !argmax || !conf || !action || !slot_stats || !status)
+    return fail(ctx, FB_ERR_INVALID_ARG, "a tensor pointer is null");
+  if (!ws) return fail(ctx, FB_ERR_WORKSPACE, "workspace is null");
+  if (hidden < 64 || hidden % 64 != 0) return fail(ctx, FB_ERR_SHAPE, "hidden must be a positive multiple of 64");
+  if (!aligned16(x) || !aligned16(w) || !aligned16(ws))
+    return fail(ctx, FB_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  return fb::launch_lm_head(ctx, pk, x, w, hidden, st, argmax, conf, action, slot_stats, ws, status,
+                            (cudaStream_t)stream);
+}
+
 int fb_gate_commit(fb_ctx* ctx, const fb_pack* pk, const int32_t* slot_stats, const fb_state* st,
                    const void* k_win, const void* v_win, void* k_pool, void* v_pool, int32_t* n_committed,
                    uint8_t* spawned, int32_t* step_counters, int32_t* status, void* stream) {

@@ -795,7 +795,7 @@ extern "C" int fb_debug_trace(long long* host_out) {
   return (int)cudaMemcpy(host_out, g_trace_ptr, (4 * 8192 + 512) * sizeof(long long), cudaMemcpyDeviceToHost);
 }
 #endif
-static int ensure_device(fb_ctx* ctx) {
+int ensure_device(fb_ctx* ctx) {
   if (ctx->dev_ready) return FB_OK;
   int dev = 0;
   if (int e = cuda_err(ctx, cudaGetDevice(&dev), "cudaGetDevice")) return e;

@@ -74,6 +74,13 @@ int launch_attn(fb_ctx*, const fb_pack*, const void* q, const void* k_win, const
                 void* ws, int32_t* status, cudaStream_t);
 int launch_scatter(fb_ctx*, const fb_pack*, const int32_t* page_table, const void* k_new, const void* v_new,
                    void* k_pool, void* v_pool, float rope_base, int32_t* status, cudaStream_t);
+int ensure_device(fb_ctx*);   // device properties, driver entry point for tensor maps, kernel attributes
+int launch_t2t_update(fb_ctx*, const fb_pack*, const fb_state*, const int32_t* argmax, const float* conf,
+                      uint8_t* action, int32_t* slot_stats, cudaStream_t);
+int launch_lm_head(fb_ctx*, const fb_pack*, const void* x, const void* w, int hidden, const fb_state*,
+                   int32_t* argmax, float* conf, uint8_t* action, int32_t* slot_stats, void* ws, int32_t* status,
+                   cudaStream_t);
+size_t lm_head_workspace_bytes(const fb_ctx*);
 int launch_embed(fb_ctx*, const fb_pack*, const void* table, int table_rows, int hidden, void* x,
                  int32_t* status, cudaStream_t);
 int launch_t2t(fb_ctx*, const fb_pack*, const void* logits, const fb_state*, int32_t* argmax,

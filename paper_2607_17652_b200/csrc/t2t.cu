@@ -192,6 +192,14 @@ int launch_t2t(fb_ctx* ctx, const fb_pack* pk, const void* logits, const fb_stat
   t2t_rows_kernel<<<rows, kRowThreads, 0, stream>>>(static_cast<const uint4*>(logits), pk->n_live, c.block_len,
                                                     c.vocab / 8, argmax, conf, status);
   if (int e = cuda_err(ctx, cudaGetLastError(), "t2t_rows_kernel launch")) return e;
+  return launch_t2t_update(ctx, pk, st, argmax, conf, action, slot_stats, stream);
+}
+
+// Eq. 1 and the block counts from (argmax, conf), whoever produced them.
+int launch_t2t_update(fb_ctx* ctx, const fb_pack* pk, const fb_state* st, const int32_t* argmax, const float* conf,
+                      uint8_t* action, int32_t* slot_stats, cudaStream_t stream) {
+  const fb_config& c = ctx->cfg;
+  const int max_slots = c.max_requests * c.wmax;
   UpdParams u;
   u.n_live = pk->n_live; u.slot_req = pk->slot_req; u.slot_s = pk->slot_s; u.L = st->L; u.tokens = st->tokens;
   u.argmax = argmax; u.conf = conf; u.action = action; u.slot_stats = slot_stats;

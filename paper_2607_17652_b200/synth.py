@@ -286,3 +286,61 @@ def make_logits(stc: Structure, tokens: np.ndarray, kind: str | None = None,
 def to_bits(t: torch.Tensor) -> np.ndarray:
     """bf16 torch tensor -> uint16 bit patterns (numpy, no copy of meaning)."""
     return t.contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def make_lm_head_inputs(stc: Structure, tokens: np.ndarray, hidden: int,
+                        seed_shift: int = 0):
+    """Hidden states x [max_slots*bl, hidden] and LM-head weights w [V, hidden]
+    (bf16) whose logits x w^T look like the "calibrated" logits of
+    :func:`make_logits`: N(0,1) noise, and on 70 % of the live rows a winner
+    token whose softmax confidence is c ~ U(0.5, 0.999), placed by moving the
+    row's hidden state along the winner's weight vector and nudged until, for
+    the bf16-rounded inputs, the confidence is at least 2e-3 away from tau_mask
+    and tau_edit and the winner leads by 0.05.  Revealed positions get the
+    winner or (30 %) another token as current token.  The [M] and EOS rows of
+    w are zero.  Returns (x, w, tokens)."""
+    wl = stc.wl
+    V, b = wl.vocab, wl.block_len
+    rows = wl.max_slots * b
+    seed = stc.seed + 7919 * seed_shift
+    w = randn_bf16((V, hidden), seed, 13, 1.0 / math.sqrt(hidden))
+    w[stc.mask_id] = 0.0
+    w[stc.eos_id] = 0.0
+    x = randn_bf16((rows, hidden), seed, 14)
+    tokens = tokens.copy()
+    rg = _rng(seed, 15)
+    live = _slot_rows(stc)
+    pick = rg.random(rows) < 0.7
+    winners = rg.integers(0, V - 2, size=rows)
+    cs = rg.uniform(0.5, 0.999, size=rows)
+    flip = rg.random(rows) < 0.3
+    thr = (float(np.float32(wl.tau_mask)), float(np.float32(wl.tau_edit)))
+    w64 = w.to(torch.float64)
+    for i in range(min(len(live), rows)):
+        if not pick[i]:
+            continue
+        wi = int(winners[i])
+        dirv = w64[wi] / float(w64[wi] @ w64[wi])            # moves z_w by 1 per unit
+        xi = x[i].to(torch.float64)
+        c = float(cs[i])
+        for _ in range(300):
+            z = w64 @ xi
+            zo = z.clone()
+            zo[wi] = -float("inf")
+            want = math.log(c / (1.0 - c)) + float(torch.logsumexp(zo, 0))
+            cand = (xi + (want - float(z[wi])) * dirv).to(torch.bfloat16).to(torch.float64)
+            z = w64 @ cand
+            zo = z.clone()
+            zo[wi] = -float("inf")
+            p = 1.0 / (1.0 + math.exp(float(torch.logsumexp(zo, 0)) - float(z[wi])))
+            if all(abs(p - t) >= 2e-3 for t in thr) and float(z[wi]) > float(zo.max()) + 0.05:
+                x[i] = cand.to(torch.bfloat16)
+                break
+            c = min(0.9995, c + 0.01) if c < 0.99 else c - 0.013
+        else:
+            raise RuntimeError("could not place a confidence away from the thresholds")
+        r, g, t = live[i]
+        col = g * b + t
+        if tokens[r, col] != stc.mask_id:
+            tokens[r, col] = (wi + 1) % (V - 2) if flip[i] else wi
+    return x, w, tokens

@@ -627,3 +627,41 @@ def test_embed_gather_bit_exact(name):
     torch.cuda.synchronize()
     has_mask = bool((opk.qtok[:live] == stc.mask_id).any())
     assert bool(int(sb.status.item()) & B.FB_ST_BAD_TOKEN) == has_mask
+
+
+# --------------------------------------------- LM head fused with the row pass
+LM_TOL = 5e-5   # fp32 tensor-core accumulation of <= 256 bf16 products per logit against fp64: |dz| < 2e-5
+
+
+@pytest.mark.parametrize("name,hidden", [("tiny", 128), ("tiny_wide", 64), ("tiny_d128_b64", 256)])
+def test_lm_head_fused_row_pass(name, hidden):
+    """Top-1 token and confidence taken from x W^T on the tensor cores, the
+    logits never written: winners bit-exact, confidences within the fp32
+    accumulation error, then Eq. 1, the block counts and gate/commit exactly
+    as with materialised logits."""
+    case = make_case(WORKLOADS[name], with_attn=False, with_logits=False)
+    stc = case["stc"]
+    wl = stc.wl
+    x, w, tokens = synth.make_lm_head_inputs(stc, case["tokens"], hidden)
+    case["tokens"] = tokens
+    ctx, st, pk, sb = gpu_objects(case)
+    ws = torch.zeros(B.lib().fb_lm_head_workspace_bytes(ctx.handle), dtype=torch.uint8, device=DEV)
+    B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+    B.fb_lm_head_t2t(ctx, pk, x.to(DEV), w.to(DEV), st, sb.argmax, sb.conf, sb.action, sb.slot_stats, ws,
+                     sb.status)
+    torch.cuda.synchronize()
+    assert int(sb.status.item()) == 0
+    ocfg = H.oracle_cfg(stc)
+    ost = H.oracle_state(stc, tokens)
+    opk = O.pack_wavefronts(ocfg, ost)
+    xhat, conf = O.lm_head_rows(ocfg, opk, H.f64(x), H.f64(w))
+    live = opk.n_live * wl.block_len
+    for thr in (np.float32(ocfg.tau_mask), np.float32(ocfg.tau_edit)):
+        assert np.abs(conf[:live] - float(thr)).min() >= MARGIN
+    np.testing.assert_array_equal(sb.argmax.cpu().numpy(), xhat)
+    np.testing.assert_allclose(sb.conf.cpu().numpy(), conf, rtol=0, atol=LM_TOL)
+    action, stats = O.t2t_update(ocfg, opk, ost, xhat, conf)
+    np.testing.assert_array_equal(sb.action.cpu().numpy(), action)
+    np.testing.assert_array_equal(sb.slot_stats.cpu().numpy(), stats)
+    np.testing.assert_array_equal(st.tokens.cpu().numpy(), ost.tokens)
+    assert int((action == O.ACT_M2T).sum()) > 0
