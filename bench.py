@@ -19,6 +19,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -278,6 +279,28 @@ def run_ours(args):
                "attn_window_in_pages": {"ms": round(ra_ms, 4),
                                         "tflops": round(attn_flops(device_structure()) / ra_ms / 1e9, 2)}}
         del ctx2, pk2, ws2
+        # next row: the row pass fused into the LM head GEMM (hidden size of a small dLLM; random inputs)
+        hidden = 2048
+        gen = torch.Generator(device=dev); gen.manual_seed(seed + 77)
+        hx = (torch.randn(rows, hidden, device=dev, generator=gen)).to(torch.bfloat16)
+        hw = (torch.randn(wl.vocab, hidden, device=dev, generator=gen) / math.sqrt(hidden)).to(torch.bfloat16)
+        lws = torch.zeros(B.lib().fb_lm_head_workspace_bytes(ctx.handle), dtype=torch.uint8, device=dev)
+        tok_keep = st.tokens.clone()
+        n3 = max(3, min(args.steps, 5))
+        ev3 = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(n3)]
+        for k in range(2 + n3):
+            e = ev3[k - 2] if k >= 2 else None
+            if e: e[0].record(stream)
+            B.fb_lm_head_t2t(ctx, pk, hx, hw, st, sb.argmax, sb.conf, sb.action, sb.slot_stats, lws, sb.status, stream)
+            if e: e[1].record(stream)
+        barrier()
+        st.tokens.copy_(tok_keep)
+        lm_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in ev3]))
+        lm_flops = 2.0 * live_now * wl.block_len * wl.vocab * hidden
+        nxt["lm_head_t2t"] = {"ms": round(lm_ms, 4), "hidden": hidden, "rows": live_now * wl.block_len,
+                              "tflops": round(lm_flops / lm_ms / 1e9, 1),
+                              "logits_bytes_not_moved": 2.0 * live_now * wl.block_len * wl.vocab * 2}
+        del hx, hw, lws
 
     # ------------------------------------------------------------ end to end
     e2e_ms, h2d, d2h = float("nan"), 0, 0
@@ -375,6 +398,7 @@ def run_ours(args):
             "device_status": status, "step_counters": counters,
         }
         if nxt:
+            nxt["lm_head_t2t"]["frac_of_measured_bf16"] = round(nxt["lm_head_t2t"]["tflops"] / peaks["bf16_tflops"], 4)
             nxt["scatter_window_kv"]["frac_of_measured_hbm"] = round(nxt["scatter_window_kv"]["gbs"] / peaks["hbm_gbs"], 4)
             line["next_rows"] = nxt
         if world == 1 and not args.no_cpu_baseline:

@@ -176,3 +176,67 @@ def test_long_context_attention_sampled_requests():
     live = synth.n_live_slots(stc) * wl.block_len
     assert bool(torch.isfinite(sb.out[:live].float()).all())
     assert bool((sb.out[live:].float() == 7.0).all())
+
+
+def test_lm_head_fused_row_pass_full_vocabulary_sampled_rows():
+    """The fused LM head at the benchmark's size (4,768 live rows, V = 151,552,
+    hidden 2048): winners and confidences of sampled rows against the oracle's
+    plain x W^T followed by its row pass; all rows against properties."""
+    wl = synth.WORKLOADS[2]
+    stc = synth.make_structure(wl)
+    tokens = synth.make_tokens(stc)
+    hidden = 2048
+    rows = wl.max_slots * wl.block_len
+    n_live = synth.n_live_slots(stc)
+    live = n_live * wl.block_len
+    w = synth.randn_bf16((wl.vocab, hidden), stc.seed, 13, 1.0 / np.sqrt(hidden))
+    x = synth.randn_bf16((rows, hidden), stc.seed, 14)
+    rg = np.random.default_rng(17)
+    sample = np.sort(rg.choice(live, size=24, replace=False))
+    sample[0], sample[-1] = 0, live - 1                     # first and last live row (ragged last row tile)
+    winners = rg.integers(0, wl.vocab - 2, size=len(sample))
+    for i, wi in zip(sample, winners):                      # a clear winner with a confidence around 0.5-0.95
+        wv = w[wi].to(torch.float64)
+        boost = rg.uniform(12.5, 15.5)
+        x[i] = (x[i].to(torch.float64) + boost * wv / float(wv @ wv)).to(torch.bfloat16)
+    ctx = B.Context(**synth.config_dict(stc))
+    st = B.DeviceState.from_numpy(DEV, stc.active, stc.prefix_len, stc.L, stc.R, tokens,
+                                  np.zeros((wl.n_requests, wl.wmax), np.uint8), stc.page_table)
+    pk = B.PackBuffers.alloc(ctx, DEV)
+    sb = B.StepBuffers(ctx, DEV)
+    ws = torch.zeros(B.lib().fb_lm_head_workspace_bytes(ctx.handle), dtype=torch.uint8, device=DEV)
+    B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+    B.fb_lm_head_t2t(ctx, pk, x.to(DEV), w.to(DEV), st, sb.argmax, sb.conf, sb.action, sb.slot_stats, ws,
+                     sb.status)
+    torch.cuda.synchronize()
+    assert int(sb.status.item()) == 0
+    # oracle on the sampled rows, packed as the live rows of a small problem of its own
+    import dataclasses
+    b = wl.block_len
+    n_slots = (len(sample) + b - 1) // b
+    mini = dataclasses.replace(wl, n_requests=n_slots, wmax=1, w_lo=1, w_hi=1, prefix_lo=0, prefix_hi=0,
+                               max_blocks=2)
+    mstc = synth.make_structure(mini)
+    mcfg = H.oracle_cfg(mstc)
+    mpk = O.pack_wavefronts(mcfg, H.oracle_state(mstc, synth.make_tokens(mstc)))
+    assert mpk.n_live == n_slots
+    xs = np.zeros((n_slots * b, hidden))
+    xs[:len(sample)] = H.f64(x[torch.from_numpy(sample)])
+    # x W^T in slices of the vocabulary (W in fp64 would not fit at once), then the oracle's row pass
+    z_all = []
+    for v0 in range(0, wl.vocab, 16384):
+        z_all.append(xs @ H.f64(w[v0:v0 + 16384]).T)
+    z = np.concatenate(z_all, axis=1)
+    full_logits = np.zeros((mcfg.max_slots * b, wl.vocab))
+    full_logits[:n_slots * b] = z
+    xo, co = O.t2t_rows(mcfg, mpk, full_logits)
+    got_a = sb.argmax.cpu().numpy()[sample]
+    got_c = sb.conf.cpu().numpy()[sample].astype(np.float64)
+    np.testing.assert_array_equal(got_a, xo[:len(sample)])
+    np.testing.assert_array_equal(got_a, winners)
+    assert np.abs(got_c - co[:len(sample)]).max() <= 2e-4, np.abs(got_c - co[:len(sample)]).max()
+    assert co[:len(sample)].min() > 0.05 and co[:len(sample)].max() > 0.9
+    # every live row: a token inside the vocabulary, a probability; padding rows as in fb_t2t_step
+    am, cf = sb.argmax.cpu().numpy(), sb.conf.cpu().numpy()
+    assert ((am[:live] >= 0) & (am[:live] < wl.vocab)).all() and ((cf[:live] > 0) & (cf[:live] <= 1)).all()
+    assert (am[live:] == -1).all() and not cf[live:].any()
