@@ -1,7 +1,8 @@
 // fb_t2t_step: the token-to-token step over the logits (Sec. 2.1, Eq. 1; the
 // counts of Eq. 2).
 //
-// Kernel 1 (bandwidth-bound): one CTA per live row streams the row's bf16
+// Kernel 1 (bandwidth-bound): one CTA (128 threads, eight 16-byte loads in
+// flight each: the best of the shapes tried) per live row streams the row's bf16
 // logits once with 16-byte loads and keeps, per thread, a running
 // (max, first index of the max, sum of exp relative to that max); a
 // warp-shuffle + shared-memory reduction merges them with the lowest-index
@@ -14,8 +15,14 @@
 
 namespace fb {
 
-constexpr int kRowThreads = 256;
-constexpr int kRowUnroll = 4;   // 16-byte loads in flight per thread
+#ifndef FB_T2T_THREADS
+#define FB_T2T_THREADS 128
+#endif
+#ifndef FB_T2T_UNROLL
+#define FB_T2T_UNROLL 8
+#endif
+constexpr int kRowThreads = FB_T2T_THREADS;
+constexpr int kRowUnroll = FB_T2T_UNROLL;   // 16-byte loads in flight per thread
 constexpr float kLog2e = 1.4426950408889634f;
 
 __device__ __forceinline__ uint4 ld_stream16(const uint4* p) {
