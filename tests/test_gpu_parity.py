@@ -633,7 +633,11 @@ def test_embed_gather_bit_exact(name):
 LM_TOL = 5e-5   # fp32 tensor-core accumulation of <= 256 bf16 products per logit against fp64: |dz| < 2e-5
 
 
-@pytest.mark.parametrize("name,hidden", [("tiny", 128), ("tiny_wide", 64), ("tiny_d128_b64", 256)])
+WORKLOADS["tiny_v1000"] = synth.tiny_workload(vocab=1000, n_requests=5, w_lo=1, w_hi=3)   # ragged last vocabulary tile
+
+
+@pytest.mark.parametrize("name,hidden", [("tiny", 128), ("tiny_wide", 64), ("tiny_d128_b64", 256),
+                                         ("tiny_v1000", 192)])
 def test_lm_head_fused_row_pass(name, hidden):
     """Top-1 token and confidence taken from x W^T on the tensor cores, the
     logits never written: winners bit-exact, confidences within the fp32
