@@ -669,3 +669,64 @@ def test_lm_head_fused_row_pass(name, hidden):
     np.testing.assert_array_equal(sb.slot_stats.cpu().numpy(), stats)
     np.testing.assert_array_equal(st.tokens.cpu().numpy(), ost.tokens)
     assert int((action == O.ACT_M2T).sum()) > 0
+
+
+def test_step_host_with_the_window_in_pages():
+    """fb_step_host in a window_in_pages context: scatter, attention over the
+    pages, T2T, pointer-bump commit -- against the same calls made one by one."""
+    wl = synth.tiny_workload(n_requests=4, prefix_lo=30, prefix_hi=260)
+    case = make_case(wl, logits_kind="calibrated", conf_shift=0.25)
+    stc = case["stc"]
+    q, kw, vw, kp, vp = case["attn"]
+    z = case["logits"]
+    ctx, st, pk, sb = gpu_objects(case, window_in_pages=1)
+    dq, dkw, dvw, dkp, dvp, dz = (t.to(DEV) for t in (q, kw, vw, kp, vp, z))
+    B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+    B.fb_scatter_window_kv(ctx, pk, st.page_table, dkw, dvw, dkp, dvp, sb.status)
+    B.fb_wavefront_attn(ctx, pk, dq, None, None, dkp, dvp, st.page_table, sb.out, sb.ws, sb.status)
+    B.fb_t2t_step(ctx, pk, dz, st, sb.argmax, sb.conf, sb.action, sb.slot_stats, sb.status)
+    B.fb_gate_commit(ctx, pk, sb.slot_stats, st, None, None, None, None, sb.n_committed, sb.spawned,
+                     sb.step_counters, sb.status)
+    torch.cuda.synchronize()
+    assert int(sb.status.item()) == 0
+    ctx2, st2, pk2, sb2 = gpu_objects(case, window_in_pages=1)
+    n_rows = synth.n_live_slots(stc) * wl.block_len
+    hkp, hvp = kp.to(DEV), vp.to(DEV)
+    dev = dict(q=torch.zeros_like(dq), k_win=torch.zeros_like(dkw), v_win=torch.zeros_like(dvw), out=sb2.out,
+               logits=torch.zeros_like(dz), k_pool=hkp, v_pool=hvp, argmax=sb2.argmax, conf=sb2.conf,
+               action=sb2.action, slot_stats=sb2.slot_stats, n_committed=sb2.n_committed, spawned=sb2.spawned,
+               step_counters=sb2.step_counters, status=sb2.status, ws=sb2.ws)
+    host = dict(h_q=q.pin_memory(), h_k_win=kw.pin_memory(), h_v_win=vw.pin_memory(), h_logits=z.pin_memory(),
+                h_n_committed=torch.full((wl.n_requests,), -1, dtype=torch.int32).pin_memory(),
+                h_spawned=torch.full((wl.n_requests,), 7, dtype=torch.uint8).pin_memory(),
+                h_step_counters=torch.full((8,), -1, dtype=torch.int32).pin_memory(),
+                h_status=torch.full((1,), -1, dtype=torch.int32).pin_memory(), n_rows=n_rows)
+    B.fb_step_host(ctx2, st2, pk2, dev, host)
+    torch.cuda.synchronize()
+    assert int(host["h_status"][0]) == 0
+    np.testing.assert_array_equal(host["h_n_committed"].numpy(), sb.n_committed.cpu().numpy())
+    np.testing.assert_array_equal(host["h_spawned"].numpy(), sb.spawned.cpu().numpy())
+    np.testing.assert_array_equal(sb2.out[:n_rows].float().cpu().numpy(), sb.out[:n_rows].float().cpu().numpy())
+    a, b2 = st.to_numpy(), st2.to_numpy()
+    for name in ("active", "prefix_len", "L", "R", "tokens", "pe_done"):
+        np.testing.assert_array_equal(a[name], b2[name], err_msg=name)
+    assert torch.equal(hkp, dkp) and torch.equal(hvp, dvp)
+    # and against the oracle: the committed prefix holds what the slot-order path would have copied
+    ocfg = H.oracle_cfg(stc)
+    ost = H.oracle_state(stc, case["tokens"])
+    opk = O.pack_wavefronts(ocfg, ost)
+    okp, ovp = H.f64(kp), H.f64(vp)
+    ref = O.wavefront_attn(ocfg, opk, H.f64(q), H.f64(kw), H.f64(vw), okp, ovp, stc.page_table)
+    max_abs, rel = H.attn_errors(sb2.out, ref, H.live_rows(opk, wl.block_len))
+    assert max_abs <= ATTN_MAX_ABS and rel <= ATTN_REL_L2
+    xhat, conf = O.t2t_rows(ocfg, opk, H.f64(z))
+    action, stats = O.t2t_update(ocfg, opk, ost, xhat, conf)
+    ncom, spawned, ctr = O.gate_commit(ocfg, opk, stats, ost, H.f64(kw), H.f64(vw), okp, ovp)
+    np.testing.assert_array_equal(host["h_n_committed"].numpy(), ncom)
+    ps = wl.page_size
+    gk, gv = H.f64(hkp.cpu()), H.f64(hvp.cpu())
+    for r in range(wl.n_requests):
+        for pos in range(int(ost.prefix_len[r])):
+            page, off = int(stc.page_table[r, pos // ps]), pos % ps
+            np.testing.assert_array_equal(gk[page, :, off], okp[page, :, off])
+            np.testing.assert_array_equal(gv[page, :, off], ovp[page, :, off])
