@@ -428,7 +428,7 @@ def run_sweep(args):
         wl = dataclasses.replace(wl, n_requests=args.requests)
     n_steps = args.steps if args.steps != 20 else 48
     inp = sweep.SweepInputs(wl, n_steps=n_steps)
-    run = sweep.SweepRunner(inp, dev)
+    run = sweep.SweepRunner(inp, dev, window_in_pages=args.window_in_pages)
 
     def one_pass(timed):
         seg, flops, live, committed = [], [], [], 0
@@ -471,7 +471,7 @@ def run_sweep(args):
         "unit": "TFLOP/s (attention FLOPs / whole-step time)",
         "n_gpus": 1, "steps": n_steps, "warmup": n_steps, "ms_per_step": round(total_ms / n_steps, 4),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": wl.name + " (sweep)", "requests": wl.n_requests, "block_len": wl.block_len,
+        "config": {"workload": wl.name + (" (sweep, window in pages)" if args.window_in_pages else " (sweep)"), "requests": wl.n_requests, "block_len": wl.block_len,
                    "wmax": wl.wmax, "slots": wl.max_slots, "live_slots": float(live.mean()),
                    "q_heads": wl.n_q_heads, "kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim,
                    "vocab": wl.vocab, "prefix_range": [wl.prefix_lo, wl.prefix_hi],
@@ -592,6 +592,9 @@ def main():
                     help="time one call only (profiler captures); the JSON line then has no step metric")
     ap.add_argument("--cpu-budget", type=float, default=12.0)
     ap.add_argument("--ref-requests", type=int, default=2)
+    ap.add_argument("--window-in-pages", action="store_true",
+                    help="with --sweep: scatter the window K/V into the pages every step (Eq. 6), attention "
+                         "over the pages, retirement as a pointer bump")
     ap.add_argument("--sweep", action="store_true",
                     help="run the serving workload as a 48-step sequence with arrivals (use with --workload 4)")
     args = ap.parse_args()

@@ -165,10 +165,11 @@ class SweepRunner:
     """Device side of the sweep: state, pools, window tensors, the logits bank
     and the four calls of a step."""
 
-    def __init__(self, inp: SweepInputs, device="cuda:0"):
+    def __init__(self, inp: SweepInputs, device="cuda:0", window_in_pages: bool = False):
         self.inp, self.dev = inp, device
+        self.resident = bool(window_in_pages)
         stc, wl = inp.stc, inp.wl
-        self.ctx = B.Context(**synth.config_dict(stc))
+        self.ctx = B.Context(**synth.config_dict(stc, window_in_pages=int(self.resident)))
         self.st = B.DeviceState.from_numpy(device, stc.active, stc.prefix_len, stc.L, stc.R, inp.tokens0(),
                                            np.zeros((wl.n_requests, wl.wmax), np.uint8), stc.page_table)
         self.pk = B.PackBuffers.alloc(self.ctx, device)
@@ -202,12 +203,18 @@ class SweepRunner:
         ev[0].record()
         B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
         ev[1].record()
-        B.fb_wavefront_attn(ctx, pk, self.q, self.kw, self.vw, self.kp, self.vp, st.page_table, sb.out, sb.ws,
-                            sb.status)
+        if self.resident:      # Eq. 6 every step, attention over the pages
+            B.fb_scatter_window_kv(ctx, pk, st.page_table, self.kw, self.vw, self.kp, self.vp, sb.status)
+            B.fb_wavefront_attn(ctx, pk, self.q, None, None, self.kp, self.vp, st.page_table, sb.out, sb.ws,
+                                sb.status)
+        else:
+            B.fb_wavefront_attn(ctx, pk, self.q, self.kw, self.vw, self.kp, self.vp, st.page_table, sb.out, sb.ws,
+                                sb.status)
         ev[2].record()
         B.fb_t2t_step(ctx, pk, self.z, st, sb.argmax, sb.conf, sb.action, sb.slot_stats, sb.status)
         ev[3].record()
-        B.fb_gate_commit(ctx, pk, sb.slot_stats, st, self.kw, self.vw, self.kp, self.vp, sb.n_committed,
+        kw, vw = (None, None) if self.resident else (self.kw, self.vw)
+        B.fb_gate_commit(ctx, pk, sb.slot_stats, st, kw, vw, self.kp, self.vp, sb.n_committed,
                          sb.spawned, sb.step_counters, sb.status)
         ev[4].record()
         torch.cuda.synchronize()

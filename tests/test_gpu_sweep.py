@@ -38,12 +38,16 @@ def _frozen_kv_matches(run, opk, ost_before, ncom, b):
     return True
 
 
-def test_serving_sweep_states_match_oracle_every_step():
+@pytest.mark.parametrize("window_in_pages", [False, True])
+def test_serving_sweep_states_match_oracle_every_step(window_in_pages):
+    """window_in_pages: the same sequence with the window K/V scattered into the
+    pages every step (Eq. 6) and retirement as a pointer bump; the frozen K/V
+    must come out the same."""
     wl = dataclasses.replace(synth.WORKLOADS[4], vocab=4096)
     n_steps = 48
     # EOS winners from the third block on, so that some requests terminate within the 48 steps
     inp = sweep.SweepInputs(wl, n_steps=n_steps, eos_min_block=2)
-    run = sweep.SweepRunner(inp)
+    run = sweep.SweepRunner(inp, window_in_pages=window_in_pages)
     stc = inp.stc
     b = wl.block_len
     ocfg = H.oracle_cfg(stc)
