@@ -19,13 +19,18 @@ int fail(fb_ctx* ctx, int code, const std::string& msg) {
   return code;
 }
 
-fb::WsLayout make_layout(const fb_config& c, int tiles_per_slot, int target_items) {
+fb::WsLayout make_layout(const fb_config& c, int tiles_per_slot, int target_items, int min_chunk_tiles) {
   fb::WsLayout w{};
   const long long qtiles = (long long)c.max_requests * c.wmax * tiles_per_slot;
   w.max_units = (int)((qtiles + c.max_requests + 1) / 2) * c.n_kv_heads;
-  // split units: at most 2 x target pieces from the coarse split, 1.2 x target more from the filler
-  w.max_items = w.max_units + 3 * target_items + 8;
-  w.max_parts = 4 * target_items + 8;
+  // split units: at most 2 x target pieces from the coarse split, 1.2 x target more from the filler;
+  // and never more than every unit cut into pieces of the minimum length (a unit spans at most the
+  // keys its page-table row can address)
+  const long long max_tiles = ((long long)c.max_pages_per_req * fb::kPage + fb::kTileN - 1) / fb::kTileN + 2;
+  const long long every = (long long)w.max_units * ((max_tiles + min_chunk_tiles - 1) / min_chunk_tiles);
+  const long long by_target = 4ll * target_items + 8;
+  w.max_parts = (int)(by_target < every ? by_target : every);
+  w.max_items = w.max_units + w.max_parts;
   size_t off = 0;
   w.header = off;  off = align_up(off + sizeof(fb::SchedHeader), 256);
   w.items = off;   off = align_up(off + (size_t)w.max_items * sizeof(fb::AttnItem), 256);
@@ -107,7 +112,7 @@ int fb_create(const fb_config* cfg, fb_ctx** out) {
     if (v >= 1 && v <= 4096) ctx->min_chunk_tiles = v;
   }
   ctx->sm_scale = c.sm_scale > 0.f ? c.sm_scale : 1.0f / sqrtf((float)c.head_dim);
-  ctx->ws = make_layout(c, ctx->tiles_per_slot, ctx->target_items);
+  ctx->ws = make_layout(c, ctx->tiles_per_slot, ctx->target_items, ctx->min_chunk_tiles);
   *out = ctx;
   return FB_OK;
 }
