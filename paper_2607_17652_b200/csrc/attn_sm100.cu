@@ -10,19 +10,25 @@
 //               works on one tile while the other is in softmax
 //   warp 3      idle (it completes the control warpgroup, which gives its
 //               registers to the softmax warpgroups with setmaxnreg)
-//   warps 4-7   softmax of tile A, one thread per query row: tcgen05.ld S (once
-//               for the row max, once more in 32-column chunks for the
-//               exponentials), lazy rescale of O, exp2 (part of it as a
-//               polynomial on the FMA pipe), P (bf16) written back over S in
-//               TMEM, epilogue
+//   warps 4-7   softmax of tile A, one thread per query row: tcgen05.ld of S in
+//               32-column chunks, exp2 against a lazily re-based reference
+//               (only the first tile of an item takes a max pass; part of the
+//               exponentials runs as a polynomial on the FMA pipe), P (bf16)
+//               kept in registers until the tile is known to be in range, then
+//               written back over S in TMEM; epilogue
 //   warps 8-11  the same for tile B
 // A Q tile is 128 rows = (128/G tokens) x (G query heads of one KV head) of one
-// slot.  A unit pairs two Q tiles of one request and KV head so that they
-// share each K/V tile from shared memory.  The mask is per tile: a tile of the
-// frozen prefix is fully visible except the ragged last one; the window tile
-// is visible up to (s+1)*bl keys for a query in window slot s.  Tiles nobody
-// can see are never loaded (the work list only spans visible tiles), and
-// ragged tiles run the MMAs on ceil(valid/16)*16 keys only.
+// slot.  A unit runs two Q tiles side by side: two tiles of one request and KV
+// head, which share each K/V tile from shared memory, or the odd tile left
+// over, run under two adjacent KV heads at once (two K/V streams, served in
+// readiness order).  The mask is per tile: a tile of the frozen prefix is
+// fully visible except the ragged last one; the window tile is visible up to
+// (s+1)*bl keys for a query in window slot s.  Tiles nobody can see are never
+// loaded (the work list only spans visible tiles), and ragged tiles run the
+// MMAs on ceil(valid/16)*16 keys only.  With the window resident in the pages
+// every key tile is a paged one over absolute positions.
+// Work items are sorted longest first by the pack kernel and drawn by the CTAs
+// from a global ticket.
 // Long key ranges are split across CTAs; partial (max, sum, O) go to the
 // workspace and a second kernel merges them in a fixed order.
 #include <cudaTypedefs.h>
