@@ -52,6 +52,8 @@ constexpr int kSmem128 = 6 * 32768 + 8192;
 #ifdef FB_TRACE
 #if FB_TRACE == 2      // light: one event per key tile from the MMA warp only
 #define FB_TR_ON(role, tag) ((role) == 1 && (tag) == 20)
+#elif FB_TRACE == 3    // tile A's softmax warps: tile boundaries and the epilogue
+#define FB_TR_ON(role, tag) ((role) == 2 && ((tag) >= 50 || (tag) == 41 || (tag) == 46))
 #else
 #define FB_TR_ON(role, tag) true
 #endif
@@ -687,13 +689,12 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           tmem_ld32(tO + c * 32, o);
           tmem_ld_wait();
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            uint4 v;
-            v.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv, __uint_as_float(o[8 * i + 1]) * inv);
-            v.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv);
-            v.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv, __uint_as_float(o[8 * i + 5]) * inv);
-            v.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv, __uint_as_float(o[8 * i + 7]) * inv);
-            dst[c * 4 + i] = v;
+          for (int i = 0; i < 2; ++i) {              // two 32-byte stores: whole sectors
+            uint32_t v[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              v[k] = pack_bf16x2(__uint_as_float(o[16 * i + 2 * k]) * inv, __uint_as_float(o[16 * i + 2 * k + 1]) * inv);
+            st_global_v8(dst + c * 4 + 2 * i, v);
           }
         }
       } else {
