@@ -40,7 +40,7 @@ KERNELS_PER_STEP = 6   # pack, attention, split-KV combine, T2T rows, T2T update
 # under profiles/, as a ratio to the algorithmic bytes of the captured (smaller)
 # case of the same workload; a full launch's traffic is that ratio times its
 # algorithmic bytes (traffic grows in proportion to the requests processed).
-NCU_TRAFFIC_RATIO = {("attn", 2): (1379.1 + 33.8) / 1366.9,   # profiles/wavefront_attn_cfg2_dram.txt (full size)
+NCU_TRAFFIC_RATIO = {("attn", 2): (1397.7 + 33.5) / 1366.9,   # profiles/wavefront_attn_cfg2_dram.txt (full size)
                      ("t2t", 2): (504.38 + 4.62) / 504.4}      # profiles/t2t_rows_cfg2_16req.txt
 
 
