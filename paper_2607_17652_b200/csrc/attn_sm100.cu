@@ -220,6 +220,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  pdl_wait();                     // the work list (and everything else) of the previous kernels is complete
   const int n_items = p.hdr->n_items;
 #ifdef FB_TRACE
   if (tid == 0) { unsigned long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); p.trace[4 * 8192 + 2 * blockIdx.x] = (long long)g; }
@@ -739,6 +740,7 @@ constexpr int kCombineSplit = 8;
 constexpr int kCombineCtasPerSm = 4;
 template <int D>
 __global__ void __launch_bounds__(256) attn_combine_kernel(const AttnParams p) {
+  pdl_wait();
   if (p.hdr->n_parts == 0) return;
   const int n_pieces = p.hdr->n_units * kCombineSplit;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -899,15 +901,19 @@ int launch_attn(fb_ctx* ctx, const fb_pack* pk, const void* q, const void* k_win
   const int grid = ctx->num_sms;
   const int combine_grid = min(ctx->ws.max_units * kCombineSplit, kCombineCtasPerSm * ctx->num_sms);
   if (c.head_dim == 64) {
-    wavefront_attn_kernel<64><<<grid, kAttnThreads, kSmem64, stream>>>(
-        ctx->tm_q, ctx->tm_kwin, ctx->tm_vwin, ctx->tm_kpool, ctx->tm_vpool, p);
-    if (int e = cuda_err(ctx, cudaGetLastError(), "wavefront_attn_kernel launch")) return e;
-    attn_combine_kernel<64><<<combine_grid, 256, 0, stream>>>(p);
+    if (int e = cuda_err(ctx, launch_pdl(wavefront_attn_kernel<64>, grid, kAttnThreads, kSmem64, stream, ctx->tm_q,
+                                         ctx->tm_kwin, ctx->tm_vwin, ctx->tm_kpool, ctx->tm_vpool, p),
+                         "wavefront_attn_kernel launch"))
+      return e;
+    return cuda_err(ctx, launch_pdl(attn_combine_kernel<64>, combine_grid, 256, 0, stream, p),
+                    "attn_combine_kernel launch");
   } else {
-    wavefront_attn_kernel<128><<<grid, kAttnThreads, kSmem128, stream>>>(
-        ctx->tm_q, ctx->tm_kwin, ctx->tm_vwin, ctx->tm_kpool, ctx->tm_vpool, p);
-    if (int e = cuda_err(ctx, cudaGetLastError(), "wavefront_attn_kernel launch")) return e;
-    attn_combine_kernel<128><<<combine_grid, 256, 0, stream>>>(p);
+    if (int e = cuda_err(ctx, launch_pdl(wavefront_attn_kernel<128>, grid, kAttnThreads, kSmem128, stream, ctx->tm_q,
+                                         ctx->tm_kwin, ctx->tm_vwin, ctx->tm_kpool, ctx->tm_vpool, p),
+                         "wavefront_attn_kernel launch"))
+      return e;
+    return cuda_err(ctx, launch_pdl(attn_combine_kernel<128>, combine_grid, 256, 0, stream, p),
+                    "attn_combine_kernel launch");
   }
   return cuda_err(ctx, cudaGetLastError(), "attn_combine_kernel launch");
 }

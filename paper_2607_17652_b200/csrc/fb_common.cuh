@@ -68,6 +68,29 @@ struct fb_ctx {
 
 namespace fb {
 
+// Launch with programmatic stream serialisation: the kernel may be scheduled while its
+// predecessor in the stream is still running and runs up to its pdl_wait() (barrier set-up, TMEM
+// allocation, descriptor prefetch); everything after pdl_wait() sees the predecessor complete.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#ifdef __CUDACC__
+// Lets the next kernel of the stream be scheduled, then waits for the previous one to be complete
+// (a no-op pair when the kernel was launched the ordinary way).
+__device__ __forceinline__ void pdl_wait() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+#endif
+
 int launch_pack(fb_ctx*, const fb_state*, const fb_pack*, void* ws, int32_t* status, cudaStream_t);
 int launch_attn(fb_ctx*, const fb_pack*, const void* q, const void* k_win, const void* v_win,
                 const void* k_pool, const void* v_pool, const int32_t* page_table, void* out,

@@ -28,6 +28,7 @@ struct GateParams {
 };
 
 __global__ void __launch_bounds__(kGateThreads) gate_commit_kernel(const GateParams p) {
+  pdl_wait();
   const int r = blockIdx.x;
   const int tid = threadIdx.x;
   __shared__ int s_c, s_first, s_P, s_done, s_spawn, s_newR;
@@ -143,7 +144,7 @@ int launch_gate(fb_ctx* ctx, const fb_pack* pk, const int32_t* slot_stats, const
   if (int e = cuda_err(ctx, cudaMemsetAsync(step_counters, 0, FB_STEP_COUNTERS * sizeof(int32_t), stream),
                        "clear step counters"))
     return e;
-  gate_commit_kernel<<<c.max_requests, kGateThreads, 0, stream>>>(p);
+  if (int e = cuda_err(ctx, launch_pdl(gate_commit_kernel, c.max_requests, kGateThreads, 0, stream, p), "gate_commit_kernel launch")) return e;
   return cuda_err(ctx, cudaGetLastError(), "gate_commit_kernel launch");
 }
 

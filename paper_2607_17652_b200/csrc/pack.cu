@@ -251,6 +251,7 @@ __device__ void build_sched(const PackParams& p) {
 }
 
 __global__ void __launch_bounds__(kPackThreads) pack_kernel(const PackParams p) {
+  pdl_wait();
   if ((int)blockIdx.x == p.n_gather_blocks) { build_sched(p); return; }
   __shared__ int sh_scan[kPackThreads / 32 + 1];
   __shared__ int s_req[kSlotsPerBlock], s_idx[kSlotsPerBlock], s_w[kSlotsPerBlock];
@@ -324,8 +325,7 @@ int launch_pack(fb_ctx* ctx, const fb_state* st, const fb_pack* out, void* ws, i
   p.resident = ctx->cfg.window_in_pages;
   p.max_items = ctx->ws.max_items; p.max_units = ctx->ws.max_units; p.max_parts = ctx->ws.max_parts;
   p.n_gather_blocks = (p.max_slots + kSlotsPerBlock - 1) / kSlotsPerBlock;
-  pack_kernel<<<p.n_gather_blocks + 1, kPackThreads, 0, stream>>>(p);
-  return cuda_err(ctx, cudaGetLastError(), "pack_kernel launch");
+  return cuda_err(ctx, launch_pdl(pack_kernel, p.n_gather_blocks + 1, kPackThreads, 0, stream, p), "pack_kernel launch");
 }
 
 }  // namespace fb

@@ -80,6 +80,7 @@ __device__ __forceinline__ void absorb8(RowAcc& a, const uint4 v, int base) {
 __global__ void __launch_bounds__(kRowThreads)
 t2t_rows_kernel(const uint4* __restrict__ logits, const int32_t* __restrict__ n_live, int bl, int nvec,
                 int32_t* __restrict__ argmax, float* __restrict__ conf, int32_t* __restrict__ status) {
+  pdl_wait();
   const int row = blockIdx.x;
   const int tid = threadIdx.x;
   if (row >= *n_live * bl) {            // padding slot: no bytes read
@@ -145,6 +146,7 @@ struct UpdParams {
 };
 
 __global__ void __launch_bounds__(128) t2t_update_kernel(const UpdParams p) {
+  pdl_wait();
   const int slot = blockIdx.x * 4 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (slot >= p.max_slots) return;
@@ -196,9 +198,10 @@ int launch_t2t(fb_ctx* ctx, const fb_pack* pk, const void* logits, const fb_stat
   const fb_config& c = ctx->cfg;
   const int max_slots = c.max_requests * c.wmax;
   const int rows = max_slots * c.block_len;
-  t2t_rows_kernel<<<rows, kRowThreads, 0, stream>>>(static_cast<const uint4*>(logits), pk->n_live, c.block_len,
-                                                    c.vocab / 8, argmax, conf, status);
-  if (int e = cuda_err(ctx, cudaGetLastError(), "t2t_rows_kernel launch")) return e;
+  if (int e = cuda_err(ctx, launch_pdl(t2t_rows_kernel, rows, kRowThreads, 0, stream, static_cast<const uint4*>(logits),
+                                       pk->n_live, c.block_len, c.vocab / 8, argmax, conf, status),
+                       "t2t_rows_kernel launch"))
+    return e;
   return launch_t2t_update(ctx, pk, st, argmax, conf, action, slot_stats, stream);
 }
 
@@ -212,8 +215,7 @@ int launch_t2t_update(fb_ctx* ctx, const fb_pack* pk, const fb_state* st, const 
   u.argmax = argmax; u.conf = conf; u.action = action; u.slot_stats = slot_stats;
   u.max_slots = max_slots; u.bl = c.block_len; u.max_blocks = c.max_blocks; u.mask_id = c.mask_id;
   u.eos_id = c.eos_id; u.tau_mask = c.tau_mask; u.tau_edit = c.tau_edit;
-  t2t_update_kernel<<<(max_slots + 3) / 4, 128, 0, stream>>>(u);
-  return cuda_err(ctx, cudaGetLastError(), "t2t_update_kernel launch");
+  return cuda_err(ctx, launch_pdl(t2t_update_kernel, (max_slots + 3) / 4, 128, 0, stream, u), "t2t_update_kernel launch");
 }
 
 }  // namespace fb
