@@ -10,7 +10,7 @@
 
 namespace fb {
 
-constexpr int kGateThreads = 256;
+constexpr int kGateThreads = 512;
 
 struct GateParams {
   const int32_t *n_live, *req_slot_begin, *slot_stats;
@@ -107,18 +107,32 @@ __global__ void __launch_bounds__(kGateThreads) gate_commit_kernel(const GatePar
   const int vec_per_tok = p.n_kv_heads * vec_per_head;
   // (window resident in the pages: nothing to copy, the prefix pointer has moved over it)
   const int total = p.k_win ? c * p.bl * vec_per_tok : 0;
-  for (int i = tid; i < total; i += kGateThreads) {
-    const int tok = i / vec_per_tok, rem = i % vec_per_tok;
-    const int h = rem / vec_per_head, v = rem % vec_per_head;
-    const int apos = P + tok;
-    const int pidx = apos / kPage;
-    if (pidx >= p.max_pages_per_req) { atomicOr(p.status, FB_ST_BAD_PAGE); continue; }
-    const int page = p.page_table[r * p.max_pages_per_req + pidx];
-    if (page < 0 || page >= p.num_pages) { atomicOr(p.status, FB_ST_BAD_PAGE); continue; }
-    const size_t src = (size_t)(first * p.bl + tok) * vec_per_tok + rem;
-    const size_t dst = (((size_t)page * p.n_kv_heads + h) * kPage + apos % kPage) * vec_per_head + v;
-    p.k_pool[dst] = p.k_win[src];
-    p.v_pool[dst] = p.v_win[src];
+  // four pieces per thread and pass, all loads issued before the first store (source and
+  // destination never overlap: window tensors against the page pool)
+  constexpr int kBatch = 4;
+  for (int i0 = tid; i0 < total; i0 += kBatch * kGateThreads) {
+    uint4 kv[kBatch], vv[kBatch];
+    size_t dst[kBatch];
+#pragma unroll
+    for (int j = 0; j < kBatch; ++j) {
+      const int i = i0 + j * kGateThreads;
+      dst[j] = ~(size_t)0;
+      if (i >= total) continue;
+      const int tok = i / vec_per_tok, rem = i % vec_per_tok;
+      const int h = rem / vec_per_head, v = rem % vec_per_head;
+      const int apos = P + tok;
+      const int pidx = apos / kPage;
+      if (pidx >= p.max_pages_per_req) { atomicOr(p.status, FB_ST_BAD_PAGE); continue; }
+      const int page = p.page_table[r * p.max_pages_per_req + pidx];
+      if (page < 0 || page >= p.num_pages) { atomicOr(p.status, FB_ST_BAD_PAGE); continue; }
+      const size_t src = (size_t)(first * p.bl + tok) * vec_per_tok + rem;
+      dst[j] = (((size_t)page * p.n_kv_heads + h) * kPage + apos % kPage) * vec_per_head + v;
+      kv[j] = p.k_win[src];
+      vv[j] = p.v_win[src];
+    }
+#pragma unroll
+    for (int j = 0; j < kBatch; ++j)
+      if (dst[j] != ~(size_t)0) { p.k_pool[dst[j]] = kv[j]; p.v_pool[dst[j]] = vv[j]; }
   }
   // the admitted block starts fully masked
   if (s_spawn) {

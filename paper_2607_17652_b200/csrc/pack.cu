@@ -8,8 +8,8 @@
 
 namespace fb {
 
-constexpr int kPackThreads = 256;
-constexpr int kSlotsPerBlock = 8;
+constexpr int kPackThreads = 1024;
+constexpr int kSlotsPerBlock = 32;
 constexpr int kCostBins = 1024;
 
 struct PackParams {
@@ -89,15 +89,15 @@ struct ReqGeom {
   int w, ntq, npairs, P, npt, nt;
   int nfull, odd, nunits;   // full pairs per KV head; leftover tile; units of the request
 };
-__device__ __forceinline__ ReqGeom req_geom(const PackParams& p, int r, int32_t* status) {
+__device__ __forceinline__ ReqGeom geom_of(const PackParams& p, int w, int prefix_len) {
   ReqGeom g;
-  g.w = live_blocks(p, r, status);
+  g.w = w;
   g.ntq = g.w * p.tiles_per_slot;
   g.npairs = (g.ntq + 1) >> 1;
   g.nfull = g.ntq >> 1;
   g.odd = g.ntq & 1;
   g.nunits = g.nfull * p.n_kv_heads + g.odd * ((p.n_kv_heads + 1) >> 1);
-  g.P = g.w ? max(p.prefix_len[r], 0) : 0;
+  g.P = g.w ? max(prefix_len, 0) : 0;
   g.npt = (g.P + kTileN - 1) / kTileN;
   g.nt = g.w ? g.npt + (g.w * p.bl + kTileN - 1) / kTileN : 0;
   if (p.resident) {       // one run of keys [0, P + w*bl), all of it paged
@@ -105,6 +105,10 @@ __device__ __forceinline__ ReqGeom req_geom(const PackParams& p, int r, int32_t*
     g.npt = g.nt;
   }
   return g;
+}
+__device__ __forceinline__ ReqGeom req_geom(const PackParams& p, int r, int32_t* status) {
+  const int w = live_blocks(p, r, status);
+  return geom_of(p, w, w ? p.prefix_len[r] : 0);
 }
 
 __device__ void build_sched(const PackParams& p) {
@@ -146,7 +150,10 @@ __device__ void build_sched(const PackParams& p) {
   }
   __syncthreads();
   const int Ct = sh_ct, fineCt = sh_fine_ct, fineFrom = sh_fine_from;
-  // phase 2 + 3: per-request bases (chunked scan), units, cost histogram
+  // phase 2 + 3: per-request bases (chunked scan), then one thread per unit of the chunk's
+  // requests: unit record, cost histogram of its items
+  __shared__ int s_ub[kPackThreads + 1], s_pb[kPackThreads], s_first[kPackThreads], s_nch[kPackThreads],
+      s_w[kPackThreads], s_P[kPackThreads];
   int unit_run = 0, part_run = 0, item_run = 0, slot_run = 0, work_run = 0;
   for (int r0 = 0; r0 < p.max_requests; r0 += kPackThreads) {
     const int r = r0 + tid;
@@ -159,69 +166,85 @@ __device__ void build_sched(const PackParams& p) {
     int tu, tp, ti, ts, tw;
     const int wbase = work_run + block_excl_scan(nunits * g.nt, &tw, sh_scan);
     work_run += tw;
-    if (g.nt) nch = (g.nt + (wbase + nunits * g.nt > fineFrom ? fineCt : Ct) - 1) / (wbase + nunits * g.nt > fineFrom ? fineCt : Ct);
-    const int ubase = unit_run + block_excl_scan(nunits, &tu, sh_scan);
+    if (g.nt) {
+      const int len = wbase + nunits * g.nt > fineFrom ? fineCt : Ct;
+      nch = (g.nt + len - 1) / len;
+    }
+    const int urel = block_excl_scan(nunits, &tu, sh_scan);
     const int pbase = part_run + block_excl_scan(nch > 1 ? nunits * nch : 0, &tp, sh_scan);
     block_excl_scan(nunits * nch, &ti, sh_scan);
-    const int first = slot_run + block_excl_scan(g.w, &ts, sh_scan);  // first slot of the request
-    unit_run += tu; part_run += tp; item_run += ti; slot_run += ts;
-    if (r < p.max_requests && nunits) {
-      for (int ul = 0; ul < g.nunits; ++ul) {
-        // Full pairs first, numbered h * nfull + pr: the pairs of one (request, KV head) are
-        // adjacent, are handed out back to back and so share their K/V through L2.  Then the
-        // leftover tile, one unit per two KV heads.
-        const int u = ubase + ul;
-        if (u >= p.max_units) continue;
-        const bool full = ul < g.nfull * p.n_kv_heads;
-        const int h = full ? ul / g.nfull : 2 * (ul - g.nfull * p.n_kv_heads);
-        const int qa = full ? 2 * (ul % g.nfull) : g.ntq - 1;
-        AttnUnit un;
-        un.req = r;
-        const int sA = qa / p.tiles_per_slot;
-        un.slotA = first + sA;
-        un.t0A = (qa % p.tiles_per_slot) * p.tokens_per_tile;
-        un.winA = (sA + 1) * p.bl;
-        un.nvisA = p.resident ? (g.P + un.winA + kTileN - 1) / kTileN : g.npt + (un.winA + kTileN - 1) / kTileN;
-        if (full) {
-          const int qb = qa + 1;
-          const int sB = qb / p.tiles_per_slot;
-          un.kvh = h | (h << 16);
-          un.slotB = first + sB;
-          un.t0B = (qb % p.tiles_per_slot) * p.tokens_per_tile;
-          un.winB = (sB + 1) * p.bl;
-          un.nvisB = p.resident ? (g.P + un.winB + kTileN - 1) / kTileN : g.npt + (un.winB + kTileN - 1) / kTileN;
-        } else if (h + 1 < p.n_kv_heads) {
-          un.kvh = h | ((h + 1) << 16);
-          un.slotB = un.slotA; un.t0B = un.t0A; un.winB = un.winA; un.nvisB = un.nvisA;
-        } else {
-          un.kvh = h | (h << 16);
-          un.slotB = -1; un.t0B = 0; un.winB = 0; un.nvisB = 0;
-        }
-        un.n_tiles = g.nt; un.n_chunks = nch;
-        un.part_base = nch > 1 ? pbase + ul * nch : -1;
-        if (nch > 1 && un.part_base + nch > p.max_parts) un.n_chunks = 0;  // cannot happen; see header
-        un.prefix_len = g.P; un.npt = g.npt; un.win_row0 = first * p.bl;
-        p.units[u] = un;
-        for (int c = 0; c < un.n_chunks; ++c) {
-          const int jb = c * g.nt / nch, je = (c + 1) * g.nt / nch;
-          int cost = item_cost(max(0, min(je, un.nvisA) - jb), max(0, min(je, un.nvisB) - jb));
-          atomicAdd(&bins[min(cost, kCostBins - 1)], 1);
-        }
+    const int first0 = slot_run + block_excl_scan(g.w, &ts, sh_scan);  // first slot of the request
+    s_ub[tid] = urel; s_pb[tid] = pbase; s_first[tid] = first0; s_nch[tid] = nch; s_w[tid] = g.w; s_P[tid] = g.P;
+    if (tid == 0) s_ub[kPackThreads] = tu;
+    __syncthreads();
+    for (int i = tid; i < tu; i += kPackThreads) {
+      // the request of unit i: the last k with s_ub[k] <= i (requests without units share
+      // their successor's base and are skipped by "last")
+      int lo = 0, hi = kPackThreads - 1;
+      while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (s_ub[mid] <= i) lo = mid; else hi = mid - 1;
+      }
+      const int k = lo, ul = i - s_ub[k];
+      const int u = unit_run + i;
+      if (u >= p.max_units) continue;
+      const ReqGeom q = geom_of(p, s_w[k], s_P[k]);
+      const int first = s_first[k], nc = s_nch[k];
+      // Full pairs first, numbered h * nfull + pr: the pairs of one (request, KV head) are
+      // adjacent, are handed out back to back and so share their K/V through L2.  Then the
+      // leftover tile, one unit per two KV heads.
+      const bool full = ul < q.nfull * p.n_kv_heads;
+      const int h = full ? ul / q.nfull : 2 * (ul - q.nfull * p.n_kv_heads);
+      const int qa = full ? 2 * (ul % q.nfull) : q.ntq - 1;
+      AttnUnit un;
+      un.req = r0 + k;
+      const int sA = qa / p.tiles_per_slot;
+      un.slotA = first + sA;
+      un.t0A = (qa % p.tiles_per_slot) * p.tokens_per_tile;
+      un.winA = (sA + 1) * p.bl;
+      un.nvisA = p.resident ? (q.P + un.winA + kTileN - 1) / kTileN : q.npt + (un.winA + kTileN - 1) / kTileN;
+      if (full) {
+        const int qb = qa + 1;
+        const int sB = qb / p.tiles_per_slot;
+        un.kvh = h | (h << 16);
+        un.slotB = first + sB;
+        un.t0B = (qb % p.tiles_per_slot) * p.tokens_per_tile;
+        un.winB = (sB + 1) * p.bl;
+        un.nvisB = p.resident ? (q.P + un.winB + kTileN - 1) / kTileN : q.npt + (un.winB + kTileN - 1) / kTileN;
+      } else if (h + 1 < p.n_kv_heads) {
+        un.kvh = h | ((h + 1) << 16);
+        un.slotB = un.slotA; un.t0B = un.t0A; un.winB = un.winA; un.nvisB = un.nvisA;
+      } else {
+        un.kvh = h | (h << 16);
+        un.slotB = -1; un.t0B = 0; un.winB = 0; un.nvisB = 0;
+      }
+      un.n_tiles = q.nt; un.n_chunks = nc;
+      un.part_base = nc > 1 ? s_pb[k] + ul * nc : -1;
+      if (nc > 1 && un.part_base + nc > p.max_parts) un.n_chunks = 0;  // cannot happen; see header
+      un.prefix_len = q.P; un.npt = q.npt; un.win_row0 = first * p.bl;
+      p.units[u] = un;
+      for (int c = 0; c < un.n_chunks; ++c) {
+        const int jb = c * q.nt / nc, je = (c + 1) * q.nt / nc;
+        int cost = item_cost(max(0, min(je, un.nvisA) - jb), max(0, min(je, un.nvisB) - jb));
+        atomicAdd(&bins[min(cost, kCostBins - 1)], 1);
       }
     }
+    unit_run += tu; part_run += tp; item_run += ti; slot_run += ts;
+    __syncthreads();                      // the chunk's tables are overwritten next
   }
   __syncthreads();
-  // descending exclusive offsets over the cost bins: thread t owns the four
-  // bins kCostBins-1-4t .. kCostBins-4-4t (largest cost first)
+  // descending exclusive offsets over the cost bins: thread t owns the bins
+  // kCostBins-1-kBinsPer*t and below (largest cost first)
   {
-    static_assert(kCostBins == 4 * kPackThreads, "four bins per thread");
-    int c[4], sum = 0;
+    constexpr int kBinsPer = kCostBins / kPackThreads;
+    static_assert(kBinsPer * kPackThreads == kCostBins && kBinsPer >= 1, "whole bins per thread");
+    int c[kBinsPer], sum = 0;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) { c[j] = bins[kCostBins - 1 - (4 * tid + j)]; sum += c[j]; }
+    for (int j = 0; j < kBinsPer; ++j) { c[j] = bins[kCostBins - 1 - (kBinsPer * tid + j)]; sum += c[j]; }
     int total_items;
     int base = block_excl_scan(sum, &total_items, sh_scan);
 #pragma unroll
-    for (int j = 0; j < 4; ++j) { bins[kCostBins - 1 - (4 * tid + j)] = base; base += c[j]; }
+    for (int j = 0; j < kBinsPer; ++j) { bins[kCostBins - 1 - (kBinsPer * tid + j)] = base; base += c[j]; }
     if (tid == 0) {
       p.hdr->n_items = min(total_items, p.max_items);
       p.hdr->n_units = min(unit_run, p.max_units);
