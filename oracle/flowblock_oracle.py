@@ -27,6 +27,10 @@ Pins (tests/test_oracle_*.py, all CPU):
   gate_commit            hand-worked Alg. 1 cases; window of one block equals
                          an independently written serial block-wise decoder;
                          packed run equals per-request runs
+  gate_commit_batch_sync one sequence: equal to gate_commit (Sec. 4.5: "at
+                         B = 1 the two are semantically identical"); copies of
+                         one sequence: equal to gate_commit; hand-worked
+                         straggler, EOS and min-rho cases; lockstep invariant
   scatter_window_kv      brute-force placement (every live window position, no
                          other pool element); attention over the page-resident
                          window equals attention over the slot-order window;
@@ -58,7 +62,8 @@ ACT_T2T = 2         # revealed position overwritten (set Delta of Eq. 1)
 ST_M0, ST_RDY, ST_M2T, ST_T2T, ST_M1, ST_EOS = range(6)
 # step_counters entries
 (CT_BLOCKS, CT_TOKENS, CT_SPAWNED, CT_FINISHED, CT_M2T, CT_T2T,
- CT_LIVE_SLOTS, CT_ACTIVE) = range(8)
+ CT_LIVE_SLOTS, CT_ACTIVE, CT_LOCKSTEP_COMMIT, CT_LOCKSTEP_ADMIT) = range(10)
+N_COUNTERS = 10
 
 
 @dataclass
@@ -81,6 +86,7 @@ class Config:
     tau_edit: float = 0.95
     theta_spawn: float = 0.5
     sm_scale: float = 0.0     # 0 -> 1/sqrt(head_dim); READING: paper silent
+    batch_sync: int = 0       # 1: the batch-synchronous wavefront of Sec. 3.2 / 4.5
 
     @property
     def max_slots(self) -> int:
@@ -446,11 +452,14 @@ def gate_commit(cfg: Config, pk: Pack, stats, st: State, k_win=None,
     block admitted now has no current-step logits; the frontier is block R-1
     as it was in this forward, even if it has just retired; an empty window
     counts as rho = 1.  The new block is all [M].
-    Returns (n_committed int32 [R], spawned uint8 [R], counters int32 [8])."""
+    Returns (n_committed int32 [R], spawned uint8 [R], counters int32 [10])."""
+    if cfg.batch_sync:
+        return gate_commit_batch_sync(cfg, pk, stats, st, k_win, v_win,
+                                      k_pool, v_pool)
     b, ps, W = cfg.block_len, cfg.page_size, cfg.wmax
     n_committed = np.zeros(cfg.max_requests, np.int32)
     spawned = np.zeros(cfg.max_requests, np.uint8)
-    ctr = np.zeros(8, np.int32)
+    ctr = np.zeros(N_COUNTERS, np.int32)
     ctr[CT_LIVE_SLOTS] = pk.n_live
     theta = np.float32(cfg.theta_spawn)
     for r in range(cfg.max_requests):
@@ -499,6 +508,95 @@ def gate_commit(cfg: Config, pk: Pack, stats, st: State, k_win=None,
             rho = np.float32(1.0)
         if (rho >= theta and st.R[r] - st.L[r] < W
                 and st.R[r] < cfg.max_blocks):
+            g = int(st.R[r])
+            st.tokens[r, g * b:(g + 1) * b] = cfg.mask_id
+            st.R[r] += 1
+            st.pe_done[r, int(st.R[r] - st.L[r]) - 1] = 0
+            spawned[r] = 1
+            ctr[CT_SPAWNED] += 1
+    ctr[CT_ACTIVE] = int((st.active == 1).sum())
+    return n_committed, spawned, ctr
+
+
+def gate_commit_batch_sync(cfg: Config, pk: Pack, stats, st: State,
+                           k_win=None, v_win=None, k_pool=None, v_pool=None):
+    """The batch-synchronous wavefront that Sec. 3.2 and the packing ablation
+    (Sec. 4.5) set against per-sequence wavefronts: the same per-block
+    predicates, but window position c retires only when it is finished in
+    EVERY sequence still in the batch (``finished.all()``) and a block is
+    admitted only when min_b rho_b clears theta_spawn.
+
+    READING: the sequences keep their own (L_r, R_r) and move them together,
+    which is the shared [L, R) whenever they start equal.  A sequence whose
+    retired block holds EOS is done and leaves the reductions at once; the
+    cascade goes on for the others.  The admission needs every remaining
+    sequence to clear the gate and to have room (R - L < W, R < n): all of
+    them get one new block or none does.  With one sequence this is
+    gate_commit itself.  counters[CT_LOCKSTEP_COMMIT] = window positions
+    retired by the batch this step, counters[CT_LOCKSTEP_ADMIT] = 1 if the
+    batch admitted."""
+    b, ps, W = cfg.block_len, cfg.page_size, cfg.wmax
+    n_committed = np.zeros(cfg.max_requests, np.int32)
+    spawned = np.zeros(cfg.max_requests, np.uint8)
+    ctr = np.zeros(N_COUNTERS, np.int32)
+    ctr[CT_LIVE_SLOTS] = pk.n_live
+    theta = np.float32(cfg.theta_spawn)
+    batch = [r for r in range(cfg.max_requests) if st.active[r] == 1]
+    first, width, pe_new, fin = {}, {}, {}, {}
+    for r in batch:
+        first[r] = int(pk.req_slot_begin[r])
+        width[r] = int(pk.req_slot_begin[r + 1]) - first[r]
+        assert width[r] == int(st.R[r]) - int(st.L[r])
+        pe_new[r], fin[r] = [], []
+        for s in range(width[r]):
+            m0, rdy, a, e, m1, _ = (int(v) for v in stats[first[r] + s])
+            pn = min(255, int(st.pe_done[r, s]) + (1 if m0 == 0 else 0))
+            pe_new[r].append(pn)
+            fin[r].append(locally_finished(cfg, m0, m1, a + e, pn))
+            ctr[CT_M2T] += a
+            ctr[CT_T2T] += e
+    # retire window position c in every sequence, or in none
+    alive, done = list(batch), []
+    c = 0
+    while alive and all(c < width[r] and fin[r][c] for r in alive):
+        for r in alive:
+            if k_win is not None:
+                P = int(st.prefix_len[r])
+                for t in range(b):
+                    page = int(st.page_table[r, (P + t) // ps])
+                    k_pool[page, :, (P + t) % ps, :] = k_win[(first[r] + c) * b + t]
+                    v_pool[page, :, (P + t) % ps, :] = v_win[(first[r] + c) * b + t]
+            st.L[r] += 1
+            st.prefix_len[r] += b
+            n_committed[r] += 1
+            if stats[first[r] + c, ST_EOS] or st.L[r] == cfg.max_blocks:
+                done.append(r)
+        alive = [r for r in alive if r not in done]
+        c += 1
+    ctr[CT_LOCKSTEP_COMMIT] = c
+    for r in batch:
+        k = int(n_committed[r])
+        for s in range(W):
+            st.pe_done[r, s] = pe_new[r][s + k] if s + k < width[r] else 0
+        ctr[CT_BLOCKS] += k
+        ctr[CT_TOKENS] += k * b
+    for r in done:
+        st.active[r] = 2
+        ctr[CT_FINISHED] += 1
+    # one admission decision for the batch
+    left = [r for r in batch if r not in done]
+
+    def clears(r):
+        w = width[r]
+        rho = (readiness(int(stats[first[r] + w - 1, ST_M0]),
+                         int(stats[first[r] + w - 1, ST_RDY]))
+               if w > 0 else np.float32(1.0))
+        return bool(rho >= theta and st.R[r] - st.L[r] < W
+                    and st.R[r] < cfg.max_blocks)
+
+    if left and all(clears(r) for r in left):
+        ctr[CT_LOCKSTEP_ADMIT] = 1
+        for r in left:
             g = int(st.R[r])
             st.tokens[r, g * b:(g + 1) * b] = cfg.mask_id
             st.R[r] += 1
