@@ -319,7 +319,7 @@ def run_ours(args):
         host = dict(h_q=hq, h_k_win=hkw, h_v_win=hvw, h_logits=hz,
                     h_n_committed=torch.zeros(wl.n_requests, dtype=torch.int32).pin_memory(),
                     h_spawned=torch.zeros(wl.n_requests, dtype=torch.uint8).pin_memory(),
-                    h_step_counters=torch.zeros(8, dtype=torch.int32).pin_memory(),
+                    h_step_counters=torch.zeros(B.FB_STEP_COUNTERS, dtype=torch.int32).pin_memory(),
                     h_status=torch.zeros(1, dtype=torch.int32).pin_memory(),
                     n_rows=synth.n_live_slots(stc1) * wl.block_len)
         devb = dict(q=q, k_win=kw, v_win=vw, out=sb.out, logits=logits, k_pool=kp, v_pool=vp,

@@ -66,7 +66,9 @@ enum { FB_STAT_M0 = 0, FB_STAT_RDY, FB_STAT_M2T, FB_STAT_T2T, FB_STAT_M1, FB_STA
 /* step_counters entries */
 enum { FB_CT_BLOCKS = 0, FB_CT_TOKENS, FB_CT_SPAWNED, FB_CT_FINISHED,
        FB_CT_M2T, FB_CT_T2T, FB_CT_LIVE_SLOTS, FB_CT_ACTIVE,
-       FB_STEP_COUNTERS = 8 };
+       FB_CT_LOCKSTEP_COMMIT, /* batch_sync: window positions the batch retired */
+       FB_CT_LOCKSTEP_ADMIT,  /* batch_sync: 1 if the batch admitted a block    */
+       FB_STEP_COUNTERS = 10 };
 
 typedef struct fb_ctx fb_ctx;
 
@@ -98,6 +100,14 @@ typedef struct {
                                 every step (fb_scatter_window_kv, Eq. 6), the
                                 attention reads every key through the page
                                 table and retirement copies nothing          */
+  int32_t batch_sync;        /* 0: per-sequence wavefronts (Sec. 3.2).  1: the
+                                batch-synchronous wavefront that Sec. 3.2 and
+                                the packing ablation set against them: window
+                                position c retires only when it is finished in
+                                every decoding sequence, and one block per
+                                sequence is admitted only when every sequence
+                                clears the gate (min over the batch of rho)
+                                and has room                                 */
 } fb_config;
 
 /* Per-request wavefront state (Sec. 3.2: (L_b, R_b), in-order commit
@@ -270,11 +280,16 @@ int fb_lm_head_t2t(fb_ctx* ctx, const fb_pack* pk, const void* x,
  * R - L < W and R < n.
  *   n_committed   [R_max] int32 blocks retired this step
  *   spawned       [R_max] uint8
- *   step_counters [8] int32 (FB_CT_*), overwritten
+ *   step_counters [FB_STEP_COUNTERS] int32 (FB_CT_*), overwritten
  * Mutates st->{active, prefix_len, L, R, tokens (new block), pe_done} and the
  * pool pages of committed blocks; frozen positions are never rewritten.
  * With window_in_pages = 1 nothing is copied (k_win, v_win, k_pool, v_pool
- * may be NULL): advancing prefix_len freezes what the scatter put in place. */
+ * may be NULL): advancing prefix_len freezes what the scatter put in place.
+ * With batch_sync = 1 the same per-block predicates feed two reductions over
+ * the decoding sequences first: a sequence retires min(its own finished
+ * prefix, the batch's), where a sequence that terminates (committed EOS, or
+ * L == n) stops counting once its last block is out; then all remaining
+ * sequences admit one block, or none does.  One extra single-CTA launch. */
 int fb_gate_commit(fb_ctx* ctx, const fb_pack* pk, const int32_t* slot_stats,
                    const fb_state* st, const void* k_win, const void* v_win,
                    void* k_pool, void* v_pool, int32_t* n_committed,

@@ -555,8 +555,11 @@ def gate_commit_batch_sync(cfg: Config, pk: Pack, stats, st: State,
             fin[r].append(locally_finished(cfg, m0, m1, a + e, pn))
             ctr[CT_M2T] += a
             ctr[CT_T2T] += e
-    # retire window position c in every sequence, or in none
-    alive, done = list(batch), []
+    # retire window position c in every sequence, or in none.  (A sequence
+    # handed in with L == n already has nothing left: it is done at once, as
+    # in gate_commit, and holds nobody back.)
+    done = [r for r in batch if st.L[r] == cfg.max_blocks]
+    alive = [r for r in batch if r not in done]
     c = 0
     while alive and all(c < width[r] and fin[r][c] for r in alive):
         for r in alive:

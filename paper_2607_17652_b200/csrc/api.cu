@@ -92,6 +92,8 @@ int fb_create(const fb_config* cfg, fb_ctx** out) {
     return fail(nullptr, FB_ERR_UNSUPPORTED, "tau_edit < tau_mask is not supported");
   if (c.window_in_pages != 0 && c.window_in_pages != 1)
     return fail(nullptr, FB_ERR_INVALID_ARG, "window_in_pages must be 0 or 1");
+  if (c.batch_sync != 0 && c.batch_sync != 1)
+    return fail(nullptr, FB_ERR_INVALID_ARG, "batch_sync must be 0 or 1");
   if ((long long)c.max_requests * c.wmax * c.block_len > (1ll << 24))
     return fail(nullptr, FB_ERR_UNSUPPORTED, "max_requests * wmax * block_len is too large");
   fb_ctx* ctx = new (std::nothrow) fb_ctx();

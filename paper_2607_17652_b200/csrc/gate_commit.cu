@@ -5,7 +5,9 @@
 // the per-slot counts; all threads then copy the retiring blocks' window K/V
 // rows into the request's pages with 16-byte accesses; thread 0 publishes the
 // new state.  Requests are independent, so no inter-CTA ordering is needed;
-// the step counters are integer atomics on a zeroed array.
+// the step counters are integer atomics on a zeroed array.  The batch-synchronous
+// variant (fb_config.batch_sync) adds a single-CTA kernel in front that reduces the
+// per-request results over the batch into two of the counters, which every CTA here reads.
 #include "fb_common.cuh"
 
 namespace fb {
@@ -25,7 +27,89 @@ struct GateParams {
   int32_t max_requests, wmax, bl, max_blocks, mask_id, s_pe, n_kv_heads, head_dim, num_pages,
       max_pages_per_req;
   float theta_spawn;
+  int32_t batch_sync;
 };
+
+// What a request's own block counts say (Alg. 1 l.7-9 before any batch rule): its window,
+// the post-edit counters after this forward, the finished prefix c (stopping after a block
+// that holds EOS), and whether retiring those c blocks ends the request.
+struct ReqEval {
+  int first, w, L, R, c;
+  bool ok, eos, ends;
+  uint8_t pe_new[8];
+  int m2t, t2t;
+};
+__device__ __forceinline__ ReqEval eval_request(const GateParams& p, int r) {
+  ReqEval e;
+  e.first = p.req_slot_begin[r];
+  e.w = p.req_slot_begin[r + 1] - e.first;
+  e.L = p.L[r]; e.R = p.R[r];
+  e.c = 0; e.eos = false; e.ends = false; e.m2t = 0; e.t2t = 0;
+  e.ok = !(e.w != e.R - e.L || e.w < 0 || e.w > p.wmax);
+  if (!e.ok) return e;
+  bool fin[8];
+  for (int s = 0; s < e.w; ++s) {
+    const int32_t* st = p.slot_stats + (e.first + s) * FB_SLOT_STATS;
+    const int m0 = st[FB_STAT_M0], m1 = st[FB_STAT_M1], nupd = st[FB_STAT_M2T] + st[FB_STAT_T2T];
+    int pn = p.pe_done[r * p.wmax + s] + (m0 == 0 ? 1 : 0);
+    pn = pn > 255 ? 255 : pn;
+    e.pe_new[s] = (uint8_t)pn;
+    // locally finished (Sec. 2.1): no masks left, and either a quiet
+    // post-edit forward or the S_pe budget is used up
+    fin[s] = m1 == 0 && ((m0 == 0 && nupd == 0) || pn >= p.s_pe);
+    e.m2t += st[FB_STAT_M2T]; e.t2t += st[FB_STAT_T2T];
+  }
+  while (e.c < e.w && fin[e.c]) {                    // Alg. 1 l.7-9, in order
+    ++e.c;
+    if (p.slot_stats[(e.first + e.c - 1) * FB_SLOT_STATS + FB_STAT_EOS]) { e.eos = true; break; }
+  }
+  e.ends = e.eos || e.L + e.c == p.max_blocks;
+  return e;
+}
+// Eq. 2 on the frontier block as it went into this forward; Eq. 3 with the window bounds
+// after c blocks have retired
+__device__ __forceinline__ bool clears_gate(const GateParams& p, const ReqEval& e, int c) {
+  float rho = 1.0f;
+  if (e.w > 0) {
+    const int32_t* st = p.slot_stats + (e.first + e.w - 1) * FB_SLOT_STATS;
+    if (st[FB_STAT_M0] != 0) rho = __fdiv_rn((float)st[FB_STAT_RDY], (float)st[FB_STAT_M0]);
+  }
+  return rho >= p.theta_spawn && e.R - (e.L + c) < p.wmax && e.R < p.max_blocks;
+}
+
+// batch_sync: the two reductions over the decoding sequences (Sec. 3.2: finished.all(),
+// min_b rho_b), one CTA, before any state is touched.  A sequence that ends with its own
+// finished prefix never holds the others back beyond it; if every sequence ends, each
+// retires its own prefix.
+__global__ void __launch_bounds__(kGateThreads) gate_batch_reduce_kernel(const GateParams p) {
+  pdl_wait();
+  __shared__ int s_min, s_max, s_all;
+  if (threadIdx.x == 0) { s_min = 0x7fffffff; s_max = 0; s_all = 1; }
+  __syncthreads();
+  for (int r = threadIdx.x; r < p.max_requests; r += kGateThreads) {
+    if (p.active[r] != 1) continue;
+    const ReqEval e = eval_request(p, r);
+    if (!e.ok) { atomicMin(&s_min, 0); continue; }   // pack and state disagree: nothing retires
+    if (e.ends) atomicMax(&s_max, e.c); else atomicMin(&s_min, e.c);
+  }
+  __syncthreads();
+  const int C = s_min != 0x7fffffff ? s_min : s_max;
+  int left = 0;
+  for (int r = threadIdx.x; r < p.max_requests; r += kGateThreads) {
+    if (p.active[r] != 1) continue;
+    const ReqEval e = eval_request(p, r);
+    if (!e.ok) { atomicAnd(&s_all, 0); continue; }
+    const int c = min(e.c, C);
+    if (e.ends && c == e.c) continue;                // done: no longer part of the batch
+    left = 1;
+    if (!clears_gate(p, e, c)) atomicAnd(&s_all, 0);
+  }
+  const int any_left = __syncthreads_or(left);
+  if (threadIdx.x == 0) {
+    p.counters[FB_CT_LOCKSTEP_COMMIT] = C;
+    p.counters[FB_CT_LOCKSTEP_ADMIT] = any_left && s_all;
+  }
+}
 
 __global__ void __launch_bounds__(kGateThreads) gate_commit_kernel(const GateParams p) {
   pdl_wait();
@@ -38,66 +122,37 @@ __global__ void __launch_bounds__(kGateThreads) gate_commit_kernel(const GatePar
     return;
   }
   if (tid == 0) {
-    const int first = p.req_slot_begin[r];
-    int w = p.req_slot_begin[r + 1] - first;
-    int L = p.L[r], R = p.R[r];
-    if (w != R - L || w < 0 || w > p.wmax) {       // pack and state disagree: leave the request alone
+    const ReqEval e = eval_request(p, r);
+    if (!e.ok) {                                   // pack and state disagree: leave the request alone
       atomicOr(p.status, FB_ST_BAD_STATE);
-      s_c = 0; s_spawn = 0; s_first = first; s_P = 0; s_newR = R;
+      s_c = 0; s_spawn = 0; s_first = e.first; s_P = 0; s_newR = e.R;
       p.n_committed[r] = 0; p.spawned[r] = 0;
-      w = -1;
-    }
-    if (w >= 0) {
-    uint8_t pe_new[8];
-    bool fin[8];
-    int m2t = 0, t2t = 0;
-    for (int s = 0; s < w; ++s) {
-      const int32_t* st = p.slot_stats + (first + s) * FB_SLOT_STATS;
-      const int m0 = st[FB_STAT_M0], m1 = st[FB_STAT_M1], nupd = st[FB_STAT_M2T] + st[FB_STAT_T2T];
-      int pn = p.pe_done[r * p.wmax + s] + (m0 == 0 ? 1 : 0);
-      pn = pn > 255 ? 255 : pn;
-      pe_new[s] = (uint8_t)pn;
-      // locally finished (Sec. 2.1): no masks left, and either a quiet
-      // post-edit forward or the S_pe budget is used up
-      fin[s] = m1 == 0 && ((m0 == 0 && nupd == 0) || pn >= p.s_pe);
-      m2t += st[FB_STAT_M2T]; t2t += st[FB_STAT_T2T];
-    }
-    int c = 0;
-    bool eos = false;
-    while (c < w && fin[c]) {                      // Alg. 1 l.7-9, in order
-      ++c;
-      if (p.slot_stats[(first + c - 1) * FB_SLOT_STATS + FB_STAT_EOS]) { eos = true; break; }
-    }
-    const int P = p.prefix_len[r];
-    s_c = c; s_first = first; s_P = P;
-    L += c;
-    for (int s = 0; s < p.wmax; ++s) p.pe_done[r * p.wmax + s] = s + c < w ? pe_new[s + c] : 0;
-    const bool done = eos || L == p.max_blocks;
-    int spawn = 0;
-    if (!done) {
-      // Eq. 2 on the frontier block as it went into this forward; Eq. 3
-      float rho = 1.0f;
-      if (w > 0) {
-        const int32_t* st = p.slot_stats + (first + w - 1) * FB_SLOT_STATS;
-        if (st[FB_STAT_M0] != 0) rho = __fdiv_rn((float)st[FB_STAT_RDY], (float)st[FB_STAT_M0]);
+    } else {
+      // batch_sync: the batch's retire count caps the sequence's own; a block holding EOS
+      // terminates only if it is among the blocks that do retire
+      const int c = p.batch_sync ? min(e.c, p.counters[FB_CT_LOCKSTEP_COMMIT]) : e.c;
+      const int w = e.w, R = e.R, L = e.L + c;
+      const int P = p.prefix_len[r];
+      s_c = c; s_first = e.first; s_P = P;
+      for (int s = 0; s < p.wmax; ++s) p.pe_done[r * p.wmax + s] = s + c < w ? e.pe_new[s + c] : 0;
+      const bool done = (c == e.c && e.eos) || L == p.max_blocks;
+      int spawn = 0;
+      if (!done) spawn = p.batch_sync ? p.counters[FB_CT_LOCKSTEP_ADMIT] : (int)clears_gate(p, e, c);
+      s_done = done; s_spawn = spawn; s_newR = R;
+      p.L[r] = L;
+      p.prefix_len[r] = P + c * p.bl;
+      p.n_committed[r] = c;
+      p.spawned[r] = (uint8_t)spawn;
+      if (done) p.active[r] = 2;
+      if (spawn) {
+        p.R[r] = R + 1;
+        p.pe_done[r * p.wmax + (R + 1 - L) - 1] = 0;
       }
-      if (rho >= p.theta_spawn && R - L < p.wmax && R < p.max_blocks) spawn = 1;
-    }
-    s_done = done; s_spawn = spawn; s_newR = R;
-    p.L[r] = L;
-    p.prefix_len[r] = P + c * p.bl;
-    p.n_committed[r] = c;
-    p.spawned[r] = (uint8_t)spawn;
-    if (done) p.active[r] = 2;
-    if (spawn) {
-      p.R[r] = R + 1;
-      p.pe_done[r * p.wmax + (R + 1 - L) - 1] = 0;
-    }
-    if (c) { atomicAdd(&p.counters[FB_CT_BLOCKS], c); atomicAdd(&p.counters[FB_CT_TOKENS], c * p.bl); }
-    if (spawn) atomicAdd(&p.counters[FB_CT_SPAWNED], 1);
-    if (done) atomicAdd(&p.counters[FB_CT_FINISHED], 1); else atomicAdd(&p.counters[FB_CT_ACTIVE], 1);
-    if (m2t) atomicAdd(&p.counters[FB_CT_M2T], m2t);
-    if (t2t) atomicAdd(&p.counters[FB_CT_T2T], t2t);
+      if (c) { atomicAdd(&p.counters[FB_CT_BLOCKS], c); atomicAdd(&p.counters[FB_CT_TOKENS], c * p.bl); }
+      if (spawn) atomicAdd(&p.counters[FB_CT_SPAWNED], 1);
+      if (done) atomicAdd(&p.counters[FB_CT_FINISHED], 1); else atomicAdd(&p.counters[FB_CT_ACTIVE], 1);
+      if (e.m2t) atomicAdd(&p.counters[FB_CT_M2T], e.m2t);
+      if (e.t2t) atomicAdd(&p.counters[FB_CT_T2T], e.t2t);
     }
   }
   __syncthreads();
@@ -158,6 +213,11 @@ int launch_gate(fb_ctx* ctx, const fb_pack* pk, const int32_t* slot_stats, const
   if (int e = cuda_err(ctx, cudaMemsetAsync(step_counters, 0, FB_STEP_COUNTERS * sizeof(int32_t), stream),
                        "clear step counters"))
     return e;
+  p.batch_sync = c.batch_sync;
+  if (c.batch_sync)
+    if (int e = cuda_err(ctx, launch_pdl(gate_batch_reduce_kernel, 1, kGateThreads, 0, stream, p),
+                         "gate_batch_reduce_kernel launch"))
+      return e;
   if (int e = cuda_err(ctx, launch_pdl(gate_commit_kernel, c.max_requests, kGateThreads, 0, stream, p), "gate_commit_kernel launch")) return e;
   return cuda_err(ctx, cudaGetLastError(), "gate_commit_kernel launch");
 }

@@ -165,11 +165,13 @@ class SweepRunner:
     """Device side of the sweep: state, pools, window tensors, the logits bank
     and the four calls of a step."""
 
-    def __init__(self, inp: SweepInputs, device="cuda:0", window_in_pages: bool = False):
+    def __init__(self, inp: SweepInputs, device="cuda:0", window_in_pages: bool = False,
+                 batch_sync: bool = False, **cfg_over):
         self.inp, self.dev = inp, device
         self.resident = bool(window_in_pages)
         stc, wl = inp.stc, inp.wl
-        self.ctx = B.Context(**synth.config_dict(stc, window_in_pages=int(self.resident)))
+        self.ctx = B.Context(**synth.config_dict(stc, window_in_pages=int(self.resident),
+                                                 batch_sync=int(bool(batch_sync)), **cfg_over))
         self.st = B.DeviceState.from_numpy(device, stc.active, stc.prefix_len, stc.L, stc.R, inp.tokens0(),
                                            np.zeros((wl.n_requests, wl.wmax), np.uint8), stc.page_table)
         self.pk = B.PackBuffers.alloc(self.ctx, device)

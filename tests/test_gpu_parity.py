@@ -199,6 +199,73 @@ def test_t2t_and_gate_commit_bit_exact(name, kind, shift, s_pe):
         assert res["ncom"].sum() >= 0
 
 
+@pytest.mark.parametrize("name,shift,s_pe", [("tiny", 0.3, 0), ("tiny_wide", 0.2, 1),
+                                             ("tiny_d128_b64", 0.1, 3)])
+def test_t2t_and_batch_synchronous_gate_bit_exact(name, shift, s_pe):
+    """The whole step with fb_config.batch_sync = 1 (Sec. 3.2: all()-gated
+    retirement, min-rho admission)."""
+    case = make_case(WORKLOADS[name], logits_kind="calibrated", conf_shift=shift)
+    run_t2t_and_gate(case, s_pe=s_pe, batch_sync=1)
+
+
+@pytest.mark.parametrize("batch_sync", [0, 1])
+@pytest.mark.parametrize("seed", range(12))
+def test_gate_commit_on_drawn_block_counts(seed, batch_sync):
+    """fb_gate_commit alone on block counts drawn from a menu (finished,
+    finished with EOS, half ready, a quarter ready, fully masked) over drawn
+    windows, so that cascades, committed EOS, sequences running out of blocks,
+    stragglers and every admission outcome occur; per-sequence and
+    batch-synchronous policy, bit-exact against the oracle, K/V freeze included."""
+    rg = np.random.default_rng(500 + seed)
+    Rn, W, n = int(rg.integers(1, 10)), int(rg.integers(1, 5)), 6
+    wl = synth.tiny_workload(n_requests=Rn, wmax=W, w_lo=1, w_hi=W, max_blocks=n,
+                             n_q_heads=8, n_kv_heads=2, prefix_lo=0, prefix_hi=90)
+    case = make_case(wl, seed=900 + seed, with_logits=False)
+    stc = case["stc"]
+    b = wl.block_len
+    # windows anywhere in [0, n], some empty, some touching n, some requests idle or done
+    for r in range(Rn):
+        L = int(rg.integers(0, n + 1))
+        stc.L[r] = L
+        stc.R[r] = min(n, L + int(rg.integers(0, W + 1)))
+        stc.active[r] = rg.choice([0, 1, 1, 1, 1, 2])
+    if seed % 4 == 0:                      # a shared window: the ablation's own setting
+        stc.L[:] = 2; stc.R[:] = min(n, 2 + W); stc.active[:] = 1
+    over = dict(batch_sync=batch_sync, s_pe=int(rg.integers(0, 3)),
+                theta_spawn=float(rg.choice([0.25, 0.5, 0.6])))
+    ctx, st, pk, sb = gpu_objects(case, **over)
+    pe0 = rg.integers(0, 3, size=(Rn, W)).astype(np.uint8)
+    st.pe_done.copy_(torch.from_numpy(pe0))
+    q, kw, vw, kp, vp = (t.to(DEV) for t in case["attn"])
+    B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+    torch.cuda.synchronize()
+    ocfg = H.oracle_cfg(stc, **over)
+    ost = H.oracle_state(stc, case["tokens"])
+    ost.pe_done[:] = pe0
+    opk = O.pack_wavefronts(ocfg, ost)
+    menu = np.array([(0, 0, 0, 0, 0, 0), (0, 0, 0, 0, 0, 1), (b, b // 2, 0, 0, b, 0),
+                     (b, b // 4, 0, 0, b, 0), (b, 0, 0, 0, b, 0), (3, 3, 3, 0, 0, 0),
+                     (0, 0, 0, 2, 0, 0)], np.int32)
+    weights = [0.45, 0.08, 0.12, 0.1, 0.1, 0.1, 0.05]
+    stats = np.zeros((ctx.max_slots, 6), np.int32)
+    stats[:opk.n_live] = menu[rg.choice(len(menu), size=opk.n_live, p=weights)]
+    sb.slot_stats.copy_(torch.from_numpy(stats))
+    B.fb_gate_commit(ctx, pk, sb.slot_stats, st, kw, vw, kp, vp, sb.n_committed, sb.spawned,
+                     sb.step_counters, sb.status)
+    torch.cuda.synchronize()
+    okw, ovw, okp, ovp = (H.f64(t) for t in case["attn"][1:])
+    ncom, spawned, ctr = O.gate_commit(ocfg, opk, stats, ost, okw, ovw, okp, ovp)
+    np.testing.assert_array_equal(sb.n_committed.cpu().numpy(), ncom)
+    np.testing.assert_array_equal(sb.spawned.cpu().numpy(), spawned)
+    np.testing.assert_array_equal(sb.step_counters.cpu().numpy(), ctr)
+    g = st.to_numpy()
+    for name in ("active", "prefix_len", "L", "R", "tokens", "pe_done"):
+        np.testing.assert_array_equal(g[name], getattr(ost, name), err_msg=name)
+    np.testing.assert_array_equal(H.f64(kp.cpu()), okp)
+    np.testing.assert_array_equal(H.f64(vp.cpu()), ovp)
+    assert int(sb.status.item()) == 0
+
+
 def test_t2t_full_vocab_rows():
     """V = 151,552 rows: many tiles per row, bf16 ties, peaked rows."""
     wl = dataclasses.replace(synth.WORKLOADS[1], n_requests=2, name="cfg1_2req")
@@ -455,7 +522,7 @@ def test_step_host_equals_the_four_calls():
     host = dict(h_q=q.pin_memory(), h_k_win=kw.pin_memory(), h_v_win=vw.pin_memory(), h_logits=z.pin_memory(),
                 h_n_committed=torch.full((wl.n_requests,), -1, dtype=torch.int32).pin_memory(),
                 h_spawned=torch.full((wl.n_requests,), 7, dtype=torch.uint8).pin_memory(),
-                h_step_counters=torch.full((8,), -1, dtype=torch.int32).pin_memory(),
+                h_step_counters=torch.full((B.FB_STEP_COUNTERS,), -1, dtype=torch.int32).pin_memory(),
                 h_status=torch.full((1,), -1, dtype=torch.int32).pin_memory(), n_rows=n_rows)
     B.fb_step_host(ctx2, st2, pk2, dev, host)
     torch.cuda.synchronize()
@@ -699,7 +766,7 @@ def test_step_host_with_the_window_in_pages():
     host = dict(h_q=q.pin_memory(), h_k_win=kw.pin_memory(), h_v_win=vw.pin_memory(), h_logits=z.pin_memory(),
                 h_n_committed=torch.full((wl.n_requests,), -1, dtype=torch.int32).pin_memory(),
                 h_spawned=torch.full((wl.n_requests,), 7, dtype=torch.uint8).pin_memory(),
-                h_step_counters=torch.full((8,), -1, dtype=torch.int32).pin_memory(),
+                h_step_counters=torch.full((B.FB_STEP_COUNTERS,), -1, dtype=torch.int32).pin_memory(),
                 h_status=torch.full((1,), -1, dtype=torch.int32).pin_memory(), n_rows=n_rows)
     B.fb_step_host(ctx2, st2, pk2, dev, host)
     torch.cuda.synchronize()

@@ -38,19 +38,20 @@ def _frozen_kv_matches(run, opk, ost_before, ncom, b):
     return True
 
 
-@pytest.mark.parametrize("window_in_pages", [False, True])
-def test_serving_sweep_states_match_oracle_every_step(window_in_pages):
+@pytest.mark.parametrize("window_in_pages,batch_sync", [(False, False), (True, False), (False, True)])
+def test_serving_sweep_states_match_oracle_every_step(window_in_pages, batch_sync):
     """window_in_pages: the same sequence with the window K/V scattered into the
     pages every step (Eq. 6) and retirement as a pointer bump; the frozen K/V
-    must come out the same."""
+    must come out the same.  batch_sync: the batch-synchronous wavefront of the
+    packing ablation on a static batch (every request there at step 0)."""
     wl = dataclasses.replace(synth.WORKLOADS[4], vocab=4096)
     n_steps = 48
     # EOS winners from the third block on, so that some requests terminate within the 48 steps
-    inp = sweep.SweepInputs(wl, n_steps=n_steps, eos_min_block=2)
-    run = sweep.SweepRunner(inp, window_in_pages=window_in_pages)
+    inp = sweep.SweepInputs(wl, n_steps=n_steps, eos_min_block=2, arrive_hi=1 if batch_sync else 24)
+    run = sweep.SweepRunner(inp, window_in_pages=window_in_pages, batch_sync=batch_sync)
     stc = inp.stc
     b = wl.block_len
-    ocfg = H.oracle_cfg(stc)
+    ocfg = H.oracle_cfg(stc, batch_sync=int(batch_sync))
     ost = H.oracle_state(stc, inp.tokens0())
     n_rows = wl.max_slots * b
     commits = spawns = edits = 0
@@ -101,6 +102,12 @@ def test_serving_sweep_states_match_oracle_every_step(window_in_pages):
         spawns += int(spawned.sum())
         edits += int((action == O.ACT_T2T).sum())
     assert (ost.active != 0).all(), "every request has arrived"
-    assert commits >= 2 * wl.n_requests and spawns >= commits
     assert edits > 0, "the re-drawn winners never produced a T2T edit"
-    assert (ost.active == 2).any(), "no request reached a committed EOS"
+    if batch_sync:
+        # the shared window: every sequence still decoding sits at the same [L, R)
+        live = ost.active == 1
+        assert len(set(ost.L[live])) <= 1 and len(set(ost.R[live])) <= 1
+        assert commits >= wl.n_requests
+    else:
+        assert commits >= 2 * wl.n_requests and spawns >= commits
+        assert (ost.active == 2).any(), "no request reached a committed EOS"

@@ -109,6 +109,10 @@ def test_committed_eos_leaves_the_batch_and_the_cascade_goes_on():
     st = state(cfg, L=[1, 0], R=[2, 2])
     (_, _), (s1, (n1, _, c1)) = both(cfg, st, {(0, 0): FIN, (1, 0): FIN, (1, 1): FIN})
     assert list(n1) == [1, 2] and list(s1.active) == [2, 2] and c1[O.CT_LOCKSTEP_COMMIT] == 2
+    # handed in with L == n already: done at once under either policy, and no obstacle
+    st = state(cfg, L=[2, 0], R=[2, 2])
+    (s0, (n0, _, _)), (s1, (n1, _, c1)) = both(cfg, st, {(1, 0): FIN, (1, 1): HALF})
+    assert list(n0) == list(n1) == [0, 1] and list(s0.active) == list(s1.active) == [2, 1]
 
 
 def run(cfg, st, logits_for, steps):
