@@ -435,9 +435,19 @@ def run_sweep(args):
     wl = synth.WORKLOADS[args.workload]
     if args.requests:
         wl = dataclasses.replace(wl, n_requests=args.requests)
+    over = {}
+    if args.wmax:
+        over["wmax"] = args.wmax
+    if args.theta is not None:
+        over["theta_spawn"] = args.theta
+    if args.block_len:
+        over["block_len"] = args.block_len
+        over["max_blocks"] = max(2, wl.max_blocks * wl.block_len // args.block_len)
+    wl = dataclasses.replace(wl, **over)
     n_steps = args.steps if args.steps != 20 else 48
-    inp = sweep.SweepInputs(wl, n_steps=n_steps)
-    run = sweep.SweepRunner(inp, dev, window_in_pages=args.window_in_pages)
+    rise = tuple(float(x) for x in args.rise_range.split(",")) if args.rise_range else None
+    inp = sweep.SweepInputs(wl, n_steps=n_steps, arrive_hi=1 if args.static_batch else 24, rise_range=rise)
+    run = sweep.SweepRunner(inp, dev, window_in_pages=args.window_in_pages, batch_sync=args.batch_sync)
 
     def one_pass(timed):
         seg, flops, live, committed = [], [], [], 0
@@ -481,14 +491,19 @@ def run_sweep(args):
         "n_gpus": 1, "steps": n_steps, "warmup": n_steps, "ms_per_step": round(total_ms / n_steps, 4),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": wl.name + (" (sweep, window in pages)" if args.window_in_pages else " (sweep)"), "requests": wl.n_requests, "block_len": wl.block_len,
-                   "wmax": wl.wmax, "slots": wl.max_slots, "live_slots": float(live.mean()),
+                   "wmax": wl.wmax, "theta_spawn": wl.theta_spawn,
+                   "policy": "batch-synchronous wavefront" if args.batch_sync else "per-sequence wavefronts",
+                   "arrivals": "all at step 0" if args.static_batch else "uniform over the first 24 steps",
+                   "confidence_rise_per_step": list(rise) if rise else 0.05,
+                   "slots": wl.max_slots, "live_slots": float(live.mean()),
                    "q_heads": wl.n_q_heads, "kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim,
                    "vocab": wl.vocab, "prefix_range": [wl.prefix_lo, wl.prefix_hi],
                    "logits": "noise bank, one winner per live row patched per step", "parallelism": "replicas x1",
                    "l2": "inputs larger than L2 (logits + KV pools >> 126 MB); no flush"},
         "sweep": {"steps_per_s": round(n_steps / total_ms * 1e3, 1),
                   "committed_tokens_per_s": round(committed / total_ms * 1e3, 1),
-                  "committed_tokens": committed, "live_slots_first_last": [int(live[0]), int(live[-1])],
+                  "committed_tokens": committed, "committed_tokens_per_step": round(committed / n_steps, 2),
+                  "live_slots_first_last": [int(live[0]), int(live[-1])],
                   "device_ms_total": round(total_ms, 3)},
         "clocks": clocks,
         "e2e": {"value": None, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
@@ -604,6 +619,14 @@ def main():
     ap.add_argument("--window-in-pages", action="store_true",
                     help="with --sweep: scatter the window K/V into the pages every step (Eq. 6), attention "
                          "over the pages, retirement as a pointer bump")
+    ap.add_argument("--batch-sync", action="store_true",
+                    help="with --sweep: the batch-synchronous wavefront of the packing ablation (fb_config.batch_sync)")
+    ap.add_argument("--static-batch", action="store_true", help="with --sweep: every request arrives at step 0")
+    ap.add_argument("--rise-range", default="",
+                    help="with --sweep: lo,hi of the per-request confidence rise per step (default 0.05 for all)")
+    ap.add_argument("--wmax", type=int, default=0, help="with --sweep: window bound W")
+    ap.add_argument("--theta", type=float, default=None, help="with --sweep: admission gate theta_spawn")
+    ap.add_argument("--block-len", type=int, default=0, help="with --sweep: block length bl")
     ap.add_argument("--sweep", action="store_true",
                     help="run the serving workload as a 48-step sequence with arrivals (use with --workload 4)")
     args = ap.parse_args()

@@ -7,8 +7,8 @@ Two parts, neither of which holds any of the decode method's logic:
 * :class:`SweepInputs` -- seeded inputs.  A fixed bank of N(0,1) bf16 logits,
   one row per slot-order row; every step one element per live row (the
   position's "winner" token) is overwritten so that the row's softmax
-  confidence is the position's target ``c = clip(c0 + 0.05 (step - spawn
-  step), 0.02, 0.995)``, nudged until, after bf16 rounding, it is at least
+  confidence is the position's target ``c = clip(c0 + rise (step - spawn
+  step), 0.02, 0.995)`` (rise = 0.05, or drawn per request), nudged until, after bf16 rounding, it is at least
   2e-3 away from both thresholds.  The confidence the patched row then has is
   returned with the patch (it follows from the bank row's sum of exponentials,
   taken once in fp64).
@@ -54,10 +54,16 @@ def sweep_structure(wl: synth.Workload, seed: int) -> synth.Structure:
 class SweepInputs:
     def __init__(self, wl: synth.Workload, n_steps: int = 48, seed: int | None = None,
                  arrive_hi: int = 24, c_rise: float = 0.05, redraw: float = 0.1,
-                 eos_frac: float = 0.25, eos_min_block: int = 8):
+                 eos_frac: float = 0.25, eos_min_block: int = 8, rise_range=None):
+        """``rise_range = (lo, hi)``: the per-step confidence rise is drawn per
+        request from U[lo, hi] instead of being ``c_rise`` for all (easy and
+        hard requests: the stragglers of a static batch)."""
         self.wl, self.n_steps = wl, n_steps
         self.seed = synth.BASE_SEED + wl.index if seed is None else seed
         self.c_rise, self.redraw = c_rise, redraw
+        self.rise = np.full(wl.n_requests, c_rise)
+        if rise_range is not None:
+            self.rise = synth._rng(self.seed, 12).uniform(rise_range[0], rise_range[1], size=wl.n_requests)
         self.stc = sweep_structure(wl, self.seed)
         Rn, b, n, V = wl.n_requests, wl.block_len, wl.max_blocks, wl.vocab
         rg = synth._rng(self.seed, 11)
@@ -123,7 +129,7 @@ class SweepInputs:
         req, col = np.concatenate(req), np.concatenate(col)
         rows = np.arange(len(req))
         w = self.winner[req, col]
-        c = np.clip(self.c0[req, col] + self.c_rise * (step - self.spawn_step[req, col // b]), 0.02, 0.995)
+        c = np.clip(self.c0[req, col] + self.rise[req] * (step - self.spawn_step[req, col // b]), 0.02, 0.995)
         noise_w = self.bank[torch.from_numpy(rows), torch.from_numpy(w)].to(torch.float64).numpy()
         others = self.sum_exp[rows] - np.exp(noise_w)
         # the largest other element: the row maximum unless the winner's own noise was it
