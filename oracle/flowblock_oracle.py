@@ -23,7 +23,11 @@ Pins (tests/test_oracle_*.py, all CPU):
                          query -> mean of visible V rows; constant V; one
                          dominant key); isolation; block causality
   t2t_rows               closed form e^a / (e^a + V - 1); ties -> lowest index
-  t2t_update             hand-worked Eq. 1 / Eq. 2 case
+  t2t_update             hand-worked Eq. 1 / Eq. 2 case; literal Delta: hand-worked
+                         rows, and no effect when tau_edit >= tau_mask; forced
+                         progress: hand-worked block, no effect where Eq. 1
+                         reveals something, termination within bl + S_pe + 1
+                         steps per block on logits that never clear a threshold
   gate_commit            hand-worked Alg. 1 cases; window of one block equals
                          an independently written serial block-wise decoder;
                          packed run equals per-request runs
@@ -57,6 +61,7 @@ FLAG_FRONTIER = 2   # slot is block R-1 of its request (readiness is read here)
 ACT_NONE = 0
 ACT_M2T = 1         # masked position revealed (set Gamma of Eq. 1)
 ACT_T2T = 2         # revealed position overwritten (set Delta of Eq. 1)
+ACT_FORCED = 3      # masked position revealed by the forced-progress rule
 
 # slot_stats columns
 ST_M0, ST_RDY, ST_M2T, ST_T2T, ST_M1, ST_EOS = range(6)
@@ -87,6 +92,8 @@ class Config:
     theta_spawn: float = 0.5
     sm_scale: float = 0.0     # 0 -> 1/sqrt(head_dim); READING: paper silent
     batch_sync: int = 0       # 1: the batch-synchronous wavefront of Sec. 3.2 / 4.5
+    delta_literal: int = 0    # 1: Delta of Eq. 1 as printed (masked positions too)
+    force_progress: int = 0   # 1: the oldest block reveals at least one mask per step
 
     @property
     def max_slots(self) -> int:
@@ -383,6 +390,21 @@ def t2t_update(cfg: Config, pk: Pack, st: State, xhat, conf):
     whenever tau_edit >= tau_mask.  Live blocks hold no prompt positions.
     Thresholds are binary32 values compared against the fp64 confidence.
 
+    ``delta_literal = 1``: Delta exactly as Eq. 1 prints it, without the
+    restriction to revealed positions: a masked position whose prediction is
+    not [M] itself is updated as soon as p > tau_edit, whatever tau_mask says
+    (it only matters when tau_edit < tau_mask).  Revealing a mask is M2T in
+    the paper's terms whichever set it came through.
+
+    ``force_progress = 1`` (READING; Eq. 1 is threshold-only and the paper
+    names no fallback): if the oldest live block of a request went into the
+    forward with masks and Eq. 1 revealed none of them, its masked position
+    with the highest confidence (lowest position on ties; confidences compared
+    in binary32, the precision the kernel holds them in) is revealed
+    (ACT_FORCED, counted as M2T).  Younger blocks are left to the thresholds:
+    their context is still immature (Sec. 2.2).  The oldest block then loses a
+    mask every step, so a request terminates whatever the logits do.
+
     Per slot: m0 = masks before the update, rdy = |{i in M_B: p_i >= tau_mask}|
     (numerator of Eq. 2; READING: M_B is the mask set that went into this
     forward), n_m2t, n_t2t, m1 = masks after, has_eos.
@@ -395,16 +417,20 @@ def t2t_update(cfg: Config, pk: Pack, st: State, xhat, conf):
     for slot in range(pk.n_live):
         r, s = int(pk.slot_req[slot]), int(pk.slot_s[slot])
         g = int(st.L[r]) + s
+        masked_before = []
         for t in range(b):
             i = slot * b + t
             col = g * b + t
             x = int(st.tokens[r, col])
             p = float(conf[i])
             if x == cfg.mask_id:
+                masked_before.append(t)
                 stats[slot, ST_M0] += 1
                 if p >= tm:
                     stats[slot, ST_RDY] += 1
-                if p > tm:
+                in_gamma = p > tm
+                in_delta = bool(cfg.delta_literal) and x != int(xhat[i]) and p > te
+                if in_gamma or in_delta:
                     st.tokens[r, col] = xhat[i]
                     action[i] = ACT_M2T
                     stats[slot, ST_M2T] += 1
@@ -412,7 +438,17 @@ def t2t_update(cfg: Config, pk: Pack, st: State, xhat, conf):
                 st.tokens[r, col] = xhat[i]
                 action[i] = ACT_T2T
                 stats[slot, ST_T2T] += 1
-            y = int(st.tokens[r, col])
+        if (cfg.force_progress and s == 0 and masked_before
+                and stats[slot, ST_M2T] == 0):
+            best = masked_before[0]
+            for t in masked_before[1:]:
+                if np.float32(conf[slot * b + t]) > np.float32(conf[slot * b + best]):
+                    best = t
+            st.tokens[r, g * b + best] = xhat[slot * b + best]
+            action[slot * b + best] = ACT_FORCED
+            stats[slot, ST_M2T] += 1
+        for t in range(b):
+            y = int(st.tokens[r, g * b + t])
             if y == cfg.mask_id:
                 stats[slot, ST_M1] += 1
             if y == cfg.eos_id:
