@@ -59,7 +59,8 @@ typedef enum {
 } fb_status;
 
 enum { FB_FLAG_OLDEST = 1, FB_FLAG_FRONTIER = 2 };          /* slot_flags  */
-enum { FB_ACT_NONE = 0, FB_ACT_M2T = 1, FB_ACT_T2T = 2 };   /* action code */
+enum { FB_ACT_NONE = 0, FB_ACT_M2T = 1, FB_ACT_T2T = 2,
+       FB_ACT_FORCED = 3 /* force_progress reveal */ };     /* action code */
 /* slot_stats columns */
 enum { FB_STAT_M0 = 0, FB_STAT_RDY, FB_STAT_M2T, FB_STAT_T2T, FB_STAT_M1, FB_STAT_EOS,
        FB_SLOT_STATS = 6 };
@@ -91,7 +92,7 @@ typedef struct {
   int32_t max_blocks;        /* n, generation blocks per request            */
   int32_t s_pe;              /* S_pe, post-edit forwards, 0..255            */
   float tau_mask;
-  float tau_edit;            /* must be >= tau_mask                         */
+  float tau_edit;            /* >= tau_mask unless delta_literal = 1        */
   float theta_spawn;
   float sm_scale;            /* 0 -> 1/sqrt(head_dim)                       */
   int32_t window_in_pages;   /* 0: this step's window K/V are passed to the
@@ -108,6 +109,19 @@ typedef struct {
                                 sequence is admitted only when every sequence
                                 clears the gate (min over the batch of rho)
                                 and has room                                 */
+  int32_t delta_literal;     /* 0: Delta of Eq. 1 on revealed positions only
+                                (the prose's reading; needs tau_edit >=
+                                tau_mask).  1: Delta as printed: a masked
+                                position whose prediction is not [M] is also
+                                updated once p > tau_edit; tau_edit may then
+                                be below tau_mask                            */
+  int32_t force_progress;    /* 1: when the oldest live block of a request
+                                went into the forward with masks and Eq. 1
+                                revealed none, its most confident masked
+                                position (lowest position on ties, binary32
+                                compare) is revealed (action FB_ACT_FORCED,
+                                counted as M2T).  Not in the paper: Eq. 1 is
+                                threshold-only; off by default               */
 } fb_config;
 
 /* Per-request wavefront state (Sec. 3.2: (L_b, R_b), in-order commit
@@ -141,7 +155,7 @@ typedef struct {
 
 /* Validates the configuration and creates a context (host memory only; no
  * CUDA call is made).  FB_ERR_UNSUPPORTED for shapes the kernels do not
- * implement, including tau_edit < tau_mask. */
+ * implement, including tau_edit < tau_mask without delta_literal. */
 int fb_create(const fb_config* cfg, fb_ctx** out);
 int fb_destroy(fb_ctx* ctx);
 const char* fb_last_error(const fb_ctx* ctx); /* ctx may be NULL */

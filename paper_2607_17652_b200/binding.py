@@ -22,6 +22,7 @@ FB_ERR_INVALID_ARG, FB_ERR_SHAPE, FB_ERR_ALIGNMENT = -1, -2, -3
 FB_ERR_UNSUPPORTED, FB_ERR_WORKSPACE, FB_ERR_CUDA = -4, -5, -6
 FB_ST_BAD_PAGE, FB_ST_BAD_TOKEN, FB_ST_BAD_STATE = 1, 2, 4
 FB_ST_NAN_LOGIT, FB_ST_DEV_TIMEOUT = 8, 16
+FB_ACT_NONE, FB_ACT_M2T, FB_ACT_T2T, FB_ACT_FORCED = 0, 1, 2, 3
 FB_SLOT_STATS, FB_STEP_COUNTERS = 6, 10
 
 EXPORTS = ["fb_create", "fb_destroy", "fb_last_error", "fb_workspace_bytes",
@@ -38,7 +39,8 @@ class fb_config(C.Structure):
         "mask_id", "eos_id", "max_blocks", "s_pe")] + \
         [(n, C.c_float) for n in ("tau_mask", "tau_edit", "theta_spawn",
                                   "sm_scale")] + \
-        [("window_in_pages", C.c_int32), ("batch_sync", C.c_int32)]
+        [("window_in_pages", C.c_int32), ("batch_sync", C.c_int32),
+         ("delta_literal", C.c_int32), ("force_progress", C.c_int32)]
 
 
 class fb_state(C.Structure):

@@ -88,8 +88,11 @@ int fb_create(const fb_config* cfg, fb_ctx** out) {
   if (c.wmax > 8) return fail(nullptr, FB_ERR_UNSUPPORTED, "wmax must be at most 8");
   if (c.vocab % 8 != 0) return fail(nullptr, FB_ERR_UNSUPPORTED, "vocab must be a multiple of 8");
   if (c.s_pe > 255) return fail(nullptr, FB_ERR_UNSUPPORTED, "s_pe must be at most 255");
-  if (c.tau_edit < c.tau_mask)
-    return fail(nullptr, FB_ERR_UNSUPPORTED, "tau_edit < tau_mask is not supported");
+  if ((c.delta_literal != 0 && c.delta_literal != 1) || (c.force_progress != 0 && c.force_progress != 1))
+    return fail(nullptr, FB_ERR_INVALID_ARG, "delta_literal and force_progress must be 0 or 1");
+  if (c.tau_edit < c.tau_mask && !c.delta_literal)
+    return fail(nullptr, FB_ERR_UNSUPPORTED,
+                "tau_edit < tau_mask needs delta_literal = 1 (with Delta on revealed positions only the order is fixed)");
   if (c.window_in_pages != 0 && c.window_in_pages != 1)
     return fail(nullptr, FB_ERR_INVALID_ARG, "window_in_pages must be 0 or 1");
   if (c.batch_sync != 0 && c.batch_sync != 1)

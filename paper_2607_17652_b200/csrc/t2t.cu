@@ -169,6 +169,7 @@ struct UpdParams {
   int32_t* slot_stats;
   int32_t max_slots, bl, max_blocks, mask_id, eos_id;
   float tau_mask, tau_edit;
+  int32_t delta_literal, force_progress;
 };
 
 __global__ void __launch_bounds__(128) t2t_update_kernel(const UpdParams p) {
@@ -185,6 +186,8 @@ __global__ void __launch_bounds__(128) t2t_update_kernel(const UpdParams p) {
   const int g = p.L[r] + p.slot_s[slot];
   int32_t* tok = p.tokens + (size_t)r * p.max_blocks * p.bl + (size_t)g * p.bl;
   int m0 = 0, rdy = 0, m2t = 0, t2t = 0, m1 = 0, eos = 0;
+  float bestp = -1.f;                               // most confident mask this lane left in place
+  int bestt = 0x7fffffff;
   for (int t = lane; t < p.bl; t += 32) {
     const int i = slot * p.bl + t;
     int x = tok[t];
@@ -194,7 +197,10 @@ __global__ void __launch_bounds__(128) t2t_update_kernel(const UpdParams p) {
     if (x == p.mask_id) {                         // Gamma of Eq. 1: strict >
       m0++;
       rdy += pr >= p.tau_mask;                    // Eq. 2 numerator: >=
-      if (pr > p.tau_mask) { x = xh; act = FB_ACT_M2T; m2t++; }
+      // Delta as printed has no "revealed" condition: with delta_literal a mask whose
+      // prediction is not [M] itself is updated once p > tau_edit as well
+      if (pr > p.tau_mask || (p.delta_literal && x != xh && pr > p.tau_edit)) { x = xh; act = FB_ACT_M2T; m2t++; }
+      else if (pr > bestp) { bestp = pr; bestt = t; }
     } else if (x != xh && pr > p.tau_edit) {      // Delta of Eq. 1, revealed only
       x = xh; act = FB_ACT_T2T; t2t++;
     }
@@ -211,6 +217,19 @@ __global__ void __launch_bounds__(128) t2t_update_kernel(const UpdParams p) {
     t2t += __shfl_xor_sync(0xffffffffu, t2t, o);
     m1 += __shfl_xor_sync(0xffffffffu, m1, o);
     eos |= __shfl_xor_sync(0xffffffffu, eos, o);
+  }
+  // forced progress: the oldest block went in with masks and Eq. 1 revealed none -> its most
+  // confident masked position (lowest position on ties) is revealed
+  if (p.force_progress && p.slot_s[slot] == 0 && m0 > 0 && m2t == 0) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float op = __shfl_xor_sync(0xffffffffu, bestp, o);
+      const int ot = __shfl_xor_sync(0xffffffffu, bestt, o);
+      if (op > bestp || (op == bestp && ot < bestt)) { bestp = op; bestt = ot; }
+    }
+    const int xh = p.argmax[slot * p.bl + bestt];
+    if (lane == 0) { tok[bestt] = xh; p.action[slot * p.bl + bestt] = FB_ACT_FORCED; }
+    m2t = 1; m1 -= xh != p.mask_id; eos |= xh == p.eos_id;
   }
   if (lane == 0) {
     int32_t* s = p.slot_stats + slot * FB_SLOT_STATS;
@@ -245,6 +264,7 @@ int launch_t2t_update(fb_ctx* ctx, const fb_pack* pk, const fb_state* st, const 
   u.argmax = argmax; u.conf = conf; u.action = action; u.slot_stats = slot_stats;
   u.max_slots = max_slots; u.bl = c.block_len; u.max_blocks = c.max_blocks; u.mask_id = c.mask_id;
   u.eos_id = c.eos_id; u.tau_mask = c.tau_mask; u.tau_edit = c.tau_edit;
+  u.delta_literal = c.delta_literal; u.force_progress = c.force_progress;
   return cuda_err(ctx, launch_pdl(t2t_update_kernel, (max_slots + 3) / 4, 128, 0, stream, u), "t2t_update_kernel launch");
 }
 

@@ -51,10 +51,13 @@ def test_create_validates_configuration():
     bad = [dict(head_dim=96), dict(page_size=32), dict(block_len=24),
            dict(n_kv_heads=3), dict(wmax=0), dict(vocab=1001), dict(wmax=9),
            dict(tau_edit=0.5), dict(s_pe=300), dict(max_requests=-1),
-           dict(tau_mask=float("nan")), dict(window_in_pages=2), dict(batch_sync=2)]
+           dict(tau_mask=float("nan")), dict(window_in_pages=2), dict(batch_sync=2),
+           dict(delta_literal=2), dict(force_progress=-1)]
     for delta in bad:
         with pytest.raises(B.FlowBlockError):
             B.Context(**dict(GOOD, **delta))
+    # thresholds the other way round are accepted only with Delta taken literally
+    B.Context(**dict(GOOD, tau_edit=0.5, delta_literal=1))
     assert B.lib().fb_create(None, None) == B.FB_ERR_INVALID_ARG
     assert b"null" in B.lib().fb_last_error(None)
 

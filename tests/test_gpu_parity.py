@@ -159,7 +159,9 @@ def run_t2t_and_gate(case, **over):
     for thr in (np.float32(ocfg.tau_mask), np.float32(ocfg.tau_edit)):
         assert np.abs(conf[:live] - float(thr)).min() >= MARGIN, \
             "generator left a confidence inside the decision margin"
+    tokens_before = ost.tokens.copy()
     action, stats = O.t2t_update(ocfg, opk, ost, xhat, conf)
+    forced_margin = forced_reveal_margin(ocfg, opk, ost, tokens_before, action, conf)
     np.testing.assert_array_equal(sb.argmax.cpu().numpy(), xhat)
     np.testing.assert_allclose(sb.conf.cpu().numpy(), conf, rtol=0, atol=CONF_TOL)
     np.testing.assert_array_equal(sb.action.cpu().numpy(), action)
@@ -183,7 +185,23 @@ def run_t2t_and_gate(case, **over):
         np.testing.assert_array_equal(H.f64(kp.cpu()), okp)
         np.testing.assert_array_equal(H.f64(vp.cpu()), ovp)
     assert int(sb.status.item()) == 0
-    return dict(action=action, stats=stats, ncom=ncom, spawned=spawned, ctr=ctr)
+    return dict(action=action, stats=stats, ncom=ncom, spawned=spawned, ctr=ctr, forced_margin=forced_margin)
+
+
+def forced_reveal_margin(ocfg, opk, ost, tokens_before, action, conf):
+    """Smallest gap between the confidence of a force-revealed position and the
+    best other masked position of its block (inf if nothing was forced)."""
+    b = ocfg.block_len
+    gap = np.inf
+    for i in np.flatnonzero(action == O.ACT_FORCED):
+        slot, r = i // b, int(opk.slot_req[i // b])
+        L_before = int(ost.L[r])          # t2t_update does not move L
+        g = L_before + int(opk.slot_s[slot])
+        masked = tokens_before[r, g * b:(g + 1) * b] == ocfg.mask_id
+        others = [conf[slot * b + t] for t in range(b) if masked[t] and slot * b + t != i]
+        if others:
+            gap = min(gap, float(conf[i] - max(others)))
+    return gap
 
 
 @pytest.mark.parametrize("name,kind,shift,s_pe", [
@@ -264,6 +282,45 @@ def test_gate_commit_on_drawn_block_counts(seed, batch_sync):
     np.testing.assert_array_equal(H.f64(kp.cpu()), okp)
     np.testing.assert_array_equal(H.f64(vp.cpu()), ovp)
     assert int(sb.status.item()) == 0
+
+
+@pytest.mark.parametrize("name,shift,thr,over", [
+    ("tiny", 0.0, (0.9, 0.6), dict(delta_literal=1)),
+    ("tiny_wide", 0.2, (0.95, 0.9), dict(delta_literal=1)),
+    ("tiny", 0.3, (0.9, 0.95), dict(delta_literal=1)),                       # usual order: no effect
+    ("tiny", -0.4, (0.9, 0.95), dict(force_progress=1)),
+    ("tiny_wide", -0.3, (0.9, 0.95), dict(force_progress=1, s_pe=0)),
+    ("tiny_d128_b64", -0.5, (0.9, 0.85), dict(force_progress=1, delta_literal=1)),
+    ("tiny_wide", -0.3, (0.9, 0.95), dict(force_progress=1, batch_sync=1))])
+def test_update_modes_bit_exact(name, shift, thr, over):
+    """Eq. 1 with Delta taken literally and / or the forced-progress rule on the
+    oldest block, whole T2T + gate step against the oracle.  The thresholds go
+    into the workload so that the generator keeps its margin around them."""
+    wl = dataclasses.replace(WORKLOADS[name], tau_mask=thr[0], tau_edit=thr[1])
+    for seed in range(20):
+        case = make_case(wl, seed=synth.BASE_SEED + 700 + seed, logits_kind="calibrated", conf_shift=shift)
+        if not over.get("force_progress"):
+            break
+        # a forced reveal compares confidences with each other: take a draw (judged by the
+        # oracle alone) in which no such comparison is closer than the decision margin
+        stc = case["stc"]
+        ocfg = H.oracle_cfg(stc, **over)
+        ost = H.oracle_state(stc, case["tokens"])
+        opk = O.pack_wavefronts(ocfg, ost)
+        xhat, conf = O.t2t_rows(ocfg, opk, H.f64(case["logits"]))
+        before = ost.tokens.copy()
+        action, _ = O.t2t_update(ocfg, opk, ost, xhat, conf)
+        if (action == O.ACT_FORCED).any() and forced_reveal_margin(ocfg, opk, ost, before, action, conf) >= MARGIN:
+            break
+    else:
+        pytest.fail("no draw with a forced reveal outside the decision margin")
+    res = run_t2t_and_gate(case, **over)
+    if over.get("force_progress"):
+        assert (res["action"] == B.FB_ACT_FORCED).any(), "no block needed the forced reveal in this draw"
+        # the reveal is decided by comparing confidences: the draw must not hinge on the last bits
+        assert res["forced_margin"] >= MARGIN
+    if thr[1] < thr[0] and shift >= 0:
+        assert (res["action"] == O.ACT_M2T).any()
 
 
 def test_t2t_full_vocab_rows():
