@@ -354,6 +354,66 @@ def test_t2t_hand_worked_rows():
     assert res["spawned"][0] == 1 and res["ncom"][0] == 0
 
 
+def test_step_replayed_from_a_cuda_graph_matches_direct_launches():
+    """The step is shape-stable (grids depend on the slot capacity, the live
+    count is read on the device), so one captured step can be replayed while
+    the state moves under it: four replays against four directly launched
+    steps, everything bit for bit (attention output included: the dynamic
+    hand-out of work items does not change any item's arithmetic)."""
+    wl = synth.tiny_workload(n_requests=5, wmax=3, w_lo=1, w_hi=2, max_blocks=12, prefix_lo=40, prefix_hi=700)
+    case = make_case(wl, with_logits=False)
+    # every row peaked (p ~ 0.9996): blocks reveal, get edited, retire and spawn at every step
+    rows = wl.max_slots * wl.block_len
+    zc = torch.zeros(rows, wl.vocab)
+    win = torch.from_numpy(np.random.default_rng(3).integers(0, wl.vocab - 2, size=rows))
+    zc[torch.arange(rows), win] = 14.0
+    z = zc.to(torch.bfloat16).to(DEV)
+    outs = []
+    for use_graph in (False, True):
+        ctx, st, pk, sb = gpu_objects(case, s_pe=0)
+        q, kw, vw, kp, vp = (t.to(DEV) for t in case["attn"])
+
+        def step():
+            B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+            B.fb_wavefront_attn(ctx, pk, q, kw, vw, kp, vp, st.page_table, sb.out, sb.ws, sb.status)
+            B.fb_t2t_step(ctx, pk, z, st, sb.argmax, sb.conf, sb.action, sb.slot_stats, sb.status)
+            B.fb_gate_commit(ctx, pk, sb.slot_stats, st, kw, vw, kp, vp, sb.n_committed, sb.spawned,
+                             sb.step_counters, sb.status)
+        trace = []
+        if use_graph:
+            g = torch.cuda.CUDAGraph()
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                snap = {k: getattr(st, k).clone() for k in ("active", "prefix_len", "L", "R", "tokens", "pe_done")}
+                pools = (kp.clone(), vp.clone())
+                step()                                  # first call: device set-up happens outside the capture
+                side.synchronize()
+                for k, v in snap.items():
+                    getattr(st, k).copy_(v)
+                kp.copy_(pools[0]); vp.copy_(pools[1])
+                side.synchronize()
+                with torch.cuda.graph(g, stream=side):
+                    step()
+            torch.cuda.current_stream().wait_stream(side)
+        for _ in range(4):
+            g.replay() if use_graph else step()
+            torch.cuda.synchronize()
+            trace.append((sb.out.clone(), sb.action.clone(), sb.n_committed.clone(), sb.spawned.clone(),
+                          sb.step_counters.clone(), st.tokens.clone(), st.L.clone(), st.R.clone(),
+                          pk.n_live.clone()))
+        assert int(sb.status.item()) == 0
+        outs.append((trace, kp.clone(), vp.clone()))
+    (ta, kpa, vpa), (tb, kpb, vpb) = outs
+    for a, b in zip(ta, tb):
+        live = int(a[8].item()) * wl.block_len
+        assert torch.equal(a[0][:live], b[0][:live])
+        for x, y in zip(a[1:], b[1:]):
+            assert torch.equal(x, y)
+    assert torch.equal(kpa, kpb) and torch.equal(vpa, vpb)
+    assert sum(int(t[2].sum()) for t in ta) > 0, "nothing retired in four steps"
+
+
 # -------------------------------------------------------------- attention
 def run_attention(case, fill_pad=False):
     stc = case["stc"]
