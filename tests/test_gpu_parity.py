@@ -77,6 +77,8 @@ WORKLOADS = {
                                             max_blocks=16),
     "tiny_g8": synth.tiny_workload(n_q_heads=16, n_kv_heads=2, head_dim=128,
                                    prefix_lo=60, prefix_hi=420, n_requests=4),
+    # a vocabulary whose 16-byte pieces (125) do not divide among the two CTAs of a row
+    "tiny_v1000": synth.tiny_workload(vocab=1000),
     "cfg0": synth.WORKLOADS[0],
     "cfg1": synth.WORKLOADS[1],
 }
@@ -207,7 +209,7 @@ def forced_reveal_margin(ocfg, opk, ost, tokens_before, action, conf):
 @pytest.mark.parametrize("name,kind,shift,s_pe", [
     ("tiny", "calibrated", 0.0, 1), ("tiny", "calibrated", 0.3, 0),
     ("tiny_wide", "calibrated", 0.2, 1), ("tiny_d128_b64", "calibrated", 0.1, 3),
-    ("tiny", "literal", 0.0, 1), ("cfg0", "normal2", 0.0, 1)])
+    ("tiny", "literal", 0.0, 1), ("cfg0", "normal2", 0.0, 1), ("tiny_v1000", "calibrated", 0.1, 1)])
 def test_t2t_and_gate_commit_bit_exact(name, kind, shift, s_pe):
     case = make_case(WORKLOADS[name], logits_kind=kind, conf_shift=shift)
     res = run_t2t_and_gate(case, s_pe=s_pe)
