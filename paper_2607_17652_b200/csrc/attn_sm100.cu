@@ -593,15 +593,18 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           tmem_ld_wait();
           tmem_ld32(tS + 64, sb); tmem_ld32(tS + 96, sb + 32);     // in flight during the first half
 #pragma unroll
-          for (int i = 0; i < 64; i += 8)
-#pragma unroll
-            for (int t = 0; t < 8; ++t) m8[t] = fmaxf(m8[t], i + t < limit ? __uint_as_float(sa[i + t]) : -INFINITY);
-          tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 64; i += 8)
+          for (int i = 0; i < 64; i += 16)
 #pragma unroll
             for (int t = 0; t < 8; ++t)
-              m8[t] = fmaxf(m8[t], 64 + i + t < limit ? __uint_as_float(sb[i + t]) : -INFINITY);
+              m8[t] = max3(m8[t], i + t < limit ? __uint_as_float(sa[i + t]) : -INFINITY,
+                           i + 8 + t < limit ? __uint_as_float(sa[i + 8 + t]) : -INFINITY);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 64; i += 16)
+#pragma unroll
+            for (int t = 0; t < 8; ++t)
+              m8[t] = max3(m8[t], 64 + i + t < limit ? __uint_as_float(sb[i + t]) : -INFINITY,
+                           64 + i + 8 + t < limit ? __uint_as_float(sb[i + 8 + t]) : -INFINITY);
           m_ref = fmaxf(fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3])), fmaxf(fmaxf(m8[4], m8[5]), fmaxf(m8[6], m8[7])));
         }
         FB_TR(2 + X, 42);
@@ -624,7 +627,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
 #pragma unroll
               for (int i = 0; i < 32; i += 2) {
                 const float2 x = __ffma2_rn(make_float2(__uint_as_float(sr[i]), __uint_as_float(sr[i + 1])), sl2v, nmb);
-                xm4[(i >> 1) & 3] = fmaxf(fmaxf(xm4[(i >> 1) & 3], x.x), x.y);
+                xm4[(i >> 1) & 3] = max3(xm4[(i >> 1) & 3], x.x, x.y);
                 float2 pv;
                 if (((i >> 1) & 3) < FB_POLY_OF4) pv = exp2_poly2(x);
                 else pv = make_float2(ex2_approx(x.x), ex2_approx(x.y));
