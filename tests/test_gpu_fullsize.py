@@ -178,6 +178,54 @@ def test_long_context_attention_sampled_requests():
     assert bool((sb.out[live:].float() == 7.0).all())
 
 
+@pytest.mark.parametrize("window_in_pages", [0, 1])
+def test_serving_structure_attention_sampled_requests(window_in_pages):
+    """The serving workload's structure at full size (128 requests, 512 slots of
+    capacity, prefixes of 512-4096 tokens, one to four live blocks each): the
+    packing of all requests bit for bit, the attention of four sampled requests
+    (first, last, and the ones with the shortest and the longest prefix)
+    against the oracle; also with the window resident in the pages (Eq. 6
+    scatter first, every key read through the page table)."""
+    wl = synth.WORKLOADS[4]
+    stc = synth.make_structure(wl)
+    tokens = synth.make_tokens(stc)
+    attn = synth.make_attn_inputs(stc)
+    ctx = B.Context(**synth.config_dict(stc, window_in_pages=window_in_pages))
+    st = B.DeviceState.from_numpy(DEV, stc.active, stc.prefix_len, stc.L, stc.R, tokens,
+                                  np.zeros((wl.n_requests, wl.wmax), np.uint8), stc.page_table)
+    pk = B.PackBuffers.alloc(ctx, DEV)
+    sb = B.StepBuffers(ctx, DEV)
+    q, kw, vw, kp, vp = (t.to(DEV) for t in attn)
+    sb.out.fill_(7.0)
+    B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+    if window_in_pages:
+        B.fb_scatter_window_kv(ctx, pk, st.page_table, kw, vw, kp, vp, sb.status)
+        B.fb_wavefront_attn(ctx, pk, q, None, None, kp, vp, st.page_table, sb.out, sb.ws, sb.status)
+    else:
+        B.fb_wavefront_attn(ctx, pk, q, kw, vw, kp, vp, st.page_table, sb.out, sb.ws, sb.status)
+    torch.cuda.synchronize()
+    assert int(sb.status.item()) == 0
+    ocfg = O.Config(**synth.config_dict(stc))
+    opk_all = O.pack_wavefronts(ocfg, H.oracle_state(stc, tokens))
+    g = pk.to_numpy()
+    assert int(g["n_live"][0]) == opk_all.n_live
+    for name in ("slot_req", "slot_s", "slot_pos0", "slot_kv_len", "slot_flags", "req_slot_begin", "qtok", "pos"):
+        np.testing.assert_array_equal(g[name], getattr(opk_all, name), err_msg=name)
+    keep = sorted({0, wl.n_requests - 1, int(np.argmin(stc.prefix_len)), int(np.argmax(stc.prefix_len))})
+    sp = H.sub_problem(stc, tokens, attn, None, keep)
+    opk = O.pack_wavefronts(sp["ocfg"], sp["ost"])
+    ref = O.wavefront_attn(sp["ocfg"], opk, sp["q"], sp["k_win"], sp["v_win"], sp["k_pool"], sp["v_pool"],
+                           sp["ost"].page_table)
+    n = len(sp["rows"])
+    got = sb.out[torch.from_numpy(sp["rows"]).to(DEV)].float().cpu().numpy().astype(np.float64)
+    err = np.abs(got - ref[:n])
+    rel = np.linalg.norm(got - ref[:n]) / np.linalg.norm(ref[:n])
+    assert err.max() <= 1e-2 and rel <= 5e-3, (err.max(), rel)
+    live = synth.n_live_slots(stc) * wl.block_len
+    assert bool(torch.isfinite(sb.out[:live].float()).all())
+    assert bool((sb.out[live:].float() == 7.0).all())
+
+
 def test_lm_head_fused_row_pass_full_vocabulary_sampled_rows():
     """The fused LM head at the benchmark's size (4,768 live rows, V = 151,552,
     hidden 2048): winners and confidences of sampled rows against the oracle's
