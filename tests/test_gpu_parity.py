@@ -237,7 +237,19 @@ def test_gate_commit_on_drawn_block_counts(seed, batch_sync):
     stragglers and every admission outcome occur; per-sequence and
     batch-synchronous policy, bit-exact against the oracle, K/V freeze included."""
     rg = np.random.default_rng(500 + seed)
-    Rn, W, n = int(rg.integers(1, 10)), int(rg.integers(1, 5)), 6
+    _gate_commit_case(rg, seed, batch_sync, int(rg.integers(1, 10)), int(rg.integers(1, 5)))
+
+
+@pytest.mark.parametrize("batch_sync", [0, 1])
+@pytest.mark.parametrize("Rn,W,seed", [(128, 4, 3), (600, 2, 4), (600, 3, 8)])
+def test_gate_commit_on_drawn_block_counts_many_requests(Rn, W, seed, batch_sync):
+    """The same with more requests than the reduction kernel has threads
+    (seeds 4 and 8 start from a shared window)."""
+    _gate_commit_case(np.random.default_rng(700 + seed), seed, batch_sync, Rn, W)
+
+
+def _gate_commit_case(rg, seed, batch_sync, Rn, W):
+    n = 6
     wl = synth.tiny_workload(n_requests=Rn, wmax=W, w_lo=1, w_hi=W, max_blocks=n,
                              n_q_heads=8, n_kv_heads=2, prefix_lo=0, prefix_hi=90)
     case = make_case(wl, seed=900 + seed, with_logits=False)
