@@ -399,9 +399,9 @@ def t2t_update(cfg: Config, pk: Pack, st: State, xhat, conf):
     ``force_progress = 1`` (READING; Eq. 1 is threshold-only and the paper
     names no fallback): if the oldest live block of a request went into the
     forward with masks and Eq. 1 revealed none of them, its masked position
-    with the highest confidence (lowest position on ties; confidences compared
-    in binary32, the precision the kernel holds them in) is revealed
-    (ACT_FORCED, counted as M2T).  Younger blocks are left to the thresholds:
+    with the highest confidence (lowest position on ties; the plain fp64
+    comparison of the confidences as given) is revealed (ACT_FORCED, counted
+    as M2T).  Younger blocks are left to the thresholds:
     their context is still immature (Sec. 2.2).  The oldest block then loses a
     mask every step, so a request terminates whatever the logits do.
 
@@ -442,7 +442,7 @@ def t2t_update(cfg: Config, pk: Pack, st: State, xhat, conf):
                 and stats[slot, ST_M2T] == 0):
             best = masked_before[0]
             for t in masked_before[1:]:
-                if np.float32(conf[slot * b + t]) > np.float32(conf[slot * b + best]):
+                if conf[slot * b + t] > conf[slot * b + best]:
                     best = t
             st.tokens[r, g * b + best] = xhat[slot * b + best]
             action[slot * b + best] = ACT_FORCED
