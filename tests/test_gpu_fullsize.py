@@ -139,14 +139,107 @@ def test_gate_commit_sampled_requests(full):
     assert c[O.CT_LIVE_SLOTS] == full["n_live"]
 
 
-def test_long_context_attention_sampled_requests():
+@pytest.fixture(scope="module")
+def longctx():
     """The long-context workload (16 requests, prefixes of 16K-32K tokens, three
-    live blocks of 64 tokens each) at full size: the first request runs as
-    whole work items, the last one falls into the stretch that the scheduler
-    cuts into filler pieces (partial results + combine kernel); all slots of
-    both against the oracle."""
+    live blocks of 64 tokens each) at full size, one whole step: pack,
+    attention, the T2T step over V = 151,552 calibrated logits, gate/commit."""
     wl = synth.WORKLOADS[3]
     stc = synth.make_structure(wl)
+    tokens = synth.make_tokens(stc)
+    n_live = synth.n_live_slots(stc)
+    z_live, tokens = synth.make_logits(stc, tokens, "calibrated", conf_shift=0.2, n_rows=n_live * wl.block_len)
+    attn = synth.make_attn_inputs(stc)
+    ctx = B.Context(**synth.config_dict(stc))
+    st = B.DeviceState.from_numpy(DEV, stc.active, stc.prefix_len, stc.L, stc.R, tokens,
+                                  np.zeros((wl.n_requests, wl.wmax), np.uint8), stc.page_table)
+    pk = B.PackBuffers.alloc(ctx, DEV)
+    sb = B.StepBuffers(ctx, DEV)
+    logits = torch.zeros(ctx.max_slots * wl.block_len, wl.vocab, dtype=torch.bfloat16, device=DEV)
+    logits[:z_live.shape[0]].copy_(z_live)
+    q, kw, vw, kp, vp = (t.to(DEV) for t in attn)
+    sb.out.fill_(7.0)
+    B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+    B.fb_wavefront_attn(ctx, pk, q, kw, vw, kp, vp, st.page_table, sb.out, sb.ws, sb.status)
+    B.fb_t2t_step(ctx, pk, logits, st, sb.argmax, sb.conf, sb.action, sb.slot_stats, sb.status)
+    B.fb_gate_commit(ctx, pk, sb.slot_stats, st, kw, vw, kp, vp, sb.n_committed, sb.spawned,
+                     sb.step_counters, sb.status)
+    torch.cuda.synchronize()
+    assert int(sb.status.item()) == 0
+    return dict(wl=wl, stc=stc, tokens=tokens, attn=attn, z_live=z_live, st=st, sb=sb, n_live=n_live,
+                keep=[0, wl.n_requests - 1])
+
+
+def test_long_context_attention_sampled_requests(longctx):
+    """The first request runs as whole work items, the last one falls into the
+    stretch that the scheduler cuts into filler pieces (partial results +
+    combine kernel); all slots of both against the oracle."""
+    wl, stc, sb = longctx["wl"], longctx["stc"], longctx["sb"]
+    hdr = sb.ws[:64].cpu().numpy().view(np.int32)
+    assert hdr[3] > 0, "no unit was split: the filler path is not exercised"
+    sp = H.sub_problem(stc, longctx["tokens"], longctx["attn"], None, longctx["keep"])
+    opk = O.pack_wavefronts(sp["ocfg"], sp["ost"])
+    ref = O.wavefront_attn(sp["ocfg"], opk, sp["q"], sp["k_win"], sp["v_win"], sp["k_pool"], sp["v_pool"],
+                           sp["ost"].page_table)
+    n = len(sp["rows"])
+    got = sb.out[torch.from_numpy(sp["rows"]).to(DEV)].float().cpu().numpy().astype(np.float64)
+    err = np.abs(got - ref[:n])
+    rel = np.linalg.norm(got - ref[:n]) / np.linalg.norm(ref[:n])
+    assert err.max() <= 1e-2 and rel <= 5e-3, (err.max(), rel)
+    assert n == 2 * 3 * wl.block_len
+    live = longctx["n_live"] * wl.block_len
+    assert bool(torch.isfinite(sb.out[:live].float()).all())
+    assert bool((sb.out[live:].float() == 7.0).all())
+
+
+def test_long_context_t2t_and_gate_sampled_requests(longctx):
+    """Eq. 1, the block counts, retirement and admission at the long-context
+    shape (bl 64, W 3, 3072 rows of 151,552 logits): every row of the two
+    sampled requests against the oracle's row pass, update and gate/commit."""
+    wl, stc, sb = longctx["wl"], longctx["stc"], longctx["sb"]
+    sp = H.sub_problem(stc, longctx["tokens"], longctx["attn"], longctx["z_live"], longctx["keep"])
+    opk = O.pack_wavefronts(sp["ocfg"], sp["ost"])
+    xhat, conf = O.t2t_rows(sp["ocfg"], opk, sp["logits"])
+    n = len(sp["rows"])
+    for thr in (np.float32(wl.tau_mask), np.float32(wl.tau_edit)):
+        assert np.abs(conf[:n] - float(thr)).min() >= 1e-3
+    action, stats = O.t2t_update(sp["ocfg"], opk, sp["ost"], xhat, conf)
+    ncom, spawned, ctr = O.gate_commit(sp["ocfg"], opk, stats, sp["ost"], sp["k_win"], sp["v_win"],
+                                       sp["k_pool"], sp["v_pool"])
+    rows = torch.from_numpy(sp["rows"]).to(DEV)
+    np.testing.assert_array_equal(sb.argmax[rows].cpu().numpy(), xhat[:n])
+    np.testing.assert_allclose(sb.conf[rows].cpu().numpy(), conf[:n], rtol=0, atol=2e-5)
+    np.testing.assert_array_equal(sb.action[rows].cpu().numpy(), action[:n])
+    assert (action[:n] == O.ACT_M2T).any() and (action[:n] == O.ACT_T2T).any()
+    slots = (sp["rows"][::wl.block_len] // wl.block_len).astype(np.int64)
+    np.testing.assert_array_equal(sb.slot_stats.cpu().numpy()[slots], stats[:len(slots)])
+    g = longctx["st"].to_numpy()
+    for r in longctx["keep"]:
+        assert int(sb.n_committed[r]) == int(ncom[r]) and int(sb.spawned[r]) == int(spawned[r])
+        for name in ("active", "prefix_len", "L", "R"):
+            assert int(g[name][r]) == int(getattr(sp["ost"], name)[r]), (name, r)
+        np.testing.assert_array_equal(g["pe_done"][r], sp["ost"].pe_done[r])
+        np.testing.assert_array_equal(g["tokens"][r], sp["ost"].tokens[r])
+    c = sb.step_counters.cpu().numpy()
+    assert c[O.CT_BLOCKS] == int(sb.n_committed.sum()) and c[O.CT_SPAWNED] == int(sb.spawned.sum())
+    assert c[O.CT_LIVE_SLOTS] == longctx["n_live"]
+
+
+@pytest.mark.parametrize("shape", ["longctx_32768_w3", "batch64_65536_w4"])
+def test_single_long_request_runs_entirely_as_split_pieces(shape):
+    """One decoding request with a very long prefix and nothing else in the
+    batch: every unit of the work list is cut along the key axis (the case that
+    drives the number of partial results to its bound; eight query heads keep
+    the oracle at seconds).  All rows against the oracle; the work list on the
+    device against the host-side plan."""
+    import dataclasses
+    if shape == "longctx_32768_w3":
+        wl = dataclasses.replace(synth.WORKLOADS[3], n_requests=4, prefix_lo=32768, prefix_hi=32768,
+                                 n_q_heads=8, n_kv_heads=2)
+    else:
+        wl = dataclasses.replace(synth.WORKLOADS[2], n_requests=4, prefix_lo=65536, prefix_hi=65536,
+                                 w_lo=4, w_hi=4, n_q_heads=8, n_kv_heads=2)
+    stc = synth.make_structure(wl, n_inactive=wl.n_requests - 1)
     tokens = synth.make_tokens(stc)
     attn = synth.make_attn_inputs(stc)
     ctx = B.Context(**synth.config_dict(stc))
@@ -160,22 +253,19 @@ def test_long_context_attention_sampled_requests():
     B.fb_wavefront_attn(ctx, pk, q, kw, vw, kp, vp, st.page_table, sb.out, sb.ws, sb.status)
     torch.cuda.synchronize()
     assert int(sb.status.item()) == 0
-    hdr = sb.ws[:64].cpu().numpy().view(np.int32)
-    assert hdr[3] > 0, "no unit was split: the filler path is not exercised"
-    keep = [0, wl.n_requests - 1]
-    sp = H.sub_problem(stc, tokens, attn, None, keep)
-    opk = O.pack_wavefronts(sp["ocfg"], sp["ost"])
-    ref = O.wavefront_attn(sp["ocfg"], opk, sp["q"], sp["k_win"], sp["v_win"], sp["k_pool"], sp["v_pool"],
-                           sp["ost"].page_table)
-    n = len(sp["rows"])
-    got = sb.out[torch.from_numpy(sp["rows"]).to(DEV)].float().cpu().numpy().astype(np.float64)
-    err = np.abs(got - ref[:n])
-    rel = np.linalg.norm(got - ref[:n]) / np.linalg.norm(ref[:n])
-    assert err.max() <= 1e-2 and rel <= 5e-3, (err.max(), rel)
-    assert n == 2 * 3 * wl.block_len
-    live = synth.n_live_slots(stc) * wl.block_len
-    assert bool(torch.isfinite(sb.out[:live].float()).all())
-    assert bool((sb.out[live:].float() == 7.0).all())
+    hdr = sb.ws[:64].cpu().numpy().view(np.int32)          # n_items, n_units, chunk length, n_parts
+    act = stc.active == 1
+    plan = ctx.attn_plan(stc.prefix_len[act], (stc.R - stc.L)[act])
+    assert (int(hdr[1]), int(hdr[0]), int(hdr[3])) == (plan["units"], plan["items"], plan["parts"])
+    assert plan["parts"] == plan["items"] > plan["units"], "every unit was meant to be split"
+    assert plan["parts"] <= plan["max_parts"]
+    ocfg = H.oracle_cfg(stc)
+    opk = O.pack_wavefronts(ocfg, H.oracle_state(stc, tokens))
+    ref = O.wavefront_attn(ocfg, opk, *(H.f64(t) for t in attn), stc.page_table)
+    rows = H.live_rows(opk, wl.block_len)
+    max_abs, rel = H.attn_errors(sb.out, ref, rows)
+    assert max_abs <= 1e-2 and rel <= 5e-3, (max_abs, rel)
+    assert bool((sb.out[len(rows):].float() == 7.0).all())
 
 
 @pytest.mark.parametrize("window_in_pages", [0, 1])

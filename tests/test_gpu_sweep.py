@@ -2,7 +2,7 @@
 arriving over 24 steps, 48 steps in all, confidences rising by 0.05 per step
 (the serving workload's structure: 512 slots, 64 blocks per request, prefixes of
 512-4096 tokens; the vocabulary is cut to 4096 so that the oracle's own row
-pass over every live row stays affordable).  After every step the tokens, the
+pass over every live row of every step stays affordable).  After every step the tokens, the
 window bounds, the prefix lengths, the per-step outputs and the frozen K/V of
 the blocks that retired are compared; commits and admissions of one step feed
 the next one on both sides."""
@@ -70,19 +70,14 @@ def test_serving_sweep_states_match_oracle_every_step(window_in_pages, batch_syn
         for name in ("slot_req", "slot_s", "slot_pos0", "slot_kv_len", "slot_flags", "req_slot_begin",
                      "qtok", "pos"):
             np.testing.assert_array_equal(g[name], getattr(opk, name), err_msg=f"{name}@{step}")
-        if step in (0, 7, 23, 47):
-            # the plain row pass of the oracle on the patched logits pins the declared
-            # winners and confidences
-            z64 = H.f64(run.z[:len(rows)].cpu())
-            full = np.zeros((n_rows, wl.vocab))
-            full[:len(rows)] = z64
-            xo, co = O.t2t_rows(ocfg, opk, full)
-            np.testing.assert_array_equal(xo[:len(rows)], cols)
-            assert np.abs(co[:len(rows)] - conf).max() < 1e-12
-        xhat = np.full(n_rows, -1, np.int32)
-        cf = np.zeros(n_rows)
-        xhat[rows] = cols
-        cf[rows] = conf
+        # Expected winners and confidences of EVERY step come from the oracle's own plain row
+        # pass over the patched logits as they stand on the device; the values the input
+        # generator declares for its patches are only cross-checked against them.
+        full = np.zeros((n_rows, wl.vocab))
+        full[:len(rows)] = H.f64(run.z[:len(rows)].cpu())
+        xhat, cf = O.t2t_rows(ocfg, opk, full)
+        np.testing.assert_array_equal(xhat[:len(rows)], cols, err_msg=f"declared winners@{step}")
+        assert np.abs(cf[:len(rows)] - conf).max() < 1e-12, f"declared confidences@{step}"
         before = dataclasses.replace(ost, prefix_len=ost.prefix_len.copy())
         action, stats = O.t2t_update(ocfg, opk, ost, xhat, cf)
         ncom, spawned, ctr = O.gate_commit(ocfg, opk, stats, ost)

@@ -2,16 +2,19 @@
 allocate device memory (an engine whose pool owns the whole device, a plugin
 in a pre-partitioned process, a loop that must avoid cudaMalloc's implicit
 synchronisation).  Its scratch is a fixed array inside the library, so the
-call takes no workspace.  Checked here against the regular entry point, twice
-in a row (the array keeps the first call's contents), and against its size
-limit.  This file sorts last on purpose: a run that stops at the first failure
+call takes no workspace.  Checked here against the CPU oracle (its work list
+never splits the key axis, a different schedule from the regular call's) and
+against the regular entry point, twice in a row (the array keeps the first
+call's contents), and against its size limit.  This file sorts last on purpose: a run that stops at the first failure
 has then already run every other test."""
 import numpy as np
 import pytest
 import torch
 
+from oracle import flowblock_oracle as O
 from paper_2607_17652_b200 import binding as B
 from paper_2607_17652_b200 import synth
+from tests import harness as H
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -30,6 +33,14 @@ def _setup(wl, seed=None):
     return stc, ctx, st, pk, sb, [t.to(DEV) for t in attn]
 
 
+def _oracle_attn(stc, q, kw, vw, kp, vp):
+    """fp64 attention of the oracle on the same bytes."""
+    ocfg = H.oracle_cfg(stc)
+    opk = O.pack_wavefronts(ocfg, H.oracle_state(stc, synth.make_tokens(stc)))
+    ref = O.wavefront_attn(ocfg, opk, *(H.f64(t.cpu()) for t in (q, kw, vw, kp, vp)), stc.page_table)
+    return ref, H.live_rows(opk, stc.wl.block_len)
+
+
 @pytest.mark.parametrize("wl", [synth.tiny_workload(prefix_lo=300, prefix_hi=2500, n_requests=5),
                                 synth.WORKLOADS[1]], ids=["tiny_long", "cfg1"])
 def test_static_scratch_attention_matches_workspace_attention(wl):
@@ -41,12 +52,16 @@ def test_static_scratch_attention_matches_workspace_attention(wl):
     torch.cuda.synchronize()
     want = sb.out[:live].float().clone()
     pack_ref = {k: v.copy() for k, v in pk.to_numpy().items()}
+    ref, ref_rows = _oracle_attn(stc, q, kw, vw, kp, vp)
+    assert len(ref_rows) == live
     for call in range(2):                       # two calls in a row share the array
         out = torch.full_like(sb.out, 3.0)
         B.fb_wavefront_attn_static(ctx, st, pk, q, kw, vw, kp, vp, out, sb.status)
         torch.cuda.synchronize()
         assert int(sb.status.item()) == 0
-        got = out[:live].float()
+        o_abs, o_rel = H.attn_errors(out, ref, ref_rows)                # against the oracle
+        assert o_abs <= ATTN_MAX_ABS and o_rel <= ATTN_REL_L2, (call, o_abs, o_rel)
+        got = out[:live].float()                                        # and against the regular call
         max_abs = float((got - want).abs().max())
         rel = float((got - want).norm() / want.norm())
         assert max_abs <= ATTN_MAX_ABS and rel <= ATTN_REL_L2, (call, max_abs, rel)
@@ -61,6 +76,9 @@ def test_static_scratch_attention_matches_workspace_attention(wl):
     out2 = torch.zeros_like(sb2.out)
     B.fb_wavefront_attn_static(ctx2, st2, pk2, q2, kw2, vw2, kp2, vp2, out2, sb2.status)
     torch.cuda.synchronize()
+    ref2, rows2 = _oracle_attn(stc2, q2, kw2, vw2, kp2, vp2)
+    o_abs, o_rel = H.attn_errors(out2, ref2, rows2)
+    assert o_abs <= ATTN_MAX_ABS and o_rel <= ATTN_REL_L2, (o_abs, o_rel)
     d = (out2[:live2].float() - sb2.out[:live2].float())
     assert float(d.abs().max()) <= ATTN_MAX_ABS
     assert float(d.norm() / sb2.out[:live2].float().norm()) <= ATTN_REL_L2
