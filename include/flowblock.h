@@ -29,6 +29,10 @@
  *   - K/V memory that a request's page table or the window tensors cover must
  *     hold finite values even where it is masked out (masked entries get
  *     weight exactly 0, and 0 * inf is not 0).
+ *   - A context belongs to one host thread at a time and to one device at a
+ *     time: the calls cache per-device set-up and tensor-map descriptors
+ *     inside it.  Use one context per thread / device; contexts are cheap.
+ *   - No environment variable is read anywhere.
  */
 #ifndef FLOWBLOCK_H
 #define FLOWBLOCK_H
@@ -160,10 +164,42 @@ int fb_create(const fb_config* cfg, fb_ctx** out);
 int fb_destroy(fb_ctx* ctx);
 const char* fb_last_error(const fb_ctx* ctx); /* ctx may be NULL */
 
+/* Execution knobs; no result depends on them beyond the rounding order of the
+ * split-KV merge.  The paper has no counterpart (it states no kernel design).
+ * 0 in a field selects the default. */
+typedef struct {
+  int32_t attn_target_items;     /* work items the key-axis split aims for
+                                    (default 2 x 148: two per SM); 1 = never
+                                    split, large = split down to the minimum  */
+  int32_t attn_min_chunk_tiles;  /* shortest key range of a split piece, in
+                                    128-key tiles (default 4)                 */
+  int64_t wait_cycles;           /* limit of every bounded device-side wait
+                                    (mbarrier, hand-off flags) in SM clock
+                                    cycles (default 2e9, about a second); when
+                                    it runs out the kernel stops issuing work,
+                                    sets FB_ST_DEV_TIMEOUT and returns        */
+} fb_tuning;
+
+/* Applies `t` to the context.  Changes fb_workspace_bytes(ctx): query it
+ * again and call before the first step.  FB_ERR_INVALID_ARG for negative or
+ * out-of-range values (attn_target_items <= 2^20, attn_min_chunk_tiles <=
+ * 4096). */
+int fb_set_tuning(fb_ctx* ctx, const fb_tuning* t);
+
 /* Bytes of device scratch the caller must pass as `ws` (256-byte aligned) to
  * fb_pack_wavefronts and fb_wavefront_attn of the same step: the attention
  * work list and the split-KV partial results. */
 size_t fb_workspace_bytes(const fb_ctx* ctx);
+
+/* Host-side mirror of the attention work-list arithmetic that
+ * fb_pack_wavefronts runs on the device (the paper has no counterpart: the
+ * work list is this library's execution plan).  For n <= max_requests decoding
+ * requests with HOST arrays h_prefix_len[n] and h_live_blocks[n] (R - L of
+ * each) it writes six int32 to h_out: units, work items and split pieces the
+ * batch produces, then the capacities max_units, max_items, max_parts that
+ * the workspace of this context is sized for.  No CUDA call is made. */
+int fb_attn_plan_host(const fb_ctx* ctx, const int32_t* h_prefix_len,
+                      const int32_t* h_live_blocks, int32_t n, int32_t* h_out);
 
 /* Sec. 3.2, Eq. 4 (gather): compacts the live blocks of all decoding
  * requests into slots, writes every array of `out`, pads the rest
@@ -239,6 +275,7 @@ int fb_embed_gather(fb_ctx* ctx, const fb_pack* pk, const void* table,
  *   - FB_ERR_UNSUPPORTED for contexts with window_in_pages = 1.
  *   - FB_ERR_WORKSPACE when the configuration's work list does not fit in
  *     8 MiB (about 100,000 (request, KV head, Q-tile pair) units).
+ *   - FB_ERR_INVALID_ARG when a member of `st` or `pk` or a tensor is NULL.
  *   - The first call on each device looks up the array's device address and
  *     sets kernel attributes; make that call outside any stream capture.
  *   - All calls on a device share the one array and it keeps the previous
@@ -314,7 +351,10 @@ int fb_gate_commit(fb_ctx* ctx, const fb_pack* pk, const int32_t* slot_stats,
  * step's q / k_win / v_win / logits from host (pinned) memory into the
  * caller's device staging buffers, runs the step, and copies n_committed,
  * spawned and step_counters back to host memory.  All asynchronous on
- * `stream`.  h_* are host pointers; everything else is as above. */
+ * `stream`.  h_* are host pointers; everything else is as above.  A harness
+ * convenience with no counterpart in the paper (its engine keeps Q/K/V and
+ * logits on the device); it is what an end-to-end timing with host buffers
+ * calls. */
 typedef struct {
   const void* h_q;
   const void* h_k_win;
@@ -322,7 +362,7 @@ typedef struct {
   const void* h_logits;
   int32_t* h_n_committed;    /* [R_max]  */
   uint8_t* h_spawned;        /* [R_max]  */
-  int32_t* h_step_counters;  /* [8]      */
+  int32_t* h_step_counters;  /* [FB_STEP_COUNTERS] */
   int32_t* h_status;         /* [1]      */
   int64_t n_rows;            /* leading rows of q / k_win / v_win / logits
                                 the caller has filled (live slots * bl);

@@ -29,7 +29,7 @@ EXPORTS = ["fb_create", "fb_destroy", "fb_last_error", "fb_workspace_bytes",
            "fb_pack_wavefronts", "fb_wavefront_attn", "fb_t2t_step",
            "fb_gate_commit", "fb_step_host", "fb_wavefront_attn_static",
            "fb_scatter_window_kv", "fb_embed_gather", "fb_lm_head_t2t",
-           "fb_lm_head_workspace_bytes"]
+           "fb_lm_head_workspace_bytes", "fb_set_tuning", "fb_attn_plan_host"]
 
 
 class fb_config(C.Structure):
@@ -41,6 +41,12 @@ class fb_config(C.Structure):
                                   "sm_scale")] + \
         [("window_in_pages", C.c_int32), ("batch_sync", C.c_int32),
          ("delta_literal", C.c_int32), ("force_progress", C.c_int32)]
+
+
+class fb_tuning(C.Structure):
+    _fields_ = [("attn_target_items", C.c_int32),
+                ("attn_min_chunk_tiles", C.c_int32),
+                ("wait_cycles", C.c_int64)]
 
 
 class fb_state(C.Structure):
@@ -87,6 +93,8 @@ def lib() -> C.CDLL:
         l.fb_last_error.restype = C.c_char_p
         l.fb_workspace_bytes.argtypes = [P]
         l.fb_workspace_bytes.restype = C.c_size_t
+        l.fb_set_tuning.argtypes = [P, C.POINTER(fb_tuning)]
+        l.fb_attn_plan_host.argtypes = [P, P, P, C.c_int32, P]
         l.fb_pack_wavefronts.argtypes = [P, C.POINTER(fb_state),
                                          C.POINTER(fb_pack), P, P, P]
         l.fb_wavefront_attn.argtypes = [P, C.POINTER(fb_pack)] + [P] * 10
@@ -136,14 +144,29 @@ def _stream(stream) -> int:
 
 
 class Context:
-    """Owns one fb_ctx."""
+    """Owns one fb_ctx.  ``tuning``: optional dict of fb_tuning fields."""
 
-    def __init__(self, **cfg):
+    def __init__(self, tuning=None, **cfg):
         self.cfg = fb_config(**cfg)
         self._h = C.c_void_p()
         rc = lib().fb_create(C.byref(self.cfg), C.byref(self._h))
         if rc != FB_OK:
             raise FlowBlockError(rc, lib().fb_last_error(None).decode())
+        if tuning:
+            self.set_tuning(**tuning)
+
+    def set_tuning(self, **tuning):
+        """fb_set_tuning; buffers sized by workspace_bytes() must be allocated after it."""
+        t = fb_tuning(**tuning)
+        self.check(lib().fb_set_tuning(self._h, C.byref(t)))
+
+    def attn_plan(self, prefix_len, live_blocks) -> dict:
+        """fb_attn_plan_host: what the attention work list of such a batch holds."""
+        p = np.ascontiguousarray(prefix_len, np.int32)
+        w = np.ascontiguousarray(live_blocks, np.int32)
+        out = np.zeros(6, np.int32)
+        self.check(lib().fb_attn_plan_host(self._h, p.ctypes.data, w.ctypes.data, len(p), out.ctypes.data))
+        return dict(zip(("units", "items", "parts", "max_units", "max_items", "max_parts"), map(int, out)))
 
     def __del__(self):
         try:

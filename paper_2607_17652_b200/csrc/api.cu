@@ -19,24 +19,27 @@ int fail(fb_ctx* ctx, int code, const std::string& msg) {
   return code;
 }
 
-fb::WsLayout make_layout(const fb_config& c, int tiles_per_slot, int target_items, int min_chunk_tiles) {
-  fb::WsLayout w{};
+}  // namespace
+
+namespace fb {
+
+WsLayout make_ws_layout(const fb_config& c, int tiles_per_slot, int target_items, int min_chunk_tiles) {
+  WsLayout w{};
   const long long qtiles = (long long)c.max_requests * c.wmax * tiles_per_slot;
   w.max_units = (int)((qtiles + c.max_requests + 1) / 2) * c.n_kv_heads;
-  // split units: at most 2 x target pieces from the coarse split, 1.2 x target more from the filler;
-  // and never more than every unit cut into pieces of the minimum length (a unit spans at most the
-  // keys its page-table row can address)
-  const long long max_tiles = ((long long)c.max_pages_per_req * fb::kPage + fb::kTileN - 1) / fb::kTileN + 2;
+  // split pieces: the bound that split_rule derives, and never more than every unit cut into
+  // pieces of the minimum length (a unit spans at most the keys its page-table row can address)
+  const long long max_tiles = ((long long)c.max_pages_per_req * kPage + kTileN - 1) / kTileN + 2;
   const long long every = (long long)w.max_units * ((max_tiles + min_chunk_tiles - 1) / min_chunk_tiles);
-  const long long by_target = 4ll * target_items + 8;
+  const long long by_target = (long long)kPartsPerTarget * target_items + 8;
   w.max_parts = (int)(by_target < every ? by_target : every);
   w.max_items = w.max_units + w.max_parts;
   size_t off = 0;
-  w.header = off;  off = align_up(off + sizeof(fb::SchedHeader), 256);
-  w.items = off;   off = align_up(off + (size_t)w.max_items * sizeof(fb::AttnItem), 256);
-  w.units = off;   off = align_up(off + (size_t)w.max_units * sizeof(fb::AttnUnit), 256);
-  w.part_ml = off; off = align_up(off + (size_t)w.max_parts * 2 * fb::kTileM * 2 * sizeof(float), 256);
-  w.part_o = off;  off = align_up(off + (size_t)w.max_parts * 2 * fb::kTileM * c.head_dim * sizeof(float), 256);
+  w.header = off;  off = align_up(off + sizeof(SchedHeader), 256);
+  w.items = off;   off = align_up(off + (size_t)w.max_items * sizeof(AttnItem), 256);
+  w.units = off;   off = align_up(off + (size_t)w.max_units * sizeof(AttnUnit), 256);
+  w.part_ml = off; off = align_up(off + (size_t)w.max_parts * 2 * kTileM * 2 * sizeof(float), 256);
+  w.part_o = off;  off = align_up(off + (size_t)w.max_parts * 2 * kTileM * c.head_dim * sizeof(float), 256);
   w.total = off;
   return w;
 }
@@ -61,7 +64,10 @@ int check_pack(fb_ctx* ctx, const fb_pack* pk) {
   return FB_OK;
 }
 
-}  // namespace
+}  // namespace fb
+
+using fb::check_pack;
+using fb::check_state;
 
 extern "C" {
 
@@ -107,24 +113,61 @@ int fb_create(const fb_config* cfg, fb_ctx** out) {
   ctx->tokens_per_tile = fb::kTileM / G;
   ctx->target_items = fb::kDefaultTargetItems;
   ctx->min_chunk_tiles = fb::kDefaultMinChunkTiles;
-  // tuning knobs of the split-KV work list (results do not depend on them)
-  if (const char* e = getenv("FB_ATTN_TARGET_ITEMS")) {
-    int v = atoi(e);
-    if (v >= 1 && v <= (1 << 20)) ctx->target_items = v;
-  }
-  if (const char* e = getenv("FB_ATTN_MIN_CHUNK_TILES")) {
-    int v = atoi(e);
-    if (v >= 1 && v <= 4096) ctx->min_chunk_tiles = v;
-  }
+  ctx->wait_cycles = fb::kDefaultWaitCycles;
   ctx->sm_scale = c.sm_scale > 0.f ? c.sm_scale : 1.0f / sqrtf((float)c.head_dim);
-  ctx->ws = make_layout(c, ctx->tiles_per_slot, ctx->target_items, ctx->min_chunk_tiles);
+  ctx->ws = fb::make_ws_layout(c, ctx->tiles_per_slot, ctx->target_items, ctx->min_chunk_tiles);
   *out = ctx;
+  return FB_OK;
+}
+
+int fb_set_tuning(fb_ctx* ctx, const fb_tuning* t) {
+  if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");
+  if (!t) return fail(ctx, FB_ERR_INVALID_ARG, "tuning is null");
+  if (t->attn_target_items < 0 || t->attn_target_items > (1 << 20) || t->attn_min_chunk_tiles < 0 ||
+      t->attn_min_chunk_tiles > 4096 || t->wait_cycles < 0)
+    return fail(ctx, FB_ERR_INVALID_ARG, "a tuning value is out of range");
+  ctx->target_items = t->attn_target_items ? t->attn_target_items : fb::kDefaultTargetItems;
+  ctx->min_chunk_tiles = t->attn_min_chunk_tiles ? t->attn_min_chunk_tiles : fb::kDefaultMinChunkTiles;
+  ctx->wait_cycles = t->wait_cycles ? (long long)t->wait_cycles : fb::kDefaultWaitCycles;
+  ctx->ws = fb::make_ws_layout(ctx->cfg, ctx->tiles_per_slot, ctx->target_items, ctx->min_chunk_tiles);
   return FB_OK;
 }
 
 int fb_destroy(fb_ctx* ctx) {
   if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");
+  fb::static_forget(ctx);
   delete ctx;
+  return FB_OK;
+}
+
+int fb_attn_plan_host(const fb_ctx* ctx, const int32_t* h_prefix_len, const int32_t* h_live_blocks, int32_t n,
+                      int32_t* h_out) {
+  if (!ctx || !h_prefix_len || !h_live_blocks || !h_out || n < 0 || n > ctx->cfg.max_requests)
+    return fail(nullptr, FB_ERR_INVALID_ARG, "fb_attn_plan_host: null argument or n outside [0, max_requests]");
+  const fb_config& c = ctx->cfg;
+  long long total = 0, units = 0;
+  for (int r = 0; r < n; ++r) {
+    if (h_live_blocks[r] < 0 || h_live_blocks[r] > c.wmax)
+      return fail(nullptr, FB_ERR_INVALID_ARG, "fb_attn_plan_host: live blocks outside [0, wmax]");
+    const fb::ReqGeom g = fb::req_geom_of(h_live_blocks[r], h_prefix_len[r], ctx->tiles_per_slot, c.block_len,
+                                          c.n_kv_heads, c.window_in_pages);
+    total += (long long)g.nunits * g.nt;
+    units += g.nt ? g.nunits : 0;
+  }
+  if (total > 0x7fffffffll) return fail(nullptr, FB_ERR_UNSUPPORTED, "fb_attn_plan_host: work list too long");
+  const fb::SplitRule rule = fb::split_rule((int)total, (int)units, ctx->target_items, ctx->min_chunk_tiles);
+  long long wbase = 0, items = 0, parts = 0;
+  for (int r = 0; r < n; ++r) {
+    const fb::ReqGeom g = fb::req_geom_of(h_live_blocks[r], h_prefix_len[r], ctx->tiles_per_slot, c.block_len,
+                                          c.n_kv_heads, c.window_in_pages);
+    const int nunits = g.nt ? g.nunits : 0;
+    const fb::ReqSplit rs = fb::req_split(rule, (int)wbase, nunits, g.nt);
+    items += rs.items(nunits);
+    parts += rs.parts(nunits);
+    wbase += (long long)nunits * g.nt;
+  }
+  h_out[0] = (int32_t)units; h_out[1] = (int32_t)items; h_out[2] = (int32_t)parts;
+  h_out[3] = ctx->ws.max_units; h_out[4] = ctx->ws.max_items; h_out[5] = ctx->ws.max_parts;
   return FB_OK;
 }
 

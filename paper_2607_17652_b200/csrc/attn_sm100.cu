@@ -33,8 +33,6 @@
 // workspace and a second kernel merges them in a fixed order.
 #include <cudaTypedefs.h>
 
-#include <cstdlib>
-
 #include "fb_common.cuh"
 #include "ptx_sm100.cuh"
 
@@ -47,21 +45,6 @@ constexpr float kRescaleThreshold = 8.0f;   // log2 units
 // offers, so two CTAs never share an SM: each CTA allocates all 512 TMEM columns.
 constexpr int kSmem64 = 120 * 1024;
 constexpr int kSmem128 = 6 * 32768 + 8192;
-
-// Optional per-role timeline of CTA 0 (debug builds with -DFB_TRACE only).
-#ifdef FB_TRACE
-#if FB_TRACE == 2      // light: one event per key tile from the MMA warp only
-#define FB_TR_ON(role, tag) ((role) == 1 && (tag) == 20)
-#elif FB_TRACE == 3    // tile A's softmax warps: tile boundaries and the epilogue
-#define FB_TR_ON(role, tag) ((role) == 2 && ((tag) >= 50 || (tag) == 41 || (tag) == 46))
-#else
-#define FB_TR_ON(role, tag) true
-#endif
-#define FB_TR(role, tag) do { if (FB_TR_ON(role, tag) && blockIdx.x == 0 && tr_n < 4096) { p.trace[(role) * 8192 + 2 * tr_n] = (tag); \
-    p.trace[(role) * 8192 + 2 * tr_n + 1] = clock64(); ++tr_n; } } while (0)
-#else
-#define FB_TR(role, tag) do { } while (0)
-#endif
 
 struct AttnParams {
   SchedHeader* hdr;
@@ -76,9 +59,6 @@ struct AttnParams {
   int32_t resident;     // 1: the window is read from the pages (every key tile is a paged one)
   float scale_log2;
   long long wait_cycles;
-#ifdef FB_TRACE
-  long long* trace;
-#endif
 };
 
 // Geometry of one work item, computed identically by every role.
@@ -109,9 +89,7 @@ __device__ __forceinline__ bool load_item(const AttnParams& p, int idx, ItemGeom
 // round-to-nearest split x = n + f, f in [-0.5, 0.5], cubic minimax fit of 2^f
 // (max relative error 7.5e-5, far below bf16 resolution), then n is added to
 // the exponent field.  Valid for -120 <= x <= 120.
-#ifndef FB_POLY_OF4
-#define FB_POLY_OF4 1      // pairs out of every 4 that take this path
-#endif
+constexpr int kPolyOf4 = 1;   // pairs out of every 4 that take this path
 __device__ __forceinline__ float2 exp2_poly2(float2 x) {
   x.x = fmaxf(x.x, -120.f);
   x.y = fmaxf(x.y, -120.f);
@@ -222,9 +200,6 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   const uint32_t tmem = *tmem_slot;
   pdl_wait();                     // the work list (and everything else) of the previous kernels is complete
   const int n_items = p.hdr->n_items;
-#ifdef FB_TRACE
-  if (tid == 0) { unsigned long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); p.trace[4 * 8192 + 2 * blockIdx.x] = (long long)g; }
-#endif
 
   // The control warpgroup (warps 0-3) hands registers to the softmax
   // warpgroups.  All four warps of a warpgroup execute the same setmaxnreg
@@ -248,7 +223,6 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     const int mine = warp >> 1;                    // the stage this warp fills
     int q_uses = 0, kfill = 0, vfill = 0, rr_k = 0, rr_v = 0;
     bool ok = true;
-    int tr_n = (leader && warp == 0) ? 0 : 1 << 30; (void)tr_n;
     // Page ids of the current request: lane i of pc_cur holds entry 32 * pc_blk + i of its
     // page-table row, pc_next the following 32 (loaded ahead), so a K/V tile costs two
     // shuffles instead of two dependent global loads.
@@ -283,7 +257,6 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         }
       }
       if (fill > 0 && !warp_wait(empty, (fill - 1) & 1, abortf, LIM)) return false;
-      FB_TR(0, isV ? 2 : 1);
       if (paged) {
 #pragma unroll
         for (int pg = 0; pg < 2; ++pg) {
@@ -305,7 +278,6 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       }
       __syncwarp();
       if (isV) ++vfill; else ++kfill;
-      FB_TR(0, isV ? 4 : 3);
       return true;
     };
     // Work items are handed out longest first through a global ticket; warp 0
@@ -319,11 +291,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         if (idx >= n_items) idx = -1;
         if (lane == 0) { s_item[k & 1] = idx; mbar_arrive(&item_full[k & 1]); }
         __syncwarp();
-        if (idx < 0) {
-          // the last CTA to run dry re-arms the ticket for the next launch
-          if (lane == 0 && atomicAdd(&p.hdr->done, 1) == (int)gridDim.x - 1) { p.hdr->ticket = 0; p.hdr->done = 0; }
-          break;
-        }
+        if (idx < 0) break;          // (the combine kernel re-arms the ticket for the next launch)
       } else {
         if (!warp_wait(&item_full[k & 1], (k >> 1) & 1, abortf, LIM)) { ok = false; break; }
         idx = s_item[k & 1];
@@ -333,13 +301,11 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       }
       ItemU g;
       if (!load_item_uniform(p, idx, g)) continue;
-      FB_TR(0, 10);
       pc_blk = (g.jb * 2) >> 5;
       pc_cur = load_pages(g.req, pc_blk);
       pc_next = load_pages(g.req, pc_blk + 1);
       if (warp == 0) {
         if (q_uses > 0 && !warp_wait(q_empty, (q_uses - 1) & 1, abortf, LIM)) { ok = false; break; }
-        FB_TR(0, 11);
         ++q_uses;
         if (leader) {
           mbar_arrive_expect_tx(q_full, ((g.nA > 0) + (g.nB > 0)) * TILE_BYTES);
@@ -373,7 +339,6 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     const bool leader = elect_one();
     int q_cnt = 0, cntPA = 0, cntPB = 0;
     bool ok = true;
-    int tr_n = leader ? 0 : 1 << 30; (void)tr_n;
     // All descriptors are built once; a k-step only adds a constant to the
     // address field (low word, no carry: shared-memory addresses fit the
     // 14-bit field).
@@ -431,15 +396,12 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       ItemU g;
       if (!load_item_uniform(p, idx, g)) continue;
       const int nA = g.nA, nB = g.nB, n = g.n;
-      FB_TR(1, 10);
       if (!warp_wait(q_full, q_cnt & 1, abortf, LIM)) { ok = false; break; }
       ++q_cnt;
-      FB_TR(1, 11);
       if (!g.dual()) {
         // ---- tiles A and B share every K/V tile
         int st = rr_k++ & 1;
         if (!wait_k(st)) { ok = false; break; }
-        FB_TR(1, 12);
         tc_fence_after();
         if (nA > 0) issue_qk(0, st, round16(g.limit(0, g.winA, p.resident)));
         if (nB > 0) issue_qk(1, st, round16(g.limit(0, g.winB, p.resident)));
@@ -448,33 +410,26 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         for (int j = 0; j < n; ++j) {
           const int sv = rr_v++ & 1;
           const int st1 = rr_k & 1;                // stage of K(j+1), if there is one
-          FB_TR(1, 20);
           if (!wait_v(sv)) { ok = false; break; }
           // K(j+1) has normally landed by now: taking its barrier here keeps the wait
           // off the P V -> next Q K^T stretch that the softmax warps are waiting for
           if (j + 1 < n) { ++rr_k; if (!wait_k(st1)) { ok = false; break; } }
-          FB_TR(1, 21);
           // tile A: O_A += P_A(j) V(j), then S_A(j+1) so that softmax A can go on
           if (j < nA) {
             const int nks = round16(g.limit(j, g.winA, p.resident)) >> 4;
             if (!warp_wait(&p_full[0], cntPA & 1, abortf, LIM)) { ok = false; break; }
-            FB_TR(1, 23);
             ++cntPA;
             tc_fence_after();
             issue_pv(0, sv, 0, nks, j > 0);
-            FB_TR(1, 24);
           }
           if (j + 1 < nA) {
-            FB_TR(1, 25);
             tc_fence_after();
             issue_qk(0, st1, round16(g.limit(j + 1, g.winA, p.resident)));
-            FB_TR(1, 26);
           }
           // tile B
           if (j < nB) {
             const int nks = round16(g.limit(j, g.winB, p.resident)) >> 4;
             if (!warp_wait(&p_full[1], cntPB & 1, abortf, LIM)) { ok = false; break; }
-            FB_TR(1, 33);
             ++cntPB;
             tc_fence_after();
             issue_pv(1, sv, 0, nks, j > 0);
@@ -493,7 +448,6 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         // ---- one Q tile under two KV heads: stream X owns K stage X and V stage X
         // (nA == nB == n, and both tiles see the same keys)
         if (!wait_k(0)) { ok = false; break; }
-        FB_TR(1, 12);
         tc_fence_after();
         issue_qk(0, 0, round16(g.limit(0, g.winA, p.resident)));
         commit(&k_empty[0]);
@@ -519,24 +473,19 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           }
           const int j = X ? jB : jA;
           if (X) { ++jB; ++cntPB; } else { ++jA; ++cntPA; }
-          FB_TR(1, X ? 33 : 23);
           if (!wait_v(X)) { ok = false; break; }
-          FB_TR(1, 34);
           tc_fence_after();
           issue_pv(X, X, 0, round16(g.limit(j, g.winA, p.resident)) >> 4, j > 0);
           commit(&v_empty[X]);
-          FB_TR(1, 35);
           if (j + 1 < n) {
             // this stream's next K tile could only be requested when its last Q K^T had
             // finished, one softmax ago: give it the time of the P V as well
             if (!wait_k(X)) { ok = false; break; }
-            FB_TR(1, 36);
             tc_fence_after();
             issue_qk(X, X, round16(g.limit(j + 1, g.winA, p.resident)));
             commit(&k_empty[X]);
             if (--qk_left == 0) commit(q_empty);
           }
-          FB_TR(1, 20);
           t0 = clock64();
         }
       }
@@ -558,7 +507,6 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     const float sl2 = p.scale_log2;
     int cntS = 0, cntO = 0;
     bool ok = true;
-    int tr_n = (quad == 0 && lane == 0) ? 0 : 1 << 30; (void)tr_n;
     for (int k = 0; ok; ++k) {
       if (!mbar_wait(&item_full[k & 1], (k >> 1) & 1, abortf, LIM)) { ok = false; break; }
       const int idx = s_item[k & 1];
@@ -572,9 +520,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       const int winX = X == 0 ? g.un.winA : g.un.winB;
       float m_ref = -INFINITY, l = 0.f;
       for (int j = 0; j < nMine; ++j) {
-        FB_TR(2 + X, 40);
         if (!mbar_wait(&s_full[X], cntS & 1, abortf, LIM)) { ok = false; break; }
-        FB_TR(2 + X, 41);
         ++cntS;
         tc_fence_after();
         const int limit = tile_limit(g, j, winX, p.resident);
@@ -607,7 +553,6 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                            64 + i + 8 + t < limit ? __uint_as_float(sb[i + 8 + t]) : -INFINITY);
           m_ref = fmaxf(fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3])), fmaxf(fmaxf(m8[4], m8[5]), fmaxf(m8[6], m8[7])));
         }
-        FB_TR(2 + X, 42);
         uint32_t pk[64];                       // P of this tile, packed bf16 pairs
         float tile_sum = 0.f;
 #pragma unroll 1
@@ -629,7 +574,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 const float2 x = __ffma2_rn(make_float2(__uint_as_float(sr[i]), __uint_as_float(sr[i + 1])), sl2v, nmb);
                 xm4[(i >> 1) & 3] = max3(xm4[(i >> 1) & 3], x.x, x.y);
                 float2 pv;
-                if (((i >> 1) & 3) < FB_POLY_OF4) pv = exp2_poly2(x);
+                if (((i >> 1) & 3) < kPolyOf4) pv = exp2_poly2(x);
                 else pv = make_float2(ex2_approx(x.x), ex2_approx(x.y));
                 acc2[(i >> 1) & 1] = __fadd2_rn(acc2[(i >> 1) & 1], pv);
                 pk[16 * c + (i >> 1)] = pack_bf16x2(pv.x, pv.y);
@@ -667,18 +612,13 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           tmem_st_wait();
         }
         l += tile_sum;
-        FB_TR(2 + X, 43);
         tmem_st32(tS, pk); tmem_st32(tS + 32, pk + 32);
         tmem_st_wait();
-        FB_TR(2 + X, 45);
         tc_fence_before();
         mbar_arrive(&p_full[X]);
-        FB_TR(2 + X, 46);
       }
       if (!ok) break;
-      FB_TR(2 + X, 50);
       if (!mbar_wait(&o_full[X], cntO & 1, abortf, LIM)) { ok = false; break; }
-      FB_TR(2 + X, 51);
       ++cntO;
       tc_fence_after();
       if (g.un.n_chunks <= 1) {
@@ -716,15 +656,11 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         }
       }
       tc_fence_before();
-      FB_TR(2 + X, 52);
     }
   }
   // ---------------------------------------------------------------- teardown
   tc_fence_before();
   __syncthreads();
-#ifdef FB_TRACE
-  if (tid == 0) { unsigned long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); p.trace[4 * 8192 + 2 * blockIdx.x + 1] = (long long)g; }
-#endif
   if (*abortf) {
     if (tid == 0) atomicOr(p.status, FB_ST_DEV_TIMEOUT);
     // give copies that are still in flight time to land before the CTA's
@@ -744,6 +680,9 @@ constexpr int kCombineCtasPerSm = 4;
 template <int D>
 __global__ void __launch_bounds__(256) attn_combine_kernel(const AttnParams p) {
   pdl_wait();
+  // The attention kernel is complete: re-arm its work ticket, so that the same work list can be
+  // run again (also after a launch that gave up on a bounded wait half way through its items).
+  if (blockIdx.x == 0 && threadIdx.x == 0) p.hdr->ticket = 0;
   if (p.hdr->n_parts == 0) return;
   const int n_pieces = p.hdr->n_units * kCombineSplit;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -801,16 +740,14 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const AttnParams p) {
 }
 
 // ------------------------------------------------------------------- host
-#ifdef FB_TRACE
-static long long* g_trace_ptr = nullptr;
-extern "C" int fb_debug_trace(long long* host_out) {
-  return (int)cudaMemcpy(host_out, g_trace_ptr, (4 * 8192 + 512) * sizeof(long long), cudaMemcpyDeviceToHost);
-}
-#endif
 int ensure_device(fb_ctx* ctx) {
-  if (ctx->dev_ready) return FB_OK;
   int dev = 0;
   if (int e = cuda_err(ctx, cudaGetDevice(&dev), "cudaGetDevice")) return e;
+  if (ctx->dev_ready && ctx->device == dev) return FB_OK;
+  // first use, or the caller moved the context to another device: set up again there and
+  // forget the cached tensor maps
+  ctx->dev_ready = false;
+  for (auto& mp : ctx->map_ptrs) mp = nullptr;
   cudaDeviceProp prop;
   if (int e = cuda_err(ctx, cudaGetDeviceProperties(&prop, dev), "cudaGetDeviceProperties")) return e;
   if (prop.major != 10) return set_err(ctx, FB_ERR_UNSUPPORTED, "the attention kernel needs an sm_100 device");
@@ -830,6 +767,8 @@ int ensure_device(fb_ctx* ctx) {
   if (int e = cuda_err(ctx, cudaFuncSetAttribute(wavefront_attn_kernel<128>,
                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, smem128), "smem attr"))
     return e;
+  if (int e = lm_head_device_setup(ctx)) return e;
+  ctx->device = dev;
   ctx->dev_ready = true;
   return FB_OK;
 }
@@ -892,15 +831,7 @@ int launch_attn(fb_ctx* ctx, const fb_pack* pk, const void* q, const void* k_win
   p.max_pages_per_req = c.max_pages_per_req; p.num_pages = c.num_pages;
   p.resident = c.window_in_pages;
   p.scale_log2 = ctx->sm_scale * kLog2eF;
-#ifdef FB_TRACE
-  static long long* g_trace = nullptr;
-  if (!g_trace) { cudaMalloc(&g_trace, (4 * 8192 + 512) * sizeof(long long)); }
-  cudaMemsetAsync(g_trace, 0, (4 * 8192 + 512) * sizeof(long long), stream);
-  p.trace = g_trace;
-  g_trace_ptr = g_trace;
-#endif
-  p.wait_cycles = 2000000000LL;
-  if (const char* e = getenv("FB_WAIT_CYCLES")) { long long v = atoll(e); if (v > 0) p.wait_cycles = v; }
+  p.wait_cycles = ctx->wait_cycles;
   const int grid = ctx->num_sms;
   const int combine_grid = min(ctx->ws.max_units * kCombineSplit, kCombineCtasPerSm * ctx->num_sms);
   if (c.head_dim == 64) {

@@ -54,11 +54,24 @@ fb::WsLayout unsplit_layout(const fb_ctx* c) {
 
 }  // namespace
 
+// fb_destroy calls this: the private context of a destroyed context goes with it, so a new
+// context that happens to be allocated at the same address starts from nothing.
+void fb::static_forget(const fb_ctx* ctx) {
+  std::lock_guard<std::mutex> lock(g_mu);
+  auto it = g_shadow.find(ctx);
+  if (it == g_shadow.end()) return;
+  delete it->second;
+  g_shadow.erase(it);
+}
+
 extern "C" int fb_wavefront_attn_static(fb_ctx* ctx, const fb_state* st, const fb_pack* pk, const void* q,
                                         const void* k_win, const void* v_win, const void* k_pool,
                                         const void* v_pool, void* out, int32_t* status, void* stream) {
   if (!ctx) return FB_ERR_INVALID_ARG;
-  if (!st || !pk || !q || !k_win || !v_win || !k_pool || !v_pool || !out || !status || !st->page_table)
+  // every array of the state and of the pack is read or written by the pack kernel
+  if (int e = fb::check_state(ctx, st)) return e;
+  if (int e = fb::check_pack(ctx, pk)) return e;
+  if (!q || !k_win || !v_win || !k_pool || !v_pool || !out || !status)
     return fb::set_err(ctx, FB_ERR_INVALID_ARG, "fb_wavefront_attn_static: a pointer is null");
   if (ctx->cfg.window_in_pages)
     return fb::set_err(ctx, FB_ERR_UNSUPPORTED, "fb_wavefront_attn_static: contexts with window_in_pages = 1 are not supported");
@@ -84,7 +97,6 @@ extern "C" int fb_wavefront_attn_static(fb_ctx* ctx, const fb_state* st, const f
     g_scratch_ptr[dev] = p;
   }
   fb_ctx*& sh = g_shadow[ctx];
-  if (sh && memcmp(&sh->cfg, &ctx->cfg, sizeof(fb_config)) != 0) { delete sh; sh = nullptr; }
   if (!sh) {
     sh = new fb_ctx();
     sh->cfg = ctx->cfg;
@@ -96,6 +108,7 @@ extern "C" int fb_wavefront_attn_static(fb_ctx* ctx, const fb_state* st, const f
     sh->min_chunk_tiles = 1 << 20;
     sh->ws = lay;
   }
+  sh->wait_cycles = ctx->wait_cycles;
   void* ws = g_scratch_ptr[dev];
   cudaStream_t s = (cudaStream_t)stream;
   // The work list is rebuilt from the current state by the pack kernel (it

@@ -45,6 +45,93 @@ struct WsLayout {
   int32_t max_items, max_units, max_parts;
 };
 
+// ---------------------------------------------------------------------------
+// Arithmetic of the attention work list, shared by the pack kernel (which
+// builds the list on the device) and by the host code that sizes the workspace.
+// ---------------------------------------------------------------------------
+
+// A request's Q tiles are paired two by two (a pair shares every K/V tile).
+// An odd tile left over is paired with itself across two adjacent KV heads
+// instead: the two halves stream different K/V but keep both tile slots of a
+// CTA busy, which a lone tile cannot.  nunits counts both kinds.
+struct ReqGeom {
+  int w, ntq, npairs, P, npt, nt;
+  int nfull, odd, nunits;   // full pairs per KV head; leftover tile; units of the request
+};
+__host__ __device__ inline ReqGeom req_geom_of(int w, int prefix_len, int tiles_per_slot, int bl, int n_kv_heads,
+                                               int resident) {
+  ReqGeom g;
+  g.w = w;
+  g.ntq = g.w * tiles_per_slot;
+  g.npairs = (g.ntq + 1) >> 1;
+  g.nfull = g.ntq >> 1;
+  g.odd = g.ntq & 1;
+  g.nunits = g.nfull * n_kv_heads + g.odd * ((n_kv_heads + 1) >> 1);
+  g.P = g.w ? (prefix_len > 0 ? prefix_len : 0) : 0;
+  g.npt = (g.P + kTileN - 1) / kTileN;
+  g.nt = g.w ? g.npt + (g.w * bl + kTileN - 1) / kTileN : 0;
+  if (resident) {         // one run of keys [0, P + w*bl), all of it paged
+    g.nt = g.w ? (g.P + g.w * bl + kTileN - 1) / kTileN : 0;
+    g.npt = g.nt;
+  }
+  return g;
+}
+
+// Key-axis split.  `total` = key-tile iterations of all units, `units` = units with work.
+//   ct        chunk length of the coarse split: ceil(total / target), at least min_chunk.
+//   fine_ct   chunk length of the filler pieces.  Items are handed out longest first, so the
+//             CTAs run dry within one shortest item of each other; when even the short items
+//             are long (few, long requests), the units whose work lies wholly inside the last
+//             15 % of the work are cut into pieces of 1/8 of a CTA's share (target = two items
+//             per CTA), which level that tail.
+//   fine_from work offset from which on a unit is a filler unit (INT_MAX: no filler).
+// Bound on the split pieces ("parts": chunks of units cut into more than one): a unit is only
+// cut when it is longer than its chunk length, so at most total / ct <= target coarse units are
+// cut, into at most 2 target pieces; the filler units hold at most 0.15 total + 1 tiles and
+// fine_ct >= total / (4 target), so at most 0.6 target + 1 of them are cut, into at most
+// 1.2 target + 2 pieces: parts <= 3.2 target + 2 <= kPartsPerTarget * target + 8.
+constexpr int kFillerPercent = 15;
+constexpr int kFillerDiv = 8;
+constexpr int kPartsPerTarget = 4;
+struct SplitRule { int ct, fine_ct, fine_from; };
+__host__ __device__ inline SplitRule split_rule(int total, int units, int target, int min_chunk) {
+  SplitRule s;
+  const int ct = (int)(((long long)total + target - 1) / target);
+  s.ct = ct < min_chunk ? min_chunk : ct;
+  const long long den = (long long)target * kFillerDiv;
+  const int fine = (int)((2ll * total + den - 1) / den);
+  s.fine_ct = fine < min_chunk ? min_chunk : fine;
+  const bool on = units > 0 && total / units > 2 * s.fine_ct && s.fine_ct < s.ct;
+  s.fine_from = on ? total - (int)((long long)kFillerPercent * total / 100) : 0x7fffffff;
+  return s;
+}
+// One request under the rule: its first `ufine` units take chunks of ct, the others (work
+// offset >= fine_from) chunks of fine_ct.  wbase = work offset of the request's first unit.
+struct ReqSplit {
+  int ufine, nch_c, nch_f;
+  __host__ __device__ int chunks(int ul) const { return ul < ufine ? nch_c : nch_f; }
+  __host__ __device__ int items(int nunits) const { return ufine * nch_c + (nunits - ufine) * nch_f; }
+  __host__ __device__ int parts(int nunits) const {
+    return (nch_c > 1 ? ufine * nch_c : 0) + (nch_f > 1 ? (nunits - ufine) * nch_f : 0);
+  }
+  // offset of unit ul's partial results inside the request's range (only used when chunks(ul) > 1)
+  __host__ __device__ int part_off(int ul) const {
+    return ul < ufine ? ul * nch_c : (nch_c > 1 ? ufine * nch_c : 0) + (ul - ufine) * nch_f;
+  }
+};
+__host__ __device__ inline ReqSplit req_split(const SplitRule& s, int wbase, int nunits, int nt) {
+  ReqSplit r;
+  r.ufine = nunits; r.nch_c = 0; r.nch_f = 0;
+  if (nt <= 0 || nunits <= 0) { r.ufine = 0; return r; }
+  r.nch_c = (nt + s.ct - 1) / s.ct;
+  r.nch_f = (nt + s.fine_ct - 1) / s.fine_ct;
+  if (s.fine_from != 0x7fffffff) {
+    const long long first = ((long long)s.fine_from - wbase + nt - 1) / nt;   // first unit with wbase + ul*nt >= fine_from
+    r.ufine = first < 0 ? 0 : (first > nunits ? nunits : (int)first);
+  }
+  return r;
+}
+
 }  // namespace fb
 
 struct fb_ctx {
@@ -54,11 +141,13 @@ struct fb_ctx {
   int tokens_per_tile;  // 128 / G
   int target_items;
   int min_chunk_tiles;
+  long long wait_cycles;  // limit of every bounded device-side wait, in SM clock cycles
   float sm_scale;
   fb::WsLayout ws;
   std::string err;
   // lazily initialised at the first attention launch
   bool dev_ready = false;
+  int device = -1;        // the device the lazily initialised members belong to
   int num_sms = 0;
   void* encode_fn = nullptr;
   // cached tensor maps (re-encoded when a base pointer changes)
@@ -115,6 +204,7 @@ int launch_lm_head(fb_ctx*, const fb_pack*, const void* x, const void* w, int hi
                    int32_t* argmax, float* conf, uint8_t* action, int32_t* slot_stats, void* ws, int32_t* status,
                    cudaStream_t);
 size_t lm_head_workspace_bytes(const fb_ctx*);
+int lm_head_device_setup(fb_ctx*);
 int launch_embed(fb_ctx*, const fb_pack*, const void* table, int table_rows, int hidden, void* x,
                  int32_t* status, cudaStream_t);
 int launch_t2t(fb_ctx*, const fb_pack*, const void* logits, const fb_state*, int32_t* argmax,
@@ -123,6 +213,13 @@ int launch_gate(fb_ctx*, const fb_pack*, const int32_t* slot_stats, const fb_sta
                 const void* k_win, const void* v_win, void* k_pool, void* v_pool,
                 int32_t* n_committed, uint8_t* spawned, int32_t* step_counters, int32_t* status,
                 cudaStream_t);
+
+constexpr long long kDefaultWaitCycles = 2000000000LL;   // about a second at the SM clock
+
+fb::WsLayout make_ws_layout(const fb_config& c, int tiles_per_slot, int target_items, int min_chunk_tiles);
+int check_state(fb_ctx* ctx, const fb_state* st);   // every member non-null, else FB_ERR_INVALID_ARG
+int check_pack(fb_ctx* ctx, const fb_pack* pk);
+void static_forget(const fb_ctx* ctx);              // drops what fb_wavefront_attn_static keeps per context
 
 inline int set_err(fb_ctx* ctx, int code, const std::string& msg) {
   if (ctx) ctx->err = msg;

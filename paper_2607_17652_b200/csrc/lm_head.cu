@@ -17,7 +17,6 @@
 #include <cudaTypedefs.h>
 
 #include <cfloat>
-#include <cstdlib>
 
 #include "fb_common.cuh"
 #include "ptx_sm100.cuh"
@@ -226,18 +225,17 @@ size_t lm_head_workspace_bytes(const fb_ctx* ctx) {
   return n_tiles_n * (size_t)lm_rows_pad(c) * sizeof(float4);
 }
 
+// per-device kernel attribute (called from ensure_device with that device current)
+int lm_head_device_setup(fb_ctx* ctx) {
+  return cuda_err(ctx, cudaFuncSetAttribute(lm_head_stats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            kLmSmem), "smem attr");
+}
+
 int launch_lm_head(fb_ctx* ctx, const fb_pack* pk, const void* x, const void* w, int hidden, const fb_state* st,
                    int32_t* argmax, float* conf, uint8_t* action, int32_t* slot_stats, void* ws, int32_t* status,
                    cudaStream_t stream) {
   if (int e = ensure_device(ctx)) return e;
   const fb_config& c = ctx->cfg;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (int e = cuda_err(ctx, cudaFuncSetAttribute(lm_head_stats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   kLmSmem), "smem attr"))
-      return e;
-    attr_set = true;
-  }
   const int rows = c.max_requests * c.wmax * c.block_len;
   auto fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled>(ctx->encode_fn);
   CUtensorMap tmX, tmW;
@@ -267,8 +265,7 @@ int launch_lm_head(fb_ctx* ctx, const fb_pack* pk, const void* x, const void* w,
   p.bl = c.block_len; p.vocab = c.vocab; p.hidden = hidden;
   p.n_tiles_n = (c.vocab + kLmBN - 1) / kLmBN;
   p.rows_pad = lm_rows_pad(c);
-  p.wait_cycles = 2000000000LL;
-  if (const char* e = getenv("FB_WAIT_CYCLES")) { long long v = atoll(e); if (v > 0) p.wait_cycles = v; }
+  p.wait_cycles = ctx->wait_cycles;
   lm_head_stats_kernel<<<ctx->num_sms, kLmThreads, kLmSmem, stream>>>(tmX, tmW, p);
   if (int e = cuda_err(ctx, cudaGetLastError(), "lm_head_stats_kernel launch")) return e;
   lm_head_merge_kernel<<<(rows + 7) / 8, 256, 0, stream>>>(p, argmax, conf, rows);

@@ -73,38 +73,8 @@ __device__ __forceinline__ int item_cost(int nA, int nB) {
   return (6 * n + both + 1) >> 1;
 }
 
-// A request's Q tiles are paired two by two (a pair shares every K/V tile).
-// An odd tile left over is paired with itself across two adjacent KV heads
-// instead: the two halves stream different K/V but keep both tile slots of a
-// CTA busy, which a lone tile cannot.  nunits counts both kinds.
-#ifndef FB_FILL_PCT
-#define FB_FILL_PCT 15
-#endif
-#ifndef FB_FILL_DIV
-#define FB_FILL_DIV 8
-#endif
-constexpr int kFillerPercent = FB_FILL_PCT;   // share of the key-tile work cut into filler pieces
-constexpr int kFillerDiv = FB_FILL_DIV;       // a filler piece is 1/kFillerDiv of a CTA's share
-struct ReqGeom {
-  int w, ntq, npairs, P, npt, nt;
-  int nfull, odd, nunits;   // full pairs per KV head; leftover tile; units of the request
-};
 __device__ __forceinline__ ReqGeom geom_of(const PackParams& p, int w, int prefix_len) {
-  ReqGeom g;
-  g.w = w;
-  g.ntq = g.w * p.tiles_per_slot;
-  g.npairs = (g.ntq + 1) >> 1;
-  g.nfull = g.ntq >> 1;
-  g.odd = g.ntq & 1;
-  g.nunits = g.nfull * p.n_kv_heads + g.odd * ((p.n_kv_heads + 1) >> 1);
-  g.P = g.w ? max(prefix_len, 0) : 0;
-  g.npt = (g.P + kTileN - 1) / kTileN;
-  g.nt = g.w ? g.npt + (g.w * p.bl + kTileN - 1) / kTileN : 0;
-  if (p.resident) {       // one run of keys [0, P + w*bl), all of it paged
-    g.nt = g.w ? (g.P + g.w * p.bl + kTileN - 1) / kTileN : 0;
-    g.npt = g.nt;
-  }
-  return g;
+  return req_geom_of(w, prefix_len, p.tiles_per_slot, p.bl, p.n_kv_heads, p.resident);
 }
 __device__ __forceinline__ ReqGeom req_geom(const PackParams& p, int r, int32_t* status) {
   const int w = live_blocks(p, r, status);
@@ -115,7 +85,7 @@ __device__ void build_sched(const PackParams& p) {
   __shared__ int sh_scan[kPackThreads / 32 + 1];
   __shared__ int bins[kCostBins];
   __shared__ int sh_total, sh_units;
-  __shared__ int sh_ct, sh_fine_ct, sh_fine_from;
+  __shared__ SplitRule sh_rule;
   const int tid = threadIdx.x;
   // bad states are reported once, by the gather blocks (null status here)
   // phase 1: total key-tile work -> chunk length
@@ -135,46 +105,31 @@ __device__ void build_sched(const PackParams& p) {
   __syncthreads();
   if ((tid & 31) == 0) { atomicAdd(&sh_total, mine); atomicAdd(&sh_units, mine_units); }
   __syncthreads();
-  if (tid == 0) {
-    const int ct = (sh_total + p.target_items - 1) / p.target_items;
-    sh_ct = ct < p.min_chunk_tiles ? p.min_chunk_tiles : ct;
-    // Filler: items are handed out longest first, so the CTAs run dry within one shortest
-    // item of each other.  When even the short items are long (few, long requests), the
-    // units of the last requests -- about 15 % of the work -- are cut into pieces of 1/8 of
-    // a CTA's share (target_items = two items per CTA), which level that tail.
-    const int share = (int)(2ll * sh_total / p.target_items);
-    const int fine = max(p.min_chunk_tiles, share / kFillerDiv);
-    const bool on = sh_units > 0 && sh_total / sh_units > 2 * fine && fine < sh_ct;
-    sh_fine_ct = fine;
-    sh_fine_from = on ? sh_total - (int)((long long)kFillerPercent * sh_total / 100) : 0x7fffffff;
-  }
+  if (tid == 0) sh_rule = split_rule(sh_total, sh_units, p.target_items, p.min_chunk_tiles);
   __syncthreads();
-  const int Ct = sh_ct, fineCt = sh_fine_ct, fineFrom = sh_fine_from;
+  const SplitRule rule = sh_rule;
   // phase 2 + 3: per-request bases (chunked scan), then one thread per unit of the chunk's
   // requests: unit record, cost histogram of its items
-  __shared__ int s_ub[kPackThreads + 1], s_pb[kPackThreads], s_first[kPackThreads], s_nch[kPackThreads],
+  __shared__ int s_ub[kPackThreads + 1], s_pb[kPackThreads], s_first[kPackThreads], s_wb[kPackThreads],
       s_w[kPackThreads], s_P[kPackThreads];
   int unit_run = 0, part_run = 0, item_run = 0, slot_run = 0, work_run = 0;
   for (int r0 = 0; r0 < p.max_requests; r0 += kPackThreads) {
     const int r = r0 + tid;
     ReqGeom g{};
-    int nch = 0, nunits = 0;
+    int nunits = 0;
     if (r < p.max_requests) {
       g = req_geom(p, r, nullptr);
-      nunits = g.nunits;
+      nunits = g.nt ? g.nunits : 0;
     }
     int tu, tp, ti, ts, tw;
     const int wbase = work_run + block_excl_scan(nunits * g.nt, &tw, sh_scan);
     work_run += tw;
-    if (g.nt) {
-      const int len = wbase + nunits * g.nt > fineFrom ? fineCt : Ct;
-      nch = (g.nt + len - 1) / len;
-    }
+    const ReqSplit rs = req_split(rule, wbase, nunits, g.nt);
     const int urel = block_excl_scan(nunits, &tu, sh_scan);
-    const int pbase = part_run + block_excl_scan(nch > 1 ? nunits * nch : 0, &tp, sh_scan);
-    block_excl_scan(nunits * nch, &ti, sh_scan);
+    const int pbase = part_run + block_excl_scan(rs.parts(nunits), &tp, sh_scan);
+    block_excl_scan(rs.items(nunits), &ti, sh_scan);
     const int first0 = slot_run + block_excl_scan(g.w, &ts, sh_scan);  // first slot of the request
-    s_ub[tid] = urel; s_pb[tid] = pbase; s_first[tid] = first0; s_nch[tid] = nch; s_w[tid] = g.w; s_P[tid] = g.P;
+    s_ub[tid] = urel; s_pb[tid] = pbase; s_first[tid] = first0; s_wb[tid] = wbase; s_w[tid] = g.w; s_P[tid] = g.P;
     if (tid == 0) s_ub[kPackThreads] = tu;
     __syncthreads();
     for (int i = tid; i < tu; i += kPackThreads) {
@@ -189,7 +144,8 @@ __device__ void build_sched(const PackParams& p) {
       const int u = unit_run + i;
       if (u >= p.max_units) continue;
       const ReqGeom q = geom_of(p, s_w[k], s_P[k]);
-      const int first = s_first[k], nc = s_nch[k];
+      const ReqSplit qs = req_split(rule, s_wb[k], q.nunits, q.nt);
+      const int first = s_first[k], nc = qs.chunks(ul);
       // Full pairs first, numbered h * nfull + pr: the pairs of one (request, KV head) are
       // adjacent, are handed out back to back and so share their K/V through L2.  Then the
       // leftover tile, one unit per two KV heads.
@@ -219,8 +175,10 @@ __device__ void build_sched(const PackParams& p) {
         un.slotB = -1; un.t0B = 0; un.winB = 0; un.nvisB = 0;
       }
       un.n_tiles = q.nt; un.n_chunks = nc;
-      un.part_base = nc > 1 ? s_pb[k] + ul * nc : -1;
-      if (nc > 1 && un.part_base + nc > p.max_parts) un.n_chunks = 0;  // cannot happen; see header
+      un.part_base = nc > 1 ? s_pb[k] + qs.part_off(ul) : -1;
+      // the workspace is sized for the bound on the split pieces (split_rule); a unit that
+      // would still fall outside it is dropped and FB_ST_BAD_STATE is raised below
+      if (nc > 1 && un.part_base + nc > p.max_parts) un.n_chunks = 0;
       un.prefix_len = q.P; un.npt = q.npt; un.win_row0 = first * p.bl;
       p.units[u] = un;
       for (int c = 0; c < un.n_chunks; ++c) {
@@ -248,7 +206,7 @@ __device__ void build_sched(const PackParams& p) {
     if (tid == 0) {
       p.hdr->n_items = min(total_items, p.max_items);
       p.hdr->n_units = min(unit_run, p.max_units);
-      p.hdr->chunk_tiles = Ct;
+      p.hdr->chunk_tiles = rule.ct;
       p.hdr->n_parts = part_run;
       p.hdr->total_tiles = sh_total;
       p.hdr->ticket = 0; p.hdr->done = 0;

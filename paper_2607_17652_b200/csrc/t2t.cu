@@ -18,14 +18,8 @@
 
 namespace fb {
 
-#ifndef FB_T2T_THREADS
-#define FB_T2T_THREADS 128
-#endif
-#ifndef FB_T2T_UNROLL
-#define FB_T2T_UNROLL 8
-#endif
-constexpr int kRowThreads = FB_T2T_THREADS;
-constexpr int kRowUnroll = FB_T2T_UNROLL;   // 16-byte loads in flight per thread
+constexpr int kRowThreads = 128;
+constexpr int kRowUnroll = 8;   // 16-byte loads in flight per thread
 constexpr float kLog2e = 1.4426950408889634f;
 
 __device__ __forceinline__ uint4 ld_stream16(const uint4* p) {

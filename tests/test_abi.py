@@ -38,7 +38,7 @@ def test_header_symbols_are_exported():
 
 def test_struct_layouts_match_header_order():
     hdr = open(os.path.join(ROOT, "include", "flowblock.h")).read()
-    for cls in (B.fb_config, B.fb_state, B.fb_pack, B.fb_host_io, B.fb_device_bufs):
+    for cls in (B.fb_config, B.fb_tuning, B.fb_state, B.fb_pack, B.fb_host_io, B.fb_device_bufs):
         body = re.search(r"typedef struct \{([^{}]*)\} %s;" % cls.__name__, hdr).group(1)
         body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
         names = re.findall(r"\*?\s*([A-Za-z_][A-Za-z0-9_]*)\s*[;,]", body)
@@ -106,3 +106,82 @@ def test_null_and_misaligned_arguments_are_rejected_on_the_host():
     assert lib.fb_step_host(ctx.handle, C.byref(full_st), C.byref(full_pk), None, None,
                             None) == B.FB_ERR_INVALID_ARG
     assert lib.fb_destroy(None) == B.FB_ERR_INVALID_ARG
+
+
+def test_static_entry_point_rejects_null_members_on_the_host():
+    """fb_wavefront_attn_static hands the state and pack arrays to the pack
+    kernel: a null member must come back as FB_ERR_INVALID_ARG, not reach a
+    launch."""
+    ctx = B.Context(**GOOD)
+    lib = B.lib()
+    for hole in range(7):
+        st = B.fb_state(*[None if i == hole else 0x1000 for i in range(7)])
+        pk = B.fb_pack(*([0x1000] * 9))
+        assert lib.fb_wavefront_attn_static(ctx.handle, C.byref(st), C.byref(pk), *([0x1000] * 7), None) \
+            == B.FB_ERR_INVALID_ARG, hole
+        assert b"state." in lib.fb_last_error(ctx.handle)
+    for hole in range(9):
+        st = B.fb_state(*([0x1000] * 7))
+        pk = B.fb_pack(*[None if i == hole else 0x1000 for i in range(9)])
+        assert lib.fb_wavefront_attn_static(ctx.handle, C.byref(st), C.byref(pk), *([0x1000] * 7), None) \
+            == B.FB_ERR_INVALID_ARG, hole
+        assert b"pack." in lib.fb_last_error(ctx.handle)
+    res = B.Context(**dict(GOOD, window_in_pages=1))
+    st, pk = B.fb_state(*([0x1000] * 7)), B.fb_pack(*([0x1000] * 9))
+    assert lib.fb_wavefront_attn_static(res.handle, C.byref(st), C.byref(pk), *([0x1000] * 7), None) \
+        == B.FB_ERR_UNSUPPORTED
+
+
+def test_tuning_is_validated_and_resizes_the_workspace():
+    ctx = B.Context(**GOOD)
+    base = ctx.workspace_bytes()
+    ctx.set_tuning(attn_target_items=100000)
+    assert ctx.workspace_bytes() >= base
+    ctx.set_tuning()                                   # zeros: back to the defaults
+    assert ctx.workspace_bytes() == base
+    for bad in (dict(attn_target_items=-1), dict(attn_min_chunk_tiles=5000), dict(wait_cycles=-5),
+                dict(attn_target_items=(1 << 20) + 1)):
+        with pytest.raises(B.FlowBlockError):
+            ctx.set_tuning(**bad)
+    assert B.lib().fb_set_tuning(ctx.handle, None) == B.FB_ERR_INVALID_ARG
+
+
+def _llm_cfg(**over):
+    return dict(dict(max_requests=16, wmax=3, block_len=64, n_q_heads=32, n_kv_heads=8, head_dim=128,
+                     page_size=64, num_pages=16 * 520, max_pages_per_req=520, vocab=1024, mask_id=1023,
+                     eos_id=1022, max_blocks=32, s_pe=1, tau_mask=0.9, tau_edit=0.95, theta_spawn=0.5,
+                     sm_scale=0.0), **over)
+
+
+def test_split_pieces_never_exceed_the_workspace_bound():
+    """The key-axis split of the attention work list, recomputed on the host by
+    the same arithmetic the pack kernel runs: for any batch the units, items
+    and split pieces fit what the workspace is sized for.  The hard cases are
+    few, long requests (everything becomes split pieces)."""
+    import numpy as np
+    rg = np.random.default_rng(5)
+    # one active long-context request among 16, every 64-aligned prefix in [16384, 32768]
+    ctx = B.Context(**_llm_cfg())
+    for P in range(16384, 32768 + 1, 64):
+        pl = ctx.attn_plan([P], [3])
+        assert pl["parts"] <= pl["max_parts"] and pl["items"] <= pl["max_items"], (P, pl)
+        assert pl["units"] == 24 and pl["items"] >= pl["units"]
+    # the batch-64 shape with one request of prefix 65536 and four live blocks
+    ctx = B.Context(**_llm_cfg(max_requests=64, wmax=4, block_len=32, max_pages_per_req=1030,
+                               num_pages=64 * 1030))
+    pl = ctx.attn_plan([65536], [4])
+    assert 0 < pl["parts"] <= pl["max_parts"], pl
+    # random batches, several tuning settings
+    for target, min_chunk in ((0, 0), (1, 0), (7, 1), (100000, 1), (296, 16), (50, 2)):
+        ctx.set_tuning(attn_target_items=target, attn_min_chunk_tiles=min_chunk)
+        for _ in range(300):
+            n = int(rg.integers(1, 65))
+            P = rg.integers(0, 65536, size=n)
+            if rg.random() < 0.3:
+                P[:] = rg.integers(0, 400)             # many short requests
+            w = rg.integers(0, 5, size=n)
+            pl = ctx.attn_plan(P, w)
+            assert pl["units"] <= pl["max_units"], pl
+            assert pl["items"] <= pl["max_items"], pl
+            assert pl["parts"] <= pl["max_parts"], (target, min_chunk, pl)
+    assert B.lib().fb_attn_plan_host(ctx.handle, None, None, 0, None) == B.FB_ERR_INVALID_ARG
