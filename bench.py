@@ -172,18 +172,81 @@ def combine_ranks(times_ms, work, device, world):
     return [float(x) for x in t.cpu()], [float(x) for x in w.cpu()]
 
 
+def free_port() -> int:
+    import socket
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def launch_replicas(args) -> int:
+    """`--gpus N` with N > 1 and no launcher environment: start the N ranks
+    ourselves (one process per GPU, the same command line under
+    torch.distributed.run on 127.0.0.1) and return their exit code."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def replica_env(args):
+    """(rank, world, local rank) of this process.  Under a launcher the world
+    is what was launched; a --gpus that disagrees with it is reported."""
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus and rank == 0:
+        print(f"bench.py: --gpus {args.gpus} but {world} rank(s) were launched; reporting n_gpus = {world}",
+              file=sys.stderr)
+    return rank, world, local
+
+
+def gather_ranks(record: dict, world):
+    """One small record per rank, collected on every rank (host objects: no
+    device memory is exchanged)."""
+    import torch.distributed as dist
+    if world == 1:
+        return [record]
+    out = [None] * world
+    dist.all_gather_object(out, record)
+    return out
+
+
+def run_dry(args):
+    """`--dry-run-cpu`: the replica plumbing without a GPU -- ranks over gloo,
+    rank-dependent seeds, the MAX-of-times / SUM-of-work reduction and the JSON
+    line -- with placeholder times and no kernel.  For tests of the launcher."""
+    import torch.distributed as dist
+    from paper_2607_17652_b200 import synth
+    rank, world, local = replica_env(args)
+    if world > 1:
+        dist.init_process_group("gloo")
+    wl = synth.tiny_workload()
+    stc = synth.make_structure(wl, synth.BASE_SEED + wl.index + 1000 * rank)
+    flops = attn_flops(stc)
+    (ms, e2e_ms), (flops_all,) = combine_ranks([1.0 + rank, 10.0 + rank], [flops], "cpu", world)
+    ranks = gather_ranks({"rank": rank, "local_rank": local, "seed": stc.seed, "attn_flops": flops}, world)
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "dry_run": True, "value": flops_all / ms / 1e9, "n_gpus": world,
+                          "ms_per_step": ms, "scaling": "weak",
+                          "config": {"workload": wl.name, "parallelism": f"replicas x{world}"},
+                          "e2e": {"ms_per_step": e2e_ms}, "ranks": ranks}), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 # ---------------------------------------------------------------- our arm
 def run_ours(args):
     import torch
     import torch.distributed as dist
     from paper_2607_17652_b200 import binding as B, synth
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = replica_env(args)
     torch.cuda.set_device(local)
     dev = f"cuda:{local}"
     if world > 1:
+        # replicas: NCCL only carries the MAX-of-times / SUM-of-work reduction at the end
         dist.init_process_group("nccl", device_id=torch.device(dev))
     wl = pick_workload(args)
     seed = synth.BASE_SEED + wl.index + 1000 * rank     # each rank its own batch
@@ -309,6 +372,10 @@ def run_ours(args):
                               "logits_bytes_not_moved": 2.0 * live_now * wl.block_len * wl.vocab * 2}
         del hx, hw, lws
 
+    # ------------- a step that commits: calibrated confidences, state reset before every timed step
+    if only == "all" and world == 1 and not args.no_calibrated:
+        nxt["step_calibrated"] = calibrated_step(args, wl, stc_init, dev, stream, q, kw, vw, kp, vp, logits, sb)
+
     # ------------------------------------------------------------ end to end
     e2e_ms, h2d, d2h = float("nan"), 0, 0
     if not args.no_e2e and only == "all":
@@ -339,7 +406,7 @@ def run_ours(args):
         barrier()
         e2e_ms = e0.elapsed_time(e1) / e2e_steps
         h2d = sum(host["n_rows"] * t[0].numel() * t.element_size() for t in (hq, hkw, hvw, hz))
-        d2h = wl.n_requests * 4 + wl.n_requests + 8 * 4 + 4
+        d2h = wl.n_requests * 4 + wl.n_requests + B.FB_STEP_COUNTERS * 4 + 4
     t2 = time.time()
     clocks = sampler.stop(t0, t2)
     clocks["window"] = "timed steps + end-to-end steps"
@@ -354,6 +421,8 @@ def run_ours(args):
     ms_step = total_ms / args.steps
     (ms_step_max, e2e_ms_max), (flops_all, t2tb_all) = combine_ranks(
         [ms_step, e2e_ms], [flops, t2t_bytes(stc, n_live)], dev, world)
+    ranks = gather_ranks({"rank": rank, "device": torch.cuda.get_device_name(local), "uuid": uuid, "seed": seed,
+                          "ms_per_step": round(ms_step, 4), "attn_tflop_per_step": round(flops / 1e12, 4)}, world)
 
     if rank == 0:
         peaks = load_peaks()
@@ -391,7 +460,7 @@ def run_ours(args):
                               "inputs fit in L2: a 256 MB write between the timed steps evicts them")},
             "clocks": clocks,
             "e2e": {"value": round(flops_all / e2e_ms_max / 1e9, 3),
-                    "unit": "TFLOP/s (attention FLOPs / whole-step time, host buffers)",
+                    "unit": "TFLOP/s (attention FLOPs / whole-step time)", "buffers": "host (pinned)",
                     "ms_per_step": round(e2e_ms_max, 3), "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h,
                     "t2t_gbs": round(t2tb_all / e2e_ms_max / 1e6, 2)},
@@ -405,6 +474,7 @@ def run_ours(args):
                         | {"kernel": dominant["kernel"], "peak_source": dominant["peak_source"]},
             "roofline_attn": roof_attn, "roofline_t2t": roof_t2t,
             "device_status": status, "step_counters": counters,
+            "ranks": ranks,
         }
         if nxt:
             nxt["lm_head_t2t"]["frac_of_measured_bf16"] = round(nxt["lm_head_t2t"]["tflops"] / peaks["bf16_tflops"], 4)
@@ -415,6 +485,57 @@ def run_ours(args):
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def calibrated_step(args, wl, stc, dev, stream, q, kw, vw, kp, vp, logits, sb):
+    """The bench workload's structure with confidence-calibrated logits (winner
+    confidences U(0.8, 0.999) on 70 % of the rows) and S_pe = 0, the initial
+    state restored before every timed step: each timed step reveals, edits,
+    retires blocks (KV freeze copy of Eq. 6) and admits new ones.  Device time
+    of the four calls by CUDA events; the logits of the main run are
+    overwritten."""
+    import torch
+    from paper_2607_17652_b200 import binding as B, synth
+    tokens0 = synth.make_tokens(stc)
+    n_live = synth.n_live_slots(stc)
+    z, tokens0 = synth.make_logits(stc, tokens0, "calibrated", conf_shift=0.3, n_rows=n_live * wl.block_len)
+    logits[:z.shape[0]].copy_(z)
+    ctx = B.Context(**synth.config_dict(stc, s_pe=0))
+    st = B.DeviceState.from_numpy(dev, stc.active, stc.prefix_len, stc.L, stc.R, tokens0,
+                                  np.zeros((wl.n_requests, wl.wmax), np.uint8), stc.page_table)
+    snap = {k: getattr(st, k).clone() for k in ("active", "prefix_len", "L", "R", "tokens", "pe_done")}
+    pk = B.PackBuffers.alloc(ctx, dev)
+    ws = B.alloc_workspace(ctx, dev)
+    n = max(3, min(args.steps, 10))
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(n)]
+    for k in range(3 + n):
+        for name, v in snap.items():
+            getattr(st, name).copy_(v)
+        e = evs[k - 3] if k >= 3 else None
+        if e: e[0].record(stream)
+        B.fb_pack_wavefronts(ctx, st, pk, ws, sb.status, stream)
+        if e: e[1].record(stream)
+        B.fb_wavefront_attn(ctx, pk, q, kw, vw, kp, vp, st.page_table, sb.out, ws, sb.status, stream)
+        if e: e[2].record(stream)
+        B.fb_t2t_step(ctx, pk, logits, st, sb.argmax, sb.conf, sb.action, sb.slot_stats, sb.status, stream)
+        if e: e[3].record(stream)
+        B.fb_gate_commit(ctx, pk, sb.slot_stats, st, kw, vw, kp, vp, sb.n_committed, sb.spawned,
+                         sb.step_counters, sb.status, stream)
+        if e: e[4].record(stream)
+    torch.cuda.synchronize()
+    seg = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(4)] for e in evs]).mean(0)
+    c = sb.step_counters.cpu().numpy().tolist()
+    blocks = c[0]
+    freeze_bytes = 2.0 * 2 * blocks * wl.block_len * wl.n_kv_heads * wl.head_dim * 2      # K and V, read + write
+    return {"ms": round(float(seg.sum()), 4), "pack_ms": round(float(seg[0]), 4), "attn_ms": round(float(seg[1]), 4),
+            "t2t_ms": round(float(seg[2]), 4), "gate_commit_ms": round(float(seg[3]), 4),
+            "attn_tflops": round(attn_flops(stc) / float(seg[1]) / 1e9, 2),
+            "t2t_gbs": round(t2t_bytes(stc, n_live) / float(seg[2]) / 1e6, 1),
+            "committed_blocks_per_step": blocks, "committed_tokens_per_step": c[1], "spawned_per_step": c[2],
+            "reveals_per_step": c[4], "edits_per_step": c[5], "finished_requests_per_step": c[3],
+            "kv_freeze_bytes": freeze_bytes, "kv_freeze_gbs": round(freeze_bytes / float(seg[3]) / 1e6, 1),
+            "logits": "calibrated (+0.3)", "s_pe": 0, "state": "initial state restored before every timed step",
+            "timed_steps": n, "device_status": int(sb.status.item())}
 
 
 # ------------------------------------------------------------ serving sweep
@@ -610,6 +731,9 @@ def main():
     ap.add_argument("--workload", type=int, default=DEFAULT_WORKLOAD)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-calibrated", action="store_true", help="skip next_rows.step_calibrated")
+    ap.add_argument("--dry-run-cpu", action="store_true",
+                    help="launcher / reduction plumbing only: gloo ranks on CPU, no kernel, placeholder times")
     ap.add_argument("--requests", type=int, default=0,
                     help="override the workload's request count (small cases for profiler captures)")
     ap.add_argument("--only", default="all", choices=["all", "attn", "t2t"],
@@ -631,8 +755,12 @@ def main():
                     help="run the serving workload as a 48-step sequence with arrivals (use with --workload 4)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        sys.exit(launch_replicas(args))
     if args.impl == "reference":
         run_reference(args)
+    elif args.dry_run_cpu:
+        run_dry(args)
     elif args.sweep:
         run_sweep(args)
     else:

@@ -211,7 +211,9 @@ def forced_reveal_margin(ocfg, opk, ost, tokens_before, action, conf):
     ("tiny_wide", "calibrated", 0.2, 1), ("tiny_d128_b64", "calibrated", 0.1, 3),
     ("tiny", "literal", 0.0, 1), ("cfg0", "normal2", 0.0, 1), ("tiny_v1000", "calibrated", 0.1, 1)])
 def test_t2t_and_gate_commit_bit_exact(name, kind, shift, s_pe):
-    case = make_case(WORKLOADS[name], logits_kind=kind, conf_shift=shift)
+    # the shifted case runs on a seed whose draw retires a block within this one step (most draws
+    # leave at least one mask in every oldest block)
+    case = make_case(WORKLOADS[name], seed=101 if shift >= 0.3 else None, logits_kind=kind, conf_shift=shift)
     res = run_t2t_and_gate(case, s_pe=s_pe)
     if kind == "calibrated":
         assert (res["action"] == O.ACT_M2T).any() and (res["action"] == O.ACT_T2T).any()

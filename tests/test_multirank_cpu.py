@@ -62,3 +62,35 @@ def test_flop_and_byte_counts_match_definition():
     assert bench.attn_flops(stc) == float(tot)
     n_live = synth.n_live_slots(stc)
     assert bench.t2t_bytes(stc, n_live) >= n_live * wl.block_len * wl.vocab * 2
+
+
+def _run_bench(*flags):
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items()
+           if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--dry-run-cpu", *flags],
+                       capture_output=True, text=True, timeout=300, env=env, cwd=root)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, r.stdout                       # rank 0 alone prints, one line
+    return json.loads(lines[0])
+
+
+def test_bench_starts_its_own_replicas_for_gpus_2():
+    """`python bench.py --gpus 2` with no launcher around it starts two ranks
+    itself (here over gloo, with the CUDA step left out): the line says two
+    GPUs, the ranks drew different batches, times are the MAX and work the SUM
+    over them."""
+    two = _run_bench("--gpus", "2")
+    assert two["n_gpus"] == 2 and two["config"]["parallelism"] == "replicas x2"
+    assert [r["rank"] for r in two["ranks"]] == [0, 1]
+    assert two["ranks"][0]["seed"] + 1000 == two["ranks"][1]["seed"]
+    assert two["ms_per_step"] == 2.0 and two["e2e"]["ms_per_step"] == 11.0
+    total = sum(r["attn_flops"] for r in two["ranks"])
+    assert abs(two["value"] - total / 2.0 / 1e9) < 1e-9 * total
+    one = _run_bench()
+    assert one["n_gpus"] == 1 and one["config"]["parallelism"] == "replicas x1"
+    assert one["ms_per_step"] == 1.0 and len(one["ranks"]) == 1
