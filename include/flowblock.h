@@ -177,7 +177,13 @@ typedef struct {
                                     (mbarrier, hand-off flags) in SM clock
                                     cycles (default 2e9, about a second); when
                                     it runs out the kernel stops issuing work,
-                                    sets FB_ST_DEV_TIMEOUT and returns        */
+                                    sets FB_ST_DEV_TIMEOUT and returns.  -1 is
+                                    the self-test of that path: every wait
+                                    gives up at once, so fb_wavefront_attn and
+                                    fb_lm_head_t2t do no useful work, set the
+                                    status bit and return (outputs undefined);
+                                    the next call with a positive limit runs
+                                    normally                                   */
 } fb_tuning;
 
 /* Applies `t` to the context.  Changes fb_workspace_bytes(ctx): query it

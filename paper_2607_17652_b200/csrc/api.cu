@@ -124,7 +124,7 @@ int fb_set_tuning(fb_ctx* ctx, const fb_tuning* t) {
   if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");
   if (!t) return fail(ctx, FB_ERR_INVALID_ARG, "tuning is null");
   if (t->attn_target_items < 0 || t->attn_target_items > (1 << 20) || t->attn_min_chunk_tiles < 0 ||
-      t->attn_min_chunk_tiles > 4096 || t->wait_cycles < 0)
+      t->attn_min_chunk_tiles > 4096 || t->wait_cycles < -1)
     return fail(ctx, FB_ERR_INVALID_ARG, "a tuning value is out of range");
   ctx->target_items = t->attn_target_items ? t->attn_target_items : fb::kDefaultTargetItems;
   ctx->min_chunk_tiles = t->attn_min_chunk_tiles ? t->attn_min_chunk_tiles : fb::kDefaultMinChunkTiles;

@@ -174,6 +174,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   uint64_t* item_full = bars + 20;   // [2] next work item published by the producer
   uint64_t* item_empty = bars + 22;  // [2] ... and read by the second producer, the MMA warp and the 8 softmax warps
   volatile int* s_item = reinterpret_cast<volatile int*>(bars + 24);   // [2]
+  uint64_t* drain = bars + 25;       // give-up path only: everything the MMA warp has issued is complete
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
   volatile int* abortf = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -189,6 +190,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 128); mbar_init(&o_full[i], 1);
       mbar_init(&item_full[i], 1); mbar_init(&item_empty[i], 10);
     }
+    mbar_init(drain, 1);
     fence_mbar_init();
     tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmKwin); tma_prefetch_desc(&tmVwin);
     tma_prefetch_desc(&tmKpool); tma_prefetch_desc(&tmVpool);
@@ -496,7 +498,9 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   }
   } else {
     // ------------------------------------------------- softmax + epilogue
-    // Four warps per Q tile, one thread per query row (its TMEM lane).
+    // Four warps per Q tile, one thread per query row (its TMEM lane).  Every wait is
+    // taken by the whole warp with one outcome (warp_wait): tcgen05.ld / st below are
+    // warp-wide and must never run with part of a warp gone.
     asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
     const int X = (warp - 4) >> 2;                 // 0: tile A, 1: tile B
     const int quad = warp & 3;                     // TMEM lane quadrant of this warp
@@ -508,7 +512,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     int cntS = 0, cntO = 0;
     bool ok = true;
     for (int k = 0; ok; ++k) {
-      if (!mbar_wait(&item_full[k & 1], (k >> 1) & 1, abortf, LIM)) { ok = false; break; }
+      if (!warp_wait(&item_full[k & 1], (k >> 1) & 1, abortf, LIM)) { ok = false; break; }
       const int idx = s_item[k & 1];
       __syncwarp();
       if (lane == 0) mbar_arrive(&item_empty[k & 1]);
@@ -520,7 +524,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       const int winX = X == 0 ? g.un.winA : g.un.winB;
       float m_ref = -INFINITY, l = 0.f;
       for (int j = 0; j < nMine; ++j) {
-        if (!mbar_wait(&s_full[X], cntS & 1, abortf, LIM)) { ok = false; break; }
+        if (!warp_wait(&s_full[X], cntS & 1, abortf, LIM)) { ok = false; break; }
         ++cntS;
         tc_fence_after();
         const int limit = tile_limit(g, j, winX, p.resident);
@@ -618,7 +622,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         mbar_arrive(&p_full[X]);
       }
       if (!ok) break;
-      if (!mbar_wait(&o_full[X], cntO & 1, abortf, LIM)) { ok = false; break; }
+      if (!warp_wait(&o_full[X], cntO & 1, abortf, LIM)) { ok = false; break; }
       ++cntO;
       tc_fence_after();
       if (g.un.n_chunks <= 1) {
@@ -662,9 +666,17 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   tc_fence_before();
   __syncthreads();
   if (*abortf) {
+    // A bounded wait gave up.  Nothing may still be running on this CTA's shared memory or
+    // TMEM when they are handed on: (1) the MMA warp commits everything it has issued to a
+    // barrier of its own and waits for it (bounded by a fixed number of polls: an MMA batch
+    // takes microseconds); (2) bulk copies the producers have issued land within
+    // microseconds as well, the CTA sleeps for 640 us before it leaves.
     if (tid == 0) atomicOr(p.status, FB_ST_DEV_TIMEOUT);
-    // give copies that are still in flight time to land before the CTA's
-    // shared memory is handed to the next one
+    if (warp == 1) {
+      if (elect_one()) umma_commit(drain);
+      __syncwarp();
+      for (int i = 0; i < 4096 && !mbar_test(drain, 0); ++i) __nanosleep(200);
+    }
     for (int i = 0; i < 64; ++i) __nanosleep(10000);
     __syncthreads();
   }

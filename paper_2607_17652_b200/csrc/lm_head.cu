@@ -52,6 +52,7 @@ lm_head_stats_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
   uint64_t* empty = bars + 4;               // [4] stage consumed (MMA commit)
   uint64_t* acc_full = bars + 8;            // [2] accumulator complete (MMA commit)
   uint64_t* acc_empty = bars + 10;          // [2] accumulator read out (4 epilogue warps)
+  uint64_t* drain = bars + 13;              // give-up path only
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
   volatile int* abortf = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -60,6 +61,7 @@ lm_head_stats_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     *abortf = 0;
     for (int i = 0; i < kLmStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 4); }
+    mbar_init(drain, 1);
     fence_mbar_init();
     tma_prefetch_desc(&tmX); tma_prefetch_desc(&tmW);
   }
@@ -128,7 +130,7 @@ lm_head_stats_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     bool ok = true;
     for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++i) {
       const int n = t / m_tiles, m = t % m_tiles, b = i & 1;
-      if (!mbar_wait(&acc_full[b], (i >> 1) & 1, abortf, LIM)) { ok = false; break; }
+      if (!lm_warp_wait(&acc_full[b], (i >> 1) & 1, abortf, LIM)) { ok = false; break; }   // one outcome per warp
       tc_fence_after();
       const uint32_t tacc = tmem + lane_base + b * kLmBN;
       const int col0 = n * kLmBN;
@@ -170,8 +172,15 @@ lm_head_stats_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
   tc_fence_before();
   __syncthreads();
   if (*abortf) {
+    // give-up path: the MMA warp waits for everything it has issued (own barrier, bounded
+    // polls), copies in flight land while the CTA sleeps, then TMEM and shared memory go back
     if (tid == 0) atomicOr(p.status, FB_ST_DEV_TIMEOUT);
-    for (int i = 0; i < 64; ++i) __nanosleep(10000);      // copies in flight land before the CTA's memory is reused
+    if (warp == 1) {
+      if (elect_one()) umma_commit(drain);
+      __syncwarp();
+      for (int i = 0; i < 4096 && !mbar_test(drain, 0); ++i) __nanosleep(200);
+    }
+    for (int i = 0; i < 64; ++i) __nanosleep(10000);
     __syncthreads();
   }
   if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem, 512); }

@@ -69,10 +69,12 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
 
 // Bounded wait.  Gives up after `limit` clock cycles or as soon as another
 // thread of the CTA has raised *abort; on giving up it raises *abort itself.
-// Returns true when the phase completed.
+// Returns true when the phase completed.  A negative limit is the self-test of
+// the give-up path: the wait gives up at once, whatever the barrier's state.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
                                           volatile int* abort,
                                           long long limit) {
+  if (limit < 0) { *abort = 1; return false; }
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   uint32_t spins = 0;
