@@ -45,6 +45,16 @@ Pins (tests/test_oracle_*.py, all CPU):
                          the logits; permuting the vocabulary permutes argmax
   rope_rotate            textbook special cases (position 0, d = 2 rotation,
                          norm, relative-offset invariance of q.k)
+  e4m3_decode / e4m3_quantize
+                         all 256 codes against the format's closed form and
+                         against a library conversion; round trip of every
+                         finite code; hand-worked ties, subnormals, saturation;
+                         monotonicity; power-of-two scale invariance
+  scatter_window_kv_fp8 / wavefront_attn_fp8
+                         placement as scatter_window_kv; with representable
+                         values and scale 1 both reduce to the bf16-path
+                         functions exactly; dequantised error <= half a code
+                         step; scale folded into the scores / the output
 Nothing in this file is "parity unpinned".
 
 Readings of the paper taken where it is silent or ambiguous are the named
@@ -330,6 +340,96 @@ def scatter_window_kv(cfg: Config, pk: Pack, k_new, v_new, k_pool, v_pool,
                 k = rope_rotate(k, pos, rope_base)
             k_pool[page, :, pos % ps, :] = k
             v_pool[page, :, pos % ps, :] = v_new[slot * b + t]
+
+
+# --------------------------------------------------------------------------
+# next: the KV pages held in 8 bits (FP8 E4M3)
+# --------------------------------------------------------------------------
+# READING (the paper states no numeric precision, Sec. 4.1; the cache is the
+# one Sec. 3.2 "KV Retrieval and Write-back" / Eq. 6 defines): a page stores
+# K and V as OCP FP8 E4M3 codes (1 sign, 4 exponent bits with bias 7, 3 mantissa
+# bits; no infinities, S.1111.111 is NaN, largest finite value 448) with one
+# binary32 scale per KV head for K and one for V, given by the caller:
+# stored code = e4m3(x / scale), value read back = code * scale.  One scale per
+# head and not per page, because a 64-token page is filled by several commits
+# of bl-token blocks and a per-page scale would have to re-quantise positions
+# that are already frozen (Sec. 3.1: a committed block's KV is exact and never
+# rewritten).  Where rounding decides the stored byte it is taken in binary32,
+# the precision the writer computes in: x / scale as a correctly rounded
+# binary32 quotient, then round-to-nearest-even onto the E4M3 grid, saturating
+# at +-448.
+E4M3_MAX = 448.0
+
+
+def e4m3_decode(codes) -> np.ndarray:
+    """Value of each E4M3 code (uint8 array) as float64: (-1)^s 2^(e-7) (1 + m/8)
+    for e > 0, (-1)^s 2^-6 (m/8) for e = 0; the two NaN codes give NaN."""
+    c = np.asarray(codes, np.uint8).astype(np.int64)
+    sgn = np.where(c & 0x80, -1.0, 1.0)
+    e = (c >> 3) & 0xF
+    m = (c & 7).astype(np.float64)
+    val = np.where(e > 0, np.ldexp(1.0 + m / 8.0, e - 7), np.ldexp(m / 8.0, -6))
+    val = sgn * val
+    return np.where((c & 0x7F) == 0x7F, np.nan, val)
+
+
+def e4m3_round(y) -> np.ndarray:
+    """Codes of the E4M3 values nearest to the finite numbers ``y`` (ties to
+    the even mantissa, magnitudes beyond 448 saturate to 448)."""
+    y = np.asarray(y, np.float64)
+    a = np.minimum(np.abs(y), E4M3_MAX)
+    # spacing of the grid around a: 2^(floor(log2 a) - 3) for normal values, 2^-9 below 2^-6
+    ex = np.floor(np.log2(np.maximum(a, 2.0 ** -6)))
+    step = np.exp2(ex - 3)
+    n = np.rint(a / step)                      # numpy rounds halves to even; a / step is exact (power of two)
+    v = n * step                               # may have carried into the next binade: still on the grid
+    e = np.floor(np.log2(np.maximum(v, 2.0 ** -6)))
+    is_sub = v < 2.0 ** -6
+    mant = np.where(is_sub, v / 2.0 ** -9, v / np.exp2(e - 3) - 8.0)
+    code = np.where(is_sub, mant, (e + 7) * 8 + mant).astype(np.int64)
+    code = np.where(np.signbit(y), code | 0x80, code)
+    return code.astype(np.uint8)
+
+
+def e4m3_quantize(x, scale) -> np.ndarray:
+    """Stored bytes of values ``x`` under ``scale`` (broadcast): the binary32
+    quotient x / scale rounded to E4M3."""
+    quot = (np.asarray(x, np.float64).astype(np.float32) / np.asarray(scale, np.float32)).astype(np.float64)
+    return e4m3_round(quot)
+
+
+def scatter_window_kv_fp8(cfg: Config, pk: Pack, k_new, v_new, k_pool8,
+                          v_pool8, k_scale, v_scale, page_table,
+                          rope_base: float = 0.0):
+    """scatter_window_kv into 8-bit pages: the (optionally rotated) fresh K/V
+    of every live window position are quantised with their KV head's scale and
+    stored at their absolute positions; in place on the uint8 pools
+    [num_pages, Hkv, page, d].  k_scale, v_scale [Hkv]."""
+    b, ps = cfg.block_len, cfg.page_size
+    ks = np.asarray(k_scale, np.float64)[:, None]
+    vs = np.asarray(v_scale, np.float64)[:, None]
+    for slot in range(pk.n_live):
+        r = int(pk.slot_req[slot])
+        for t in range(b):
+            pos = int(pk.slot_pos0[slot]) + t
+            page = int(page_table[r, pos // ps])
+            k = k_new[slot * b + t]
+            if rope_base > 0.0:
+                k = rope_rotate(k, pos, rope_base)
+            k_pool8[page, :, pos % ps, :] = e4m3_quantize(k, ks)
+            v_pool8[page, :, pos % ps, :] = e4m3_quantize(v_new[slot * b + t], vs)
+
+
+def wavefront_attn_fp8(cfg: Config, pk: Pack, q, k_pool8, v_pool8, k_scale,
+                       v_scale, page_table, only_slots=None) -> np.ndarray:
+    """wavefront_attn over 8-bit pages with the window resident in them: every
+    key and value is what the page gives back, code * scale of its KV head, in
+    float64; the queries are used as given."""
+    ks = np.asarray(k_scale, np.float64)[None, :, None, None]
+    vs = np.asarray(v_scale, np.float64)[None, :, None, None]
+    kd = e4m3_decode(k_pool8) * ks
+    vd = e4m3_decode(v_pool8) * vs
+    return wavefront_attn(cfg, pk, q, None, None, kd, vd, page_table, only_slots)
 
 
 def embed_gather(cfg: Config, pk: Pack, table):

@@ -201,6 +201,26 @@ def make_attn_inputs(stc: Structure, fill_unused: float | None = None):
     return q, k_win, v_win, k_pool, v_pool
 
 
+def make_fp8_kv(stc: Structure, amax: float = 6.0):
+    """8-bit KV pools for the FP8-page variant: per-KV-head scales (what a
+    calibration pass would hand over: ``amax`` standard deviations of N(0,1)
+    map to the top of the E4M3 range, times a per-head factor in [0.5, 2] so
+    that heads differ) and pools of random E4M3 bytes, drawn as N(0,1) / scale
+    and cast with the library's float8 type.  Returns (k_pool8, v_pool8) uint8
+    [num_pages, Hkv, page, d] and (k_scale, v_scale) float32 [Hkv]."""
+    wl = stc.wl
+    rg = _rng(stc.seed, 15)
+    ks = (amax / 448.0 * rg.uniform(0.5, 2.0, size=wl.n_kv_heads)).astype(np.float32)
+    vs = (amax / 448.0 * rg.uniform(0.5, 2.0, size=wl.n_kv_heads)).astype(np.float32)
+    shape = (stc.num_pages, wl.n_kv_heads, wl.page_size, wl.head_dim)
+    pools = []
+    for stream, sc in ((4, ks), (5, vs)):
+        x = randn_bf16(shape, stc.seed, stream).to(torch.float32)
+        x = (x / torch.from_numpy(sc)[None, :, None, None]).clamp_(-448.0, 448.0)
+        pools.append(x.to(torch.float8_e4m3fn).view(torch.uint8))
+    return pools[0], pools[1], torch.from_numpy(ks), torch.from_numpy(vs)
+
+
 def _slot_rows(stc: Structure):
     """(request, block, token) of every live row in slot order -- plain
     enumeration of live blocks, used only to place winners and tokens."""
