@@ -254,6 +254,43 @@ int fb_scatter_window_kv(fb_ctx* ctx, const fb_pack* pk,
                          const void* v_new, void* k_pool, void* v_pool,
                          float rope_base, int32_t* status, void* stream);
 
+/* The cache of Sec. 3.2 "KV Retrieval and Write-back" (Eq. 6) held in 8 bits.
+ * The paper states no numeric precision (Sec. 4.1); this is the reading taken:
+ * a page stores K and V as OCP FP8 E4M3 bytes (largest finite value 448, no
+ * infinities) and the caller supplies one fp32 scale per KV head for K and one
+ * for V (calibration is the model's business): stored byte = e4m3(x / scale),
+ * value read back = byte * scale.  x / scale is the correctly rounded fp32
+ * quotient, rounded to nearest even onto the E4M3 grid, saturating at +-448.
+ * One scale per head rather than per page: a page is filled by several commits
+ * and frozen positions are never rewritten.  Contexts need window_in_pages = 1
+ * (the scatter is the quantiser, so every key the attention reads is a paged
+ * 8-bit one) and head_dim = 128; FB_ERR_UNSUPPORTED otherwise.
+ *   k_pool8, v_pool8  [num_pages, n_kv_heads, 64, head_dim] uint8 (E4M3)
+ *   k_scale, v_scale  [n_kv_heads] fp32, positive, DEVICE pointers
+ *
+ * fb_scatter_window_kv_fp8: fb_scatter_window_kv into such pages (the rotary
+ * embedding, if asked for, is applied in fp32 before the division).
+ *
+ * fb_wavefront_attn_fp8: fb_wavefront_attn over such pages.  Both products run
+ * on the tensor cores in 8 bits: the queries are rounded to E4M3 after an exact
+ * per-row power-of-two scaling, and the softmax weights are rounded to E4M3
+ * (three mantissa bits) before they multiply V; accumulation is fp32, the
+ * row sums are taken from the unrounded weights.  Against exact arithmetic on
+ * the values the pages hold this costs a few percent of relative error per
+ * output row (the parity tests state and derive the bound); it is the price of
+ * the 8-bit tensor-core rate.  fb_gate_commit works unchanged (with the window
+ * in the pages it copies nothing); fb_step_host does not drive these calls. */
+int fb_scatter_window_kv_fp8(fb_ctx* ctx, const fb_pack* pk,
+                             const int32_t* page_table, const void* k_new,
+                             const void* v_new, void* k_pool8, void* v_pool8,
+                             const float* k_scale, const float* v_scale,
+                             float rope_base, int32_t* status, void* stream);
+int fb_wavefront_attn_fp8(fb_ctx* ctx, const fb_pack* pk, const void* q,
+                          const void* k_pool8, const void* v_pool8,
+                          const float* k_scale, const float* v_scale,
+                          const int32_t* page_table, void* out, void* ws,
+                          int32_t* status, void* stream);
+
 /* Sec. 3.2 Eq. 4 feeding the model: input embeddings of the packed window,
  * x[i, :] = table[qtok[i], :] for the rows of live slots (rows of padding
  * slots are not written).

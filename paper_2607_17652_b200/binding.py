@@ -29,7 +29,8 @@ EXPORTS = ["fb_create", "fb_destroy", "fb_last_error", "fb_workspace_bytes",
            "fb_pack_wavefronts", "fb_wavefront_attn", "fb_t2t_step",
            "fb_gate_commit", "fb_step_host", "fb_wavefront_attn_static",
            "fb_scatter_window_kv", "fb_embed_gather", "fb_lm_head_t2t",
-           "fb_lm_head_workspace_bytes", "fb_set_tuning", "fb_attn_plan_host"]
+           "fb_lm_head_workspace_bytes", "fb_set_tuning", "fb_attn_plan_host",
+           "fb_scatter_window_kv_fp8", "fb_wavefront_attn_fp8"]
 
 
 class fb_config(C.Structure):
@@ -106,6 +107,9 @@ def lib() -> C.CDLL:
                                                C.POINTER(fb_pack)] + [P] * 8
         l.fb_scatter_window_kv.argtypes = [P, C.POINTER(fb_pack)] + [P] * 5 + \
             [C.c_float, P, P]
+        l.fb_scatter_window_kv_fp8.argtypes = [P, C.POINTER(fb_pack)] + [P] * 7 + \
+            [C.c_float, P, P]
+        l.fb_wavefront_attn_fp8.argtypes = [P, C.POINTER(fb_pack)] + [P] * 10
         l.fb_embed_gather.argtypes = [P, C.POINTER(fb_pack), P, C.c_int32,
                                       C.c_int32, P, P, P]
         l.fb_lm_head_workspace_bytes.argtypes = [P]
@@ -275,6 +279,28 @@ def fb_scatter_window_kv(ctx: Context, pk: PackBuffers, page_table, k_new, v_new
         ctx.handle, C.byref(p), _ptr(page_table), _ptr(k_new), _ptr(v_new),
         _ptr(k_pool), _ptr(v_pool), C.c_float(rope_base), _ptr(status),
         _stream(stream)))
+
+
+def fb_scatter_window_kv_fp8(ctx: Context, pk: PackBuffers, page_table, k_new, v_new,
+                             k_pool8, v_pool8, k_scale, v_scale, status,
+                             rope_base: float = 0.0, stream=None):
+    """Eq. 6 into 8-bit (E4M3) pages with per-KV-head scales."""
+    p = pk.c()
+    ctx.check(lib().fb_scatter_window_kv_fp8(
+        ctx.handle, C.byref(p), _ptr(page_table), _ptr(k_new), _ptr(v_new),
+        _ptr(k_pool8), _ptr(v_pool8), _ptr(k_scale), _ptr(v_scale),
+        C.c_float(rope_base), _ptr(status), _stream(stream)))
+
+
+def fb_wavefront_attn_fp8(ctx: Context, pk: PackBuffers, q, k_pool8, v_pool8,
+                          k_scale, v_scale, page_table, out, ws, status,
+                          stream=None):
+    """Attention over 8-bit (E4M3) pages, window resident in the pages."""
+    p = pk.c()
+    ctx.check(lib().fb_wavefront_attn_fp8(
+        ctx.handle, C.byref(p), _ptr(q), _ptr(k_pool8), _ptr(v_pool8),
+        _ptr(k_scale), _ptr(v_scale), _ptr(page_table), _ptr(out), _ptr(ws),
+        _ptr(status), _stream(stream)))
 
 
 def fb_embed_gather(ctx: Context, pk: PackBuffers, table, x, status, stream=None):

@@ -221,6 +221,45 @@ int fb_scatter_window_kv(fb_ctx* ctx, const fb_pack* pk, const int32_t* page_tab
                             (cudaStream_t)stream);
 }
 
+static int check_fp8_ctx(fb_ctx* ctx) {
+  if (!ctx->cfg.window_in_pages)
+    return fail(ctx, FB_ERR_UNSUPPORTED, "8-bit KV pages need a context with window_in_pages = 1 (the window is quantised into the pages by the scatter)");
+  if (ctx->cfg.head_dim != 128) return fail(ctx, FB_ERR_UNSUPPORTED, "8-bit KV pages: head_dim must be 128");
+  return FB_OK;
+}
+
+int fb_scatter_window_kv_fp8(fb_ctx* ctx, const fb_pack* pk, const int32_t* page_table, const void* k_new,
+                             const void* v_new, void* k_pool8, void* v_pool8, const float* k_scale,
+                             const float* v_scale, float rope_base, int32_t* status, void* stream) {
+  if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");
+  if (int e = check_pack(ctx, pk)) return e;
+  if (int e = check_fp8_ctx(ctx)) return e;
+  if (!page_table || !k_new || !v_new || !k_pool8 || !v_pool8 || !k_scale || !v_scale || !status)
+    return fail(ctx, FB_ERR_INVALID_ARG, "a tensor pointer is null");
+  if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_pool8) || !aligned16(v_pool8))
+    return fail(ctx, FB_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  if (!(rope_base == rope_base) || rope_base < 0.f) return fail(ctx, FB_ERR_INVALID_ARG, "rope_base is NaN or negative");
+  return fb::launch_scatter_fp8(ctx, pk, page_table, k_new, v_new, k_pool8, v_pool8, k_scale, v_scale, rope_base,
+                                status, (cudaStream_t)stream);
+}
+
+int fb_wavefront_attn_fp8(fb_ctx* ctx, const fb_pack* pk, const void* q, const void* k_pool8, const void* v_pool8,
+                          const float* k_scale, const float* v_scale, const int32_t* page_table, void* out,
+                          void* ws, int32_t* status, void* stream) {
+  if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");
+  if (int e = check_pack(ctx, pk)) return e;
+  if (int e = check_fp8_ctx(ctx)) return e;
+  if (!q || !k_pool8 || !v_pool8 || !k_scale || !v_scale || !page_table || !out)
+    return fail(ctx, FB_ERR_INVALID_ARG, "a tensor pointer is null");
+  if (!ws) return fail(ctx, FB_ERR_WORKSPACE, "workspace is null");
+  if (!status) return fail(ctx, FB_ERR_INVALID_ARG, "status is null");
+  if (!aligned16(q) || !aligned16(k_pool8) || !aligned16(v_pool8) || !aligned16(out))
+    return fail(ctx, FB_ERR_ALIGNMENT, "tensor pointers must be 16-byte aligned");
+  if (reinterpret_cast<uintptr_t>(ws) & 255u) return fail(ctx, FB_ERR_ALIGNMENT, "workspace must be 256-byte aligned");
+  return fb::launch_attn_fp8(ctx, pk, q, k_pool8, v_pool8, k_scale, v_scale, page_table, out, ws, status,
+                             (cudaStream_t)stream);
+}
+
 int fb_embed_gather(fb_ctx* ctx, const fb_pack* pk, const void* table, int32_t table_rows, int32_t hidden,
                     void* x, int32_t* status, void* stream) {
   if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");

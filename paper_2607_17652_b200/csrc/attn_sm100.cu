@@ -45,6 +45,10 @@ constexpr float kRescaleThreshold = 8.0f;   // log2 units
 // offers, so two CTAs never share an SM: each CTA allocates all 512 TMEM columns.
 constexpr int kSmem64 = 120 * 1024;
 constexpr int kSmem128 = 6 * 32768 + 8192;
+constexpr int kSmemF8 = 2 * 32768 + 6 * 16384 + 8192;   // Q staging (bf16), Q / K / V tiles in 8 bits
+// 8-bit pages: the exponentials are taken 2^4 above the reference, so that E4M3 (normal down to
+// 2^-6, largest value 448) holds P from 2^-10 of the reference up to the 2^8 bound of the lazy re-base
+constexpr float kF8PShift = 4.0f;
 
 struct AttnParams {
   SchedHeader* hdr;
@@ -57,6 +61,8 @@ struct AttnParams {
   int32_t* status;
   int32_t bl, n_q_heads, n_kv_heads, group, max_pages_per_req, num_pages;
   int32_t resident;     // 1: the window is read from the pages (every key tile is a paged one)
+  const float* k_scale; // 8-bit pages only: value = code * scale of the KV head, [n_kv_heads]
+  const float* v_scale;
   float scale_log2;
   long long wait_cycles;
 };
@@ -148,18 +154,27 @@ __device__ __forceinline__ int tile_limit(const ItemGeom& g, int j, int winX, in
 }
 __device__ __forceinline__ int round16(int x) { return (x + 15) & ~15; }
 
-template <int D>
+// F8: the KV pages hold FP8 E4M3 bytes (window resident in the pages, D = 128).  Both products
+// then run as kind::f8f6f4 MMAs: the softmax warps convert their Q tile to E4M3 once per item
+// (per-row power-of-two scale, undone in the row's score factor together with the K scale of
+// the KV head) and write P as E4M3; O is scaled by the V scale of the KV head at the end.
+template <int D, bool F8>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKwin,
                       const __grid_constant__ CUtensorMap tmVwin, const __grid_constant__ CUtensorMap tmKpool,
                       const __grid_constant__ CUtensorMap tmVpool, const AttnParams p) {
-  constexpr int NH = D / 64;                 // 64-element halves of the head dim
-  constexpr int TILE_BYTES = NH * 16384;     // one 128-row operand tile
-  constexpr int PAGE_BYTES = NH * 8192;      // one 64-row page of it
+  static_assert(!F8 || D == 128, "8-bit pages: head_dim 128 only (one 128-byte swizzle row per key)");
+  constexpr int NH = D / 64;                 // 64-element halves of the head dim (bf16 tiles)
+  constexpr int Q_TILE_BYTES = NH * 16384;   // one 128-row bf16 tile
+  constexpr int NHKV = F8 ? 1 : NH;          // 16 KB blocks of a K/V tile
+  constexpr int TILE_BYTES = NHKV * 16384;   // one 128-key K or V tile
+  constexpr int PAGE_BYTES = NHKV * 8192;    // one 64-key page of it
+  constexpr int KSTEPS = F8 ? D / 32 : D / 16;   // MMAs per Q K^T
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sQ = smem;                        // [2] tiles A, B
-  uint8_t* sK = sQ + 2 * TILE_BYTES;         // [2] stages
+  uint8_t* sQ = smem;                        // [2] tiles A, B (bf16, as loaded)
+  uint8_t* sQ8 = sQ + 2 * Q_TILE_BYTES;      // [2] the same in E4M3 (F8 only)
+  uint8_t* sK = sQ8 + (F8 ? 2 * 16384 : 0);  // [2] stages
   uint8_t* sV = sK + 2 * TILE_BYTES;         // [2] stages
   uint64_t* bars = reinterpret_cast<uint64_t*>(sV + 2 * TILE_BYTES);
   uint64_t* q_full = bars + 0;
@@ -175,6 +190,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   uint64_t* item_empty = bars + 22;  // [2] ... and read by the second producer, the MMA warp and the 8 softmax warps
   volatile int* s_item = reinterpret_cast<volatile int*>(bars + 24);   // [2]
   uint64_t* drain = bars + 25;       // give-up path only: everything the MMA warp has issued is complete
+  uint64_t* q8_full = bars + 26;     // [2] F8: tile X converted to E4M3 by its 128 softmax threads
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
   volatile int* abortf = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -191,6 +207,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       mbar_init(&item_full[i], 1); mbar_init(&item_empty[i], 10);
     }
     mbar_init(drain, 1);
+    mbar_init(&q8_full[0], 128); mbar_init(&q8_full[1], 128);
     fence_mbar_init();
     tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmKwin); tma_prefetch_desc(&tmVwin);
     tma_prefetch_desc(&tmKpool); tma_prefetch_desc(&tmVpool);
@@ -268,7 +285,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           mbar_arrive_expect_tx(full, npg * PAGE_BYTES);
           for (int pg = 0; pg < npg; ++pg) {
             const int y = (page[pg] * p.n_kv_heads + kvh) * kPage;
-            for (int h = 0; h < NH; ++h)
+            for (int h = 0; h < NHKV; ++h)
               tma_load_2d(dst + h * 16384 + pg * 8192, isV ? &tmVpool : &tmKpool, full, h * 64, y);
           }
         }
@@ -310,13 +327,13 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         if (q_uses > 0 && !warp_wait(q_empty, (q_uses - 1) & 1, abortf, LIM)) { ok = false; break; }
         ++q_uses;
         if (leader) {
-          mbar_arrive_expect_tx(q_full, ((g.nA > 0) + (g.nB > 0)) * TILE_BYTES);
+          mbar_arrive_expect_tx(q_full, ((g.nA > 0) + (g.nB > 0)) * Q_TILE_BYTES);
           if (g.nA > 0)
             for (int h = 0; h < NH; ++h)
               tma_load_3d(sQ + h * 16384, &tmQ, q_full, h * 64, g.kvhA * p.group, g.rowA);
           if (g.nB > 0)
             for (int h = 0; h < NH; ++h)
-              tma_load_3d(sQ + TILE_BYTES + h * 16384, &tmQ, q_full, h * 64, g.kvhB * p.group, g.rowB);
+              tma_load_3d(sQ + Q_TILE_BYTES + h * 16384, &tmQ, q_full, h * 64, g.kvhB * p.group, g.rowB);
         }
         __syncwarp();
       }
@@ -339,43 +356,52 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   } else if (warp == 1) {
     // ---------------------------------------------------------- MMA issuer
     const bool leader = elect_one();
-    int q_cnt = 0, cntPA = 0, cntPB = 0;
+    int q_cnt = 0, q8A = 0, q8B = 0, cntPA = 0, cntPB = 0;
     bool ok = true;
     // All descriptors are built once; a k-step only adds a constant to the
     // address field (low word, no carry: shared-memory addresses fit the
     // 14-bit field).
-    const uint32_t idesc_pv = umma_idesc_bf16(128, D, 0, 1);
-    const uint32_t idesc_qk_full = umma_idesc_bf16(128, kTileN, 0, 0);
-    const uint64_t dQ0 = smem_desc_sw128(smem_u32(sQ), 16, 1024);
+    const uint32_t idesc_pv = F8 ? umma_idesc_e4m3(128, D, 0, 1) : umma_idesc_bf16(128, D, 0, 1);
+    const uint32_t idesc_qk_full = F8 ? umma_idesc_e4m3(128, kTileN, 0, 0) : umma_idesc_bf16(128, kTileN, 0, 0);
+    constexpr int QOP_BYTES = F8 ? 16384 : Q_TILE_BYTES;       // the Q tile the MMAs read
+    const uint64_t dQ0 = smem_desc_sw128(smem_u32(F8 ? sQ8 : sQ), 16, 1024);
     const uint64_t dK0 = smem_desc_sw128(smem_u32(sK), 16, 1024);
     const uint64_t dV0 = smem_desc_sw128(smem_u32(sV), 16384, 1024);
     // S_X = Q_X K^T over `ncols` keys of K stage `st`; X is 0 (tile A) or 1 (tile B)
     auto issue_qk = [&](const int X, int st, int ncols) {
-      const uint32_t idesc = ncols == kTileN ? idesc_qk_full : umma_idesc_bf16(128, ncols, 0, 0);
-      const uint64_t qa = dQ0 + (uint32_t)((X * TILE_BYTES) >> 4), kb = dK0 + (uint32_t)((st * TILE_BYTES) >> 4);
+      const uint32_t idesc = ncols == kTileN ? idesc_qk_full
+                             : (F8 ? umma_idesc_e4m3(128, ncols, 0, 0) : umma_idesc_bf16(128, ncols, 0, 0));
+      const uint64_t qa = dQ0 + (uint32_t)((X * QOP_BYTES) >> 4), kb = dK0 + (uint32_t)((st * TILE_BYTES) >> 4);
       const uint32_t d = tmem + X * 128;
       if (leader) {
 #pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
+        for (int ks = 0; ks < KSTEPS; ++ks) {          // 32 bytes of the 128-byte row per step
           const uint32_t off = ((ks >> 2) * 16384 + (ks & 3) * 32) >> 4;
-          umma_ss(d, qa + off, kb + off, idesc, ks > 0 ? 1u : 0u);
+          if (F8) umma_ss_f8(d, qa + off, kb + off, idesc, ks > 0 ? 1u : 0u);
+          else umma_ss(d, qa + off, kb + off, idesc, ks > 0 ? 1u : 0u);
         }
         umma_commit(&s_full[X]);
       }
       __syncwarp();
     };
-    // O_X (+)= P_X V over k-steps [ks0, ks1) of V stage `st`; P_X is read from TMEM
+    // O_X (+)= P_X V over k-steps [ks0, ks1) of V stage `st`; P_X is read from TMEM.  A step
+    // is 16 keys (bf16) or 32 keys (E4M3): 8 TMEM columns of P and 2 KB / 4 KB of V rows.
+    constexpr int PV_STEPS = F8 ? 4 : 8, PV_STEP_BYTES = F8 ? 4096 : 2048;
     auto issue_pv = [&](const int X, int st, int ks0, int ks1, bool acc) {
       const uint64_t vb = dV0 + (uint32_t)((st * TILE_BYTES) >> 4);
       const uint32_t d = tmem + 256 + X * 128, a = tmem + X * 128;
       if (leader) {
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          if (ks >= ks0 && ks < ks1)
-            umma_ts(d, a + ks * 8, vb + (uint32_t)((ks * 2048) >> 4), idesc_pv, (acc || ks > 0) ? 1u : 0u);
+        for (int ks = 0; ks < PV_STEPS; ++ks)
+          if (ks >= ks0 && ks < ks1) {
+            if (F8) umma_ts_f8(d, a + ks * 8, vb + (uint32_t)((ks * PV_STEP_BYTES) >> 4), idesc_pv, (acc || ks > 0) ? 1u : 0u);
+            else umma_ts(d, a + ks * 8, vb + (uint32_t)((ks * PV_STEP_BYTES) >> 4), idesc_pv, (acc || ks > 0) ? 1u : 0u);
+          }
       }
       __syncwarp();
     };
+    // k-steps of P V that cover the first `lim` keys of a tile
+    auto pv_steps = [&](int lim) { return F8 ? (lim + 31) >> 5 : round16(lim) >> 4; };
     auto commit = [&](uint64_t* bar) { if (leader) umma_commit(bar); __syncwarp(); };
     // fills consumed from each K / V stage (see the producer)
     int kuse0 = 0, kuse1 = 0, vuse0 = 0, vuse1 = 0, rr_k = 0, rr_v = 0;
@@ -398,7 +424,12 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       ItemU g;
       if (!load_item_uniform(p, idx, g)) continue;
       const int nA = g.nA, nB = g.nB, n = g.n;
-      if (!warp_wait(q_full, q_cnt & 1, abortf, LIM)) { ok = false; break; }
+      if (F8) {     // the tiles in E4M3, written by the softmax warps
+        if (nA > 0 && !warp_wait(&q8_full[0], q8A & 1, abortf, LIM)) { ok = false; break; }
+        if (nB > 0 && !warp_wait(&q8_full[1], q8B & 1, abortf, LIM)) { ok = false; break; }
+        q8A += nA > 0; q8B += nB > 0;
+        fence_proxy_async_smem();
+      } else if (!warp_wait(q_full, q_cnt & 1, abortf, LIM)) { ok = false; break; }
       ++q_cnt;
       if (!g.dual()) {
         // ---- tiles A and B share every K/V tile
@@ -418,7 +449,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           if (j + 1 < n) { ++rr_k; if (!wait_k(st1)) { ok = false; break; } }
           // tile A: O_A += P_A(j) V(j), then S_A(j+1) so that softmax A can go on
           if (j < nA) {
-            const int nks = round16(g.limit(j, g.winA, p.resident)) >> 4;
+            const int nks = pv_steps(g.limit(j, g.winA, p.resident));
             if (!warp_wait(&p_full[0], cntPA & 1, abortf, LIM)) { ok = false; break; }
             ++cntPA;
             tc_fence_after();
@@ -430,7 +461,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           }
           // tile B
           if (j < nB) {
-            const int nks = round16(g.limit(j, g.winB, p.resident)) >> 4;
+            const int nks = pv_steps(g.limit(j, g.winB, p.resident));
             if (!warp_wait(&p_full[1], cntPB & 1, abortf, LIM)) { ok = false; break; }
             ++cntPB;
             tc_fence_after();
@@ -477,7 +508,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           if (X) { ++jB; ++cntPB; } else { ++jA; ++cntPA; }
           if (!wait_v(X)) { ok = false; break; }
           tc_fence_after();
-          issue_pv(X, X, 0, round16(g.limit(j, g.winA, p.resident)) >> 4, j > 0);
+          issue_pv(X, X, 0, pv_steps(g.limit(j, g.winA, p.resident)), j > 0);
           commit(&v_empty[X]);
           if (j + 1 < n) {
             // this stream's next K tile could only be requested when its last Q K^T had
@@ -508,8 +539,10 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
     const uint32_t tS = tmem + lane_base + X * 128;
     const uint32_t tO = tmem + lane_base + 256 + X * 128;
-    const float sl2 = p.scale_log2;
-    int cntS = 0, cntO = 0;
+    float sl2 = p.scale_log2;          // F8: per item and row (K scale of the KV head, Q scale of the row)
+    float out_scale = 1.0f;            // F8: V scale of the KV head
+    constexpr float kShift = F8 ? kF8PShift : 0.f;
+    int cntS = 0, cntO = 0, qcnt = 0;
     bool ok = true;
     for (int k = 0; ok; ++k) {
       if (!warp_wait(&item_full[k & 1], (k >> 1) & 1, abortf, LIM)) { ok = false; break; }
@@ -519,9 +552,49 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       if (idx < 0) break;
       ItemGeom g;
       if (!load_item(p, idx, g)) continue;
+      const int q_par = qcnt & 1;        // phase of q_full that carries this item's Q tiles
+      ++qcnt;
       const int nMine = X == 0 ? g.nA : g.nB;
       if (nMine == 0) continue;
       const int winX = X == 0 ? g.un.winA : g.un.winB;
+      if constexpr (F8) {
+        // This thread's Q row, bf16 -> E4M3 with the power of two that brings its largest
+        // magnitude into [128, 256) (exact), into the tile the MMAs read.  The 128-byte swizzle
+        // puts 16-byte piece c of row r at piece c ^ (r & 7) of its 128-byte line.
+        if (!warp_wait(q_full, q_par, abortf, LIM)) { ok = false; break; }
+        const uint8_t* src = sQ + X * Q_TILE_BYTES + (row >> 3) * 1024 + (row & 7) * 128;
+        uint4 qv[16];
+#pragma unroll
+        for (int c = 0; c < 16; ++c)
+          qv[c] = *reinterpret_cast<const uint4*>(src + (c >> 3) * 16384 + (((c & 7) ^ (row & 7)) << 4));
+        uint32_t am = 0;                 // largest |x| as bf16 bits (sign cleared: integer order = magnitude order)
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          const uint32_t w[4] = {qv[c].x, qv[c].y, qv[c].z, qv[c].w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) am = max(am, max(w[i] & 0x7fffu, (w[i] >> 16) & 0x7fffu));
+        }
+        int kq = 134 - (int)(am >> 7);   // biased exponent of the bf16 -> 2^kq * amax in [128, 256)
+        kq = am < 0x80u ? 0 : min(max(kq, -100), 100);      // zero / subnormal rows: no scaling
+        const float f = __int_as_float((kq + 127) << 23);
+        uint8_t* dst = sQ8 + X * 16384 + (row >> 3) * 1024 + (row & 7) * 128;
+#pragma unroll
+        for (int c8 = 0; c8 < 8; ++c8) {
+          const uint4 a = qv[2 * c8], b = qv[2 * c8 + 1];
+          const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+          uint32_t o[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            o[i] = pack_e4m3x4(__uint_as_float(w[2 * i] << 16) * f, __uint_as_float(w[2 * i] & 0xffff0000u) * f,
+                               __uint_as_float(w[2 * i + 1] << 16) * f, __uint_as_float(w[2 * i + 1] & 0xffff0000u) * f);
+          *reinterpret_cast<uint4*>(dst + ((c8 ^ (row & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+        fence_proxy_async_smem();
+        mbar_arrive(&q8_full[X]);
+        const int kvh = X == 0 ? g.kvhA : g.kvhB;
+        sl2 = p.scale_log2 * __ldg(&p.k_scale[kvh]) * __int_as_float((127 - kq) << 23);
+        out_scale = __ldg(&p.v_scale[kvh]);
+      }
       float m_ref = -INFINITY, l = 0.f;
       for (int j = 0; j < nMine; ++j) {
         if (!warp_wait(&s_full[X], cntS & 1, abortf, LIM)) { ok = false; break; }
@@ -557,11 +630,11 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                            64 + i + 8 + t < limit ? __uint_as_float(sb[i + 8 + t]) : -INFINITY);
           m_ref = fmaxf(fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3])), fmaxf(fmaxf(m8[4], m8[5]), fmaxf(m8[6], m8[7])));
         }
-        uint32_t pk[64];                       // P of this tile, packed bf16 pairs
+        uint32_t pk[F8 ? 32 : 64];             // P of this tile: packed bf16 pairs, or E4M3 four to a word
         float tile_sum = 0.f;
 #pragma unroll 1
         for (int attempt = 0; attempt < 2; ++attempt) {
-          const float mb = m_ref * sl2;
+          const float mb = m_ref * sl2 - kShift;
           float2 acc2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
           float xm4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
           const float2 sl2v = make_float2(sl2, sl2), nmb = make_float2(-mb, -mb);
@@ -573,6 +646,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             tmem_ld_wait();
             if (c < 3) tmem_ld32(tS + 32 * (c + 1), sc[(c + 1) & 1]);   // next chunk in flight
             if (limit >= 32 * c + 32) {
+              float2 prev = make_float2(0.f, 0.f);
 #pragma unroll
               for (int i = 0; i < 32; i += 2) {
                 const float2 x = __ffma2_rn(make_float2(__uint_as_float(sr[i]), __uint_as_float(sr[i + 1])), sl2v, nmb);
@@ -581,9 +655,15 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 if (((i >> 1) & 3) < kPolyOf4) pv = exp2_poly2(x);
                 else pv = make_float2(ex2_approx(x.x), ex2_approx(x.y));
                 acc2[(i >> 1) & 1] = __fadd2_rn(acc2[(i >> 1) & 1], pv);
-                pk[16 * c + (i >> 1)] = pack_bf16x2(pv.x, pv.y);
+                if constexpr (F8) {
+                  if (i & 2) pk[8 * c + (i >> 2)] = pack_e4m3x4(prev.x, prev.y, pv.x, pv.y);
+                  prev = pv;
+                } else {
+                  pk[16 * c + (i >> 1)] = pack_bf16x2(pv.x, pv.y);
+                }
               }
             } else {
+              float2 prev = make_float2(0.f, 0.f);
 #pragma unroll
               for (int i = 0; i < 32; i += 2) {
                 const bool v0 = 32 * c + i < limit, v1 = 32 * c + i + 1 < limit;
@@ -592,7 +672,12 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 if (v1) xm4[1] = fmaxf(xm4[1], x1);
                 const float p0 = v0 ? ex2_approx(x0) : 0.f, p1 = v1 ? ex2_approx(x1) : 0.f;
                 acc2[0].x += p0 + p1;
-                pk[16 * c + (i >> 1)] = pack_bf16x2(p0, p1);
+                if constexpr (F8) {
+                  if (i & 2) pk[8 * c + (i >> 2)] = pack_e4m3x4(prev.x, prev.y, p0, p1);
+                  prev = make_float2(p0, p1);
+                } else {
+                  pk[16 * c + (i >> 1)] = pack_bf16x2(p0, p1);
+                }
               }
             }
           }
@@ -602,8 +687,8 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           if (!__any_sync(0xffffffffu, grow)) break;
           // rare: re-base this row's reference, rescale what has been accumulated so far
           // (O is quiescent: the commit behind this S also covered the previous P V)
-          const float alpha = grow ? ex2_approx(-xmax) : 1.0f;
-          if (grow) { m_ref += xmax / sl2; l *= alpha; }
+          const float alpha = grow ? ex2_approx(kShift - xmax) : 1.0f;
+          if (grow) { m_ref += (xmax - kShift) / sl2; l *= alpha; }
 #pragma unroll
           for (int c = 0; c < D / 32; ++c) {
             uint32_t o[32];
@@ -616,7 +701,8 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           tmem_st_wait();
         }
         l += tile_sum;
-        tmem_st32(tS, pk); tmem_st32(tS + 32, pk + 32);
+        tmem_st32(tS, pk);
+        if constexpr (!F8) tmem_st32(tS + 32, pk + 32);
         tmem_st_wait();
         tc_fence_before();
         mbar_arrive(&p_full[X]);
@@ -630,7 +716,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         const int grow_ = slot * p.bl + t0 + row / p.group;
         const int head = (X == 0 ? g.kvhA : g.kvhB) * p.group + row % p.group;
         uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)grow_ * p.n_q_heads + head) * D);
-        const float inv = 1.0f / l;
+        const float inv = out_scale / l;
 #pragma unroll
         for (int c = 0; c < D / 32; ++c) {
           uint32_t o[32];
@@ -647,8 +733,8 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         }
       } else {
         const size_t prow = ((size_t)(g.un.part_base + g.chunk) * 2 + X) * kTileM + row;
-        p.part_ml[prow * 2 + 0] = m_ref * sl2;
-        p.part_ml[prow * 2 + 1] = l;
+        p.part_ml[prow * 2 + 0] = m_ref * sl2 - kShift;     // the reference the exponentials were taken against
+        p.part_ml[prow * 2 + 1] = l / out_scale;            // (the merge divides by the sum: the V scale goes in here)
         uint4* dst = reinterpret_cast<uint4*>(p.part_o + prow * D);
 #pragma unroll
         for (int c = 0; c < D / 32; ++c) {
@@ -773,11 +859,14 @@ int ensure_device(fb_ctx* ctx) {
     return set_err(ctx, FB_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
   ctx->encode_fn = fn;
   const int smem64 = kSmem64, smem128 = kSmem128;
-  if (int e = cuda_err(ctx, cudaFuncSetAttribute(wavefront_attn_kernel<64>,
+  if (int e = cuda_err(ctx, cudaFuncSetAttribute(wavefront_attn_kernel<64, false>,
                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, smem64), "smem attr"))
     return e;
-  if (int e = cuda_err(ctx, cudaFuncSetAttribute(wavefront_attn_kernel<128>,
+  if (int e = cuda_err(ctx, cudaFuncSetAttribute(wavefront_attn_kernel<128, false>,
                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, smem128), "smem attr"))
+    return e;
+  if (int e = cuda_err(ctx, cudaFuncSetAttribute(wavefront_attn_kernel<128, true>,
+                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemF8), "smem attr"))
     return e;
   if (int e = lm_head_device_setup(ctx)) return e;
   ctx->device = dev;
@@ -786,14 +875,43 @@ int ensure_device(fb_ctx* ctx) {
 }
 
 static int encode(fb_ctx* ctx, CUtensorMap* m, const void* base, int rank, const cuuint64_t* dims,
-                  const cuuint64_t* strides, const cuuint32_t* box) {
+                  const cuuint64_t* strides, const cuuint32_t* box,
+                  CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16) {
   cuuint32_t es[3] = {1, 1, 1};
   auto fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled>(ctx->encode_fn);
-  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims, strides, box, es,
+  CUresult r = fn(m, dtype, rank, const_cast<void*>(base), dims, strides, box, es,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return set_err(ctx, FB_ERR_CUDA, "cuTensorMapEncodeTiled failed: " + std::to_string((int)r));
   return FB_OK;
+}
+
+static void fill_params(fb_ctx* ctx, AttnParams& p, const int32_t* page_table, void* out, void* ws, int32_t* status) {
+  const fb_config& c = ctx->cfg;
+  uint8_t* w = static_cast<uint8_t*>(ws);
+  p.hdr = reinterpret_cast<SchedHeader*>(w + ctx->ws.header);
+  p.items = reinterpret_cast<const AttnItem*>(w + ctx->ws.items);
+  p.units = reinterpret_cast<const AttnUnit*>(w + ctx->ws.units);
+  p.page_table = page_table;
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.part_ml = reinterpret_cast<float*>(w + ctx->ws.part_ml);
+  p.part_o = reinterpret_cast<float*>(w + ctx->ws.part_o);
+  p.status = status;
+  p.bl = c.block_len; p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.group = ctx->group;
+  p.max_pages_per_req = c.max_pages_per_req; p.num_pages = c.num_pages;
+  p.resident = c.window_in_pages;
+  p.k_scale = nullptr; p.v_scale = nullptr;
+  p.scale_log2 = ctx->sm_scale * kLog2eF;
+  p.wait_cycles = ctx->wait_cycles;
+}
+
+static int encode_q(fb_ctx* ctx, const void* q) {
+  const fb_config& c = ctx->cfg;
+  const cuuint64_t rows = (cuuint64_t)c.max_requests * c.wmax * c.block_len, D = c.head_dim;
+  cuuint64_t dims[3] = {D, (cuuint64_t)c.n_q_heads, rows};
+  cuuint64_t str[2] = {D * 2, (cuuint64_t)c.n_q_heads * D * 2};
+  cuuint32_t box[3] = {64, (cuuint32_t)ctx->group, (cuuint32_t)ctx->tokens_per_tile};
+  return encode(ctx, &ctx->tm_q, q, 3, dims, str, box);
 }
 
 int launch_attn(fb_ctx* ctx, const fb_pack* pk, const void* q, const void* k_win, const void* v_win,
@@ -805,13 +923,8 @@ int launch_attn(fb_ctx* ctx, const fb_pack* pk, const void* q, const void* k_win
   const cuuint64_t rows = (cuuint64_t)c.max_requests * c.wmax * c.block_len;
   const cuuint64_t D = c.head_dim;
   const void* ptrs[5] = {q, k_win, v_win, k_pool, v_pool};
-  if (memcmp(ptrs, ctx->map_ptrs, sizeof(ptrs)) != 0) {
-    {
-      cuuint64_t dims[3] = {D, (cuuint64_t)c.n_q_heads, rows};
-      cuuint64_t str[2] = {D * 2, (cuuint64_t)c.n_q_heads * D * 2};
-      cuuint32_t box[3] = {64, (cuuint32_t)ctx->group, (cuuint32_t)ctx->tokens_per_tile};
-      if (int e = encode(ctx, &ctx->tm_q, q, 3, dims, str, box)) return e;
-    }
+  if (ctx->maps_f8 || memcmp(ptrs, ctx->map_ptrs, sizeof(ptrs)) != 0) {
+    if (int e = encode_q(ctx, q)) return e;
     {
       cuuint64_t dims[3] = {D, (cuuint64_t)c.n_kv_heads, rows};
       cuuint64_t str[2] = {D * 2, (cuuint64_t)c.n_kv_heads * D * 2};
@@ -828,40 +941,58 @@ int launch_attn(fb_ctx* ctx, const fb_pack* pk, const void* q, const void* k_win
       if (int e = encode(ctx, &ctx->tm_vpool, v_pool, 2, dims, str, box)) return e;
     }
     memcpy(ctx->map_ptrs, ptrs, sizeof(ptrs));
+    ctx->maps_f8 = false;
   }
-  uint8_t* w = static_cast<uint8_t*>(ws);
   AttnParams p;
-  p.hdr = reinterpret_cast<SchedHeader*>(w + ctx->ws.header);
-  p.items = reinterpret_cast<const AttnItem*>(w + ctx->ws.items);
-  p.units = reinterpret_cast<const AttnUnit*>(w + ctx->ws.units);
-  p.page_table = page_table;
-  p.out = static_cast<__nv_bfloat16*>(out);
-  p.part_ml = reinterpret_cast<float*>(w + ctx->ws.part_ml);
-  p.part_o = reinterpret_cast<float*>(w + ctx->ws.part_o);
-  p.status = status;
-  p.bl = c.block_len; p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.group = ctx->group;
-  p.max_pages_per_req = c.max_pages_per_req; p.num_pages = c.num_pages;
-  p.resident = c.window_in_pages;
-  p.scale_log2 = ctx->sm_scale * kLog2eF;
-  p.wait_cycles = ctx->wait_cycles;
+  fill_params(ctx, p, page_table, out, ws, status);
   const int grid = ctx->num_sms;
   const int combine_grid = min(ctx->ws.max_units * kCombineSplit, kCombineCtasPerSm * ctx->num_sms);
   if (c.head_dim == 64) {
-    if (int e = cuda_err(ctx, launch_pdl(wavefront_attn_kernel<64>, grid, kAttnThreads, kSmem64, stream, ctx->tm_q,
+    if (int e = cuda_err(ctx, launch_pdl(wavefront_attn_kernel<64, false>, grid, kAttnThreads, kSmem64, stream, ctx->tm_q,
                                          ctx->tm_kwin, ctx->tm_vwin, ctx->tm_kpool, ctx->tm_vpool, p),
                          "wavefront_attn_kernel launch"))
       return e;
     return cuda_err(ctx, launch_pdl(attn_combine_kernel<64>, combine_grid, 256, 0, stream, p),
                     "attn_combine_kernel launch");
-  } else {
-    if (int e = cuda_err(ctx, launch_pdl(wavefront_attn_kernel<128>, grid, kAttnThreads, kSmem128, stream, ctx->tm_q,
-                                         ctx->tm_kwin, ctx->tm_vwin, ctx->tm_kpool, ctx->tm_vpool, p),
-                         "wavefront_attn_kernel launch"))
-      return e;
-    return cuda_err(ctx, launch_pdl(attn_combine_kernel<128>, combine_grid, 256, 0, stream, p),
-                    "attn_combine_kernel launch");
   }
-  return cuda_err(ctx, cudaGetLastError(), "attn_combine_kernel launch");
+  if (int e = cuda_err(ctx, launch_pdl(wavefront_attn_kernel<128, false>, grid, kAttnThreads, kSmem128, stream, ctx->tm_q,
+                                       ctx->tm_kwin, ctx->tm_vwin, ctx->tm_kpool, ctx->tm_vpool, p),
+                       "wavefront_attn_kernel launch"))
+    return e;
+  return cuda_err(ctx, launch_pdl(attn_combine_kernel<128>, combine_grid, 256, 0, stream, p),
+                  "attn_combine_kernel launch");
+}
+
+// Attention over 8-bit pages (window resident in the pages, head_dim 128): the pools are E4M3
+// bytes, one (page, KV head) is a 64 x 128-byte tile = one TMA box.
+int launch_attn_fp8(fb_ctx* ctx, const fb_pack* pk, const void* q, const void* k_pool8, const void* v_pool8,
+                    const float* k_scale, const float* v_scale, const int32_t* page_table, void* out, void* ws,
+                    int32_t* status, cudaStream_t stream) {
+  (void)pk;
+  if (int e = ensure_device(ctx)) return e;
+  const fb_config& c = ctx->cfg;
+  const void* ptrs[5] = {q, nullptr, nullptr, k_pool8, v_pool8};
+  if (!ctx->maps_f8 || memcmp(ptrs, ctx->map_ptrs, sizeof(ptrs)) != 0) {
+    if (int e = encode_q(ctx, q)) return e;
+    cuuint64_t dims[2] = {128, (cuuint64_t)c.num_pages * c.n_kv_heads * kPage};
+    cuuint64_t str[1] = {128};
+    cuuint32_t box[2] = {128, 64};
+    if (int e = encode(ctx, &ctx->tm_kpool, k_pool8, 2, dims, str, box, CU_TENSOR_MAP_DATA_TYPE_UINT8)) return e;
+    if (int e = encode(ctx, &ctx->tm_vpool, v_pool8, 2, dims, str, box, CU_TENSOR_MAP_DATA_TYPE_UINT8)) return e;
+    ctx->tm_kwin = ctx->tm_kpool; ctx->tm_vwin = ctx->tm_vpool;        // never used: every key tile is a paged one
+    memcpy(ctx->map_ptrs, ptrs, sizeof(ptrs));
+    ctx->maps_f8 = true;
+  }
+  AttnParams p;
+  fill_params(ctx, p, page_table, out, ws, status);
+  p.k_scale = k_scale; p.v_scale = v_scale;
+  const int combine_grid = min(ctx->ws.max_units * kCombineSplit, kCombineCtasPerSm * ctx->num_sms);
+  if (int e = cuda_err(ctx, launch_pdl(wavefront_attn_kernel<128, true>, ctx->num_sms, kAttnThreads, (size_t)kSmemF8, stream,
+                                       ctx->tm_q, ctx->tm_kwin, ctx->tm_vwin, ctx->tm_kpool, ctx->tm_vpool, p),
+                       "wavefront_attn_kernel (8-bit pages) launch"))
+    return e;
+  return cuda_err(ctx, launch_pdl(attn_combine_kernel<128>, combine_grid, 256, 0, stream, p),
+                  "attn_combine_kernel launch");
 }
 
 }  // namespace fb

@@ -152,6 +152,7 @@ struct fb_ctx {
   void* encode_fn = nullptr;
   // cached tensor maps (re-encoded when a base pointer changes)
   const void* map_ptrs[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+  bool maps_f8 = false;   // the cached pool maps describe 8-bit pages
   CUtensorMap tm_q, tm_kwin, tm_vwin, tm_kpool, tm_vpool;
 };
 
@@ -195,6 +196,12 @@ int launch_pack(fb_ctx*, const fb_state*, const fb_pack*, void* ws, int32_t* sta
 int launch_attn(fb_ctx*, const fb_pack*, const void* q, const void* k_win, const void* v_win,
                 const void* k_pool, const void* v_pool, const int32_t* page_table, void* out,
                 void* ws, int32_t* status, cudaStream_t);
+int launch_attn_fp8(fb_ctx*, const fb_pack*, const void* q, const void* k_pool8, const void* v_pool8,
+                    const float* k_scale, const float* v_scale, const int32_t* page_table, void* out, void* ws,
+                    int32_t* status, cudaStream_t);
+int launch_scatter_fp8(fb_ctx*, const fb_pack*, const int32_t* page_table, const void* k_new, const void* v_new,
+                       void* k_pool8, void* v_pool8, const float* k_scale, const float* v_scale, float rope_base,
+                       int32_t* status, cudaStream_t);
 int launch_scatter(fb_ctx*, const fb_pack*, const int32_t* page_table, const void* k_new, const void* v_new,
                    void* k_pool, void* v_pool, float rope_base, int32_t* status, cudaStream_t);
 int ensure_device(fb_ctx*);   // device properties, driver entry point for tensor maps, kernel attributes

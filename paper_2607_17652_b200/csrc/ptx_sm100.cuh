@@ -178,6 +178,31 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem,
       : "memory");
 }
 
+// The same two with 8-bit operands (kind::f8f6f4; the formats are in the
+// instruction descriptor): 32 elements of K per instruction.
+__device__ __forceinline__ void umma_ss_f8(uint32_t d_tmem, uint64_t a_desc,
+                                           uint64_t b_desc, uint32_t idesc,
+                                           uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}\n" ::"r"(
+          d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_ts_f8(uint32_t d_tmem, uint32_t a_tmem,
+                                           uint64_t b_desc, uint32_t idesc,
+                                           uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], [%1], %2, %3, p;\n\t}\n" ::"r"(
+          d_tmem),
+      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
 // Shared-memory matrix descriptor for a 128-byte-swizzled operand tile whose
 // rows are 128 B (64 bf16) and whose 8-row groups are 1024 B apart.
 //   K-major  (rows = M or N index, 128 B along K): SBO = 1024, LBO unused.
@@ -205,6 +230,20 @@ __host__ __device__ __forceinline__ uint32_t umma_idesc_bf16(int M, int N,
   d |= 1u << 4;                         // D format: f32
   d |= 1u << 7;                         // A format: bf16
   d |= 1u << 10;                        // B format: bf16
+  d |= (uint32_t)(a_mn & 1) << 15;      // A major
+  d |= (uint32_t)(b_mn & 1) << 16;      // B major
+  d |= (uint32_t)((N >> 3) & 0x3F) << 17;
+  d |= (uint32_t)((M >> 4) & 0x1F) << 24;
+  return d;
+}
+
+// Instruction descriptor, kind::f8f6f4, E4M3 x E4M3 -> fp32 (format code 0 for
+// both operands); an MN-major operand is allowed for 8-bit formats.
+__host__ __device__ __forceinline__ uint32_t umma_idesc_e4m3(int M, int N,
+                                                             int a_mn,
+                                                             int b_mn) {
+  uint32_t d = 0;
+  d |= 1u << 4;                         // D format: f32
   d |= (uint32_t)(a_mn & 1) << 15;      // A major
   d |= (uint32_t)(b_mn & 1) << 16;      // B major
   d |= (uint32_t)((N >> 3) & 0x3F) << 17;
@@ -270,6 +309,18 @@ __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+// four floats -> four E4M3 bytes (round to nearest even, saturating at 448), a in the lowest byte
+__device__ __forceinline__ uint32_t pack_e4m3x4(float a, float b, float c, float d) {
+  uint32_t r;
+  asm("{\n\t.reg .b16 lo, hi;\n\t"
+      "cvt.rn.satfinite.e4m3x2.f32 lo, %2, %1;\n\t"
+      "cvt.rn.satfinite.e4m3x2.f32 hi, %4, %3;\n\t"
+      "mov.b32 %0, {lo, hi};\n\t}\n"
+      : "=r"(r)
+      : "f"(a), "f"(b), "f"(c), "f"(d));
+  return r;
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {

@@ -10,6 +10,8 @@
 // position), so a thread moves 16-byte pieces: with the rotary embedding a
 // thread owns the two pieces that hold elements i and i + d/2 of eight pairs,
 // and the rotation angles come from a per-slot table in shared memory.
+#include <cuda_fp8.h>
+
 #include "fb_common.cuh"
 
 namespace fb {
@@ -24,6 +26,7 @@ struct ScatterParams {
   int32_t* status;
   int32_t bl, n_kv_heads, head_dim, max_pages_per_req, num_pages;
   float rope_base;
+  const float *k_scale, *v_scale;   // 8-bit pages: [n_kv_heads]
 };
 
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
@@ -33,6 +36,22 @@ __device__ __forceinline__ uint32_t to_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// stored byte of x under `scale`: the binary32 quotient, rounded to nearest even onto the E4M3
+// grid, saturating at +-448
+__device__ __forceinline__ uint32_t e4m3x4(float a, float b, float c, float d, float scale) {
+  const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(__fdiv_rn(a, scale), __fdiv_rn(b, scale)), __NV_SATFINITE, __NV_E4M3);
+  const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(__fdiv_rn(c, scale), __fdiv_rn(d, scale)), __NV_SATFINITE, __NV_E4M3);
+  return lo | (hi << 16);
+}
+// eight bf16 (one 16-byte piece) -> eight E4M3 bytes
+__device__ __forceinline__ uint2 quant8(const uint4 v, float scale) {
+  return make_uint2(e4m3x4(bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y), scale),
+                    e4m3x4(bf16_lo(v.z), bf16_hi(v.z), bf16_lo(v.w), bf16_hi(v.w), scale));
+}
+
+// F8: the pools hold E4M3 bytes (8-byte pieces instead of 16-byte ones), each value divided by
+// the scale of its KV head before it is rounded.
+template <bool F8>
 __global__ void __launch_bounds__(kScatterThreads) scatter_window_kv_kernel(const ScatterParams p) {
   const int slot = blockIdx.x;
   if (slot >= *p.n_live) return;
@@ -80,9 +99,18 @@ __global__ void __launch_bounds__(kScatterThreads) scatter_window_kv_kernel(cons
     if (page < 0 || page >= p.num_pages) { atomicOr(p.status, FB_ST_BAD_PAGE); continue; }
     const size_t src = (size_t)(slot * p.bl + t) * vpt + h * vph + v;
     const size_t dst = (((size_t)page * p.n_kv_heads + h) * kPage + pos % kPage) * vph + v;
+    [[maybe_unused]] uint2* k8 = reinterpret_cast<uint2*>(p.k_pool);
+    [[maybe_unused]] uint2* v8 = reinterpret_cast<uint2*>(p.v_pool);
+    [[maybe_unused]] float ksc = 1.f, vsc = 1.f;
+    if constexpr (F8) { ksc = p.k_scale[h]; vsc = p.v_scale[h]; }
     if (!rope) {
-      p.k_pool[dst] = p.k_new[src];
-      p.v_pool[dst] = p.v_new[src];
+      if constexpr (F8) {
+        k8[dst] = quant8(p.k_new[src], ksc);
+        v8[dst] = quant8(p.v_new[src], vsc);
+      } else {
+        p.k_pool[dst] = p.k_new[src];
+        p.v_pool[dst] = p.v_new[src];
+      }
       continue;
     }
     const uint4 a = p.k_new[src], b = p.k_new[src + vph / 2];      // elements i0.. and i0 + d/2..
@@ -93,17 +121,31 @@ __global__ void __launch_bounds__(kScatterThreads) scatter_window_kv_kernel(cons
       c[k] = a2.x; s[k] = a2.y;
     }
     const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
-    uint32_t lo[4], hi[4];
+    if constexpr (F8) {
+      float lo[8], hi[8];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const float x0 = bf16_lo(aw[k]), x1 = bf16_hi(aw[k]), y0 = bf16_lo(bw[k]), y1 = bf16_hi(bw[k]);
-      lo[k] = to_bf16x2(x0 * c[2 * k] - y0 * s[2 * k], x1 * c[2 * k + 1] - y1 * s[2 * k + 1]);
-      hi[k] = to_bf16x2(y0 * c[2 * k] + x0 * s[2 * k], y1 * c[2 * k + 1] + x1 * s[2 * k + 1]);
+      for (int k = 0; k < 4; ++k) {
+        const float x0 = bf16_lo(aw[k]), x1 = bf16_hi(aw[k]), y0 = bf16_lo(bw[k]), y1 = bf16_hi(bw[k]);
+        lo[2 * k] = x0 * c[2 * k] - y0 * s[2 * k]; lo[2 * k + 1] = x1 * c[2 * k + 1] - y1 * s[2 * k + 1];
+        hi[2 * k] = y0 * c[2 * k] + x0 * s[2 * k]; hi[2 * k + 1] = y1 * c[2 * k + 1] + x1 * s[2 * k + 1];
+      }
+      k8[dst] = make_uint2(e4m3x4(lo[0], lo[1], lo[2], lo[3], ksc), e4m3x4(lo[4], lo[5], lo[6], lo[7], ksc));
+      k8[dst + vph / 2] = make_uint2(e4m3x4(hi[0], hi[1], hi[2], hi[3], ksc), e4m3x4(hi[4], hi[5], hi[6], hi[7], ksc));
+      v8[dst] = quant8(p.v_new[src], vsc);
+      v8[dst + vph / 2] = quant8(p.v_new[src + vph / 2], vsc);
+    } else {
+      uint32_t lo[4], hi[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float x0 = bf16_lo(aw[k]), x1 = bf16_hi(aw[k]), y0 = bf16_lo(bw[k]), y1 = bf16_hi(bw[k]);
+        lo[k] = to_bf16x2(x0 * c[2 * k] - y0 * s[2 * k], x1 * c[2 * k + 1] - y1 * s[2 * k + 1]);
+        hi[k] = to_bf16x2(y0 * c[2 * k] + x0 * s[2 * k], y1 * c[2 * k + 1] + x1 * s[2 * k + 1]);
+      }
+      p.k_pool[dst] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+      p.k_pool[dst + vph / 2] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+      p.v_pool[dst] = p.v_new[src];
+      p.v_pool[dst + vph / 2] = p.v_new[src + vph / 2];
     }
-    p.k_pool[dst] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-    p.k_pool[dst + vph / 2] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-    p.v_pool[dst] = p.v_new[src];
-    p.v_pool[dst + vph / 2] = p.v_new[src + vph / 2];
   }
   }
 }
@@ -121,9 +163,29 @@ int launch_scatter(fb_ctx* ctx, const fb_pack* pk, const int32_t* page_table, co
   p.bl = c.block_len; p.n_kv_heads = c.n_kv_heads; p.head_dim = c.head_dim;
   p.max_pages_per_req = c.max_pages_per_req; p.num_pages = c.num_pages;
   p.rope_base = rope_base;
+  p.k_scale = p.v_scale = nullptr;
   const dim3 grid(c.max_requests * c.wmax, c.n_kv_heads >= 4 ? 4 : 1);
-  scatter_window_kv_kernel<<<grid, kScatterThreads, 0, stream>>>(p);
+  scatter_window_kv_kernel<false><<<grid, kScatterThreads, 0, stream>>>(p);
   return cuda_err(ctx, cudaGetLastError(), "scatter_window_kv_kernel launch");
+}
+
+int launch_scatter_fp8(fb_ctx* ctx, const fb_pack* pk, const int32_t* page_table, const void* k_new,
+                       const void* v_new, void* k_pool8, void* v_pool8, const float* k_scale, const float* v_scale,
+                       float rope_base, int32_t* status, cudaStream_t stream) {
+  const fb_config& c = ctx->cfg;
+  ScatterParams p;
+  p.n_live = pk->n_live; p.slot_req = pk->slot_req; p.slot_pos0 = pk->slot_pos0;
+  p.page_table = page_table;
+  p.k_new = static_cast<const uint4*>(k_new); p.v_new = static_cast<const uint4*>(v_new);
+  p.k_pool = static_cast<uint4*>(k_pool8); p.v_pool = static_cast<uint4*>(v_pool8);
+  p.status = status;
+  p.bl = c.block_len; p.n_kv_heads = c.n_kv_heads; p.head_dim = c.head_dim;
+  p.max_pages_per_req = c.max_pages_per_req; p.num_pages = c.num_pages;
+  p.rope_base = rope_base;
+  p.k_scale = k_scale; p.v_scale = v_scale;
+  const dim3 grid(c.max_requests * c.wmax, c.n_kv_heads >= 4 ? 4 : 1);
+  scatter_window_kv_kernel<true><<<grid, kScatterThreads, 0, stream>>>(p);
+  return cuda_err(ctx, cudaGetLastError(), "scatter_window_kv_kernel (8-bit pages) launch");
 }
 
 // fb_embed_gather: x[i, :] = table[qtok[i], :] for live rows; one warp per row, 16-byte pieces.
