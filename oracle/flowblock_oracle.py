@@ -261,6 +261,26 @@ def wavefront_attn(cfg: Config, pk: Pack, q, k_win, v_win, k_pool, v_pool,
     return out
 
 
+def wavefront_attn_weight_norms(cfg: Config, pk: Pack, q, k_win, k_pool, page_table) -> np.ndarray:
+    """sum_i w_i^2 of the softmax weights of every live query row and head,
+    [S*bl, Hq] (1/n for n equal weights, 1 when one key takes everything).  Not
+    part of the method: the tests of approximate kernels scale their
+    element-wise error bounds with it (independent per-weight errors of relative
+    size eps leave eps * sqrt(sum w_i^2) * rms(v) in an output element)."""
+    b, Hq, Hkv = cfg.block_len, cfg.n_q_heads, cfg.n_kv_heads
+    G = Hq // Hkv
+    sc = _scale(cfg)
+    out = np.zeros((cfg.max_slots * b, Hq), np.float64)
+    for slot in range(pk.n_live):
+        K = visible_keys(cfg, pk, slot, k_win, k_pool, page_table)
+        for h in range(Hq):
+            sco = sc * (q[slot * b:(slot + 1) * b, h, :] @ K[:, h // G, :].T)
+            w = np.exp(sco - sco.max(axis=1, keepdims=True))
+            w = w / w.sum(axis=1, keepdims=True)
+            out[slot * b:(slot + 1) * b, h] = (w * w).sum(axis=1)
+    return out
+
+
 def dense_mask_attn_bruteforce(cfg: Config, st_prefix_len, st_wlive, q_req,
                                k_phys, v_phys, C: int) -> np.ndarray:
     """Literal Eq. 5 in the paper's own physical layout, for tiny sizes.

@@ -145,3 +145,19 @@ def test_synthetic_fp8_pools_are_plain_bytes_with_finite_values():
     assert np.isfinite(O.e4m3_decode(k8.numpy())).all() and np.isfinite(O.e4m3_decode(v8.numpy())).all()
     assert ks.dtype == torch.float32 and len(ks) == wl.n_kv_heads and (vs > 0).all()
     assert len(np.unique(k8.numpy())) > 100                    # the codes in use span the format
+
+
+def test_weight_norms_closed_forms():
+    """sum w^2 is 1/n for the n equal weights of a zero query and 1 when one key dominates."""
+    wl, stc, cfg, st, pk, q, kw, vw, kp, vp = _case(seed=4)
+    O.scatter_window_kv(cfg, pk, kw, vw, kp, vp, st.page_table)
+    n2 = O.wavefront_attn_weight_norms(cfg, pk, np.zeros_like(q), None, kp, st.page_table)
+    b = wl.block_len
+    for slot in range(pk.n_live):
+        np.testing.assert_allclose(n2[slot * b:(slot + 1) * b], 1.0 / int(pk.slot_kv_len[slot]), rtol=1e-12)
+    assert not n2[pk.n_live * b:].any()
+    kp2 = kp.copy()
+    r = int(pk.slot_req[0])
+    kp2[int(st.page_table[r, 0]), :, 0, :] = 50.0                 # position 0 of request r
+    n2 = O.wavefront_attn_weight_norms(cfg, pk, np.ones_like(q), None, kp2, st.page_table)
+    assert int(st.prefix_len[r]) > 0 and np.abs(n2[:b] - 1.0).max() < 1e-9
