@@ -18,10 +18,11 @@ s = scale * sum_d q_d k_d with independent errors on the q_d, another
 2.65e-2 * rms(q) * rms(k) = 2.65e-2 for N(0,1) queries and keys: 3.75e-2 per
 weight in all, independent across keys.  With values independent of the
 weights the output row inherits the same relative error, so rel-L2 is expected
-at 3.75e-2; the bound is 1.5 x that.  Element-wise the error has standard
-deviation 3.75e-2 * sqrt(sum w_i^2), at most about 0.3 * 3.75e-2 for the
-shortest key sets here; over 10^5..10^6 elements the largest is ~5.5 sigma:
-bound 8e-2.  Cases in which both roundings are exact (zero queries; one key
+at 3.75e-2; the bound is 1.5 x that.  Element-wise the error of a row has
+standard deviation 3.75e-2 * sqrt(sum w_i^2) * rms(v) (rms(v) = 1 here); the
+oracle gives sum w_i^2 per row, and with up to 10^6 elements compared the
+bound is 6 of those standard deviations plus the 1e-2 of the bf16 output.
+Cases in which both roundings are exact (zero queries; one key
 that dominates) must meet the bf16 path's tolerance instead, which pins the key
 set, the paging, the scales and the normalisation tightly."""
 import dataclasses
@@ -37,7 +38,8 @@ from tests import harness as H
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
-F8_REL_L2, F8_MAX_ABS = 1.5 * 3.75e-2, 8e-2
+F8_EPS_W = 3.75e-2
+F8_REL_L2 = 1.5 * F8_EPS_W
 EXACT_MAX_ABS, EXACT_REL_L2 = 1e-2, 5e-3
 
 SHAPES = {
@@ -93,15 +95,28 @@ def _run(c, q=None, k8=None, v8=None, scatter=True):
                                c["stc"].page_table)
     rows = H.live_rows(c["opk"], c["wl"].block_len)
     assert bool((sb.out[len(rows):].float() == 7.0).all())           # rows of padding slots are not written
+    c["pools_f64"] = (O.e4m3_decode(ok8) * c["ks"].numpy()[None, :, None, None], H.f64(q))
     return sb.out, ref, rows
+
+
+def _within_f8_bound(c, out, ref, rows):
+    """rel-L2 of all live rows and the row-scaled element-wise bound of the module docstring."""
+    kd, q64 = c["pools_f64"]
+    n2 = O.wavefront_attn_weight_norms(c["ocfg"], c["opk"], q64, None, kd, c["stc"].page_table)
+    g = out.float().cpu().numpy().astype(np.float64)[rows]
+    err = np.abs(g - ref[rows])
+    allowed = 6.0 * F8_EPS_W * np.sqrt(n2[rows])[:, :, None] + 1e-2
+    rel = float(np.linalg.norm(g - ref[rows]) / np.linalg.norm(ref[rows]))
+    worst = float((err / allowed).max())
+    return rel, worst
 
 
 @pytest.mark.parametrize("name", list(SHAPES))
 def test_scatter_bytes_bit_exact_and_attention_within_the_derived_bound(name):
     c = _setup(SHAPES[name])
     out, ref, rows = _run(c)
-    max_abs, rel = H.attn_errors(out, ref, rows)
-    assert rel <= F8_REL_L2 and max_abs <= F8_MAX_ABS, (max_abs, rel)
+    rel, worst = _within_f8_bound(c, out, ref, rows)
+    assert rel <= F8_REL_L2 and worst <= 1.0, (rel, worst)
     assert rel >= 2e-3, "an error this small means the 8-bit products did not run"
 
 
@@ -109,8 +124,8 @@ def test_scatter_bytes_bit_exact_and_attention_within_the_derived_bound(name):
 def test_split_kv_changes_nothing_beyond_rounding(target):
     c = _setup(SHAPES["long"], tuning=dict(attn_target_items=target))
     out, ref, rows = _run(c)
-    max_abs, rel = H.attn_errors(out, ref, rows)
-    assert rel <= F8_REL_L2 and max_abs <= F8_MAX_ABS, (target, max_abs, rel)
+    rel, worst = _within_f8_bound(c, out, ref, rows)
+    assert rel <= F8_REL_L2 and worst <= 1.0, (target, rel, worst)
     hdr = c["sb"].ws[:64].cpu().numpy().view(np.int32)
     assert (hdr[3] > 0) == (target > 1)
 
