@@ -378,3 +378,50 @@ def test_lm_head_fused_row_pass_full_vocabulary_sampled_rows():
     am, cf = sb.argmax.cpu().numpy(), sb.conf.cpu().numpy()
     assert ((am[:live] >= 0) & (am[:live] < wl.vocab)).all() and ((cf[:live] > 0) & (cf[:live] <= 1)).all()
     assert (am[live:] == -1).all() and not cf[live:].any()
+
+
+def test_fp8_pages_attention_sampled_requests_at_the_bench_size():
+    """The 8-bit-page attention at the benchmark's size (64 requests, prefixes
+    1K-8K): scatter (quantiser) + attention, six sampled requests against the
+    oracle with the tolerance tests/test_gpu_fp8.py derives (rel-L2 at most 1.5 x
+    3.75e-2; element-wise 6 standard deviations of the row's rounding error
+    plus the bf16 output's 1e-2)."""
+    wl = synth.WORKLOADS[2]
+    stc = synth.make_structure(wl)
+    tokens = synth.make_tokens(stc)
+    q, kw, vw, _, _ = synth.make_attn_inputs(stc)
+    k8, v8, ks, vs = synth.make_fp8_kv(stc)
+    ctx = B.Context(**synth.config_dict(stc, window_in_pages=1))
+    st = B.DeviceState.from_numpy(DEV, stc.active, stc.prefix_len, stc.L, stc.R, tokens,
+                                  np.zeros((wl.n_requests, wl.wmax), np.uint8), stc.page_table)
+    pk = B.PackBuffers.alloc(ctx, DEV)
+    sb = B.StepBuffers(ctx, DEV)
+    dk8, dv8, dks, dvs = k8.to(DEV), v8.to(DEV), ks.to(DEV), vs.to(DEV)
+    sb.out.fill_(7.0)
+    B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+    B.fb_scatter_window_kv_fp8(ctx, pk, st.page_table, kw.to(DEV), vw.to(DEV), dk8, dv8, dks, dvs, sb.status)
+    B.fb_wavefront_attn_fp8(ctx, pk, q.to(DEV), dk8, dv8, dks, dvs, st.page_table, sb.out, sb.ws, sb.status)
+    torch.cuda.synchronize()
+    assert int(sb.status.item()) == 0
+    order = np.argsort(stc.prefix_len)
+    keep = sorted({int(order[0]), int(order[-1]), int(np.argmax(stc.R - stc.L)), 5, 23, 41})
+    # the sampled requests as a problem of their own; the 8-bit pools go through the same page remap
+    # as bf16 tensors of code values (sub_problem only moves rows around), then back to bytes
+    as_bf16 = lambda t8: t8.to(torch.float32).to(torch.bfloat16)        # codes 0..255 are exact in bf16
+    sp = H.sub_problem(stc, tokens, (q, kw, vw, as_bf16(k8), as_bf16(v8)), None, keep)
+    opk = O.pack_wavefronts(sp["ocfg"], sp["ost"])
+    ok8, ov8 = sp["k_pool"].astype(np.uint8), sp["v_pool"].astype(np.uint8)
+    O.scatter_window_kv_fp8(sp["ocfg"], opk, sp["k_win"], sp["v_win"], ok8, ov8, ks.numpy(), vs.numpy(),
+                            sp["ost"].page_table)
+    ref = O.wavefront_attn_fp8(sp["ocfg"], opk, sp["q"], ok8, ov8, ks.numpy(), vs.numpy(), sp["ost"].page_table)
+    n = len(sp["rows"])
+    got = sb.out[torch.from_numpy(sp["rows"]).to(DEV)].float().cpu().numpy().astype(np.float64)
+    rel = np.linalg.norm(got - ref[:n]) / np.linalg.norm(ref[:n])
+    kd = O.e4m3_decode(ok8) * ks.numpy()[None, :, None, None]
+    n2 = O.wavefront_attn_weight_norms(sp["ocfg"], opk, sp["q"], None, kd, sp["ost"].page_table)
+    allowed = 6.0 * 3.75e-2 * np.sqrt(n2[:n])[:, :, None] + 1e-2
+    worst = float((np.abs(got - ref[:n]) / allowed).max())
+    assert rel <= 1.5 * 3.75e-2 and worst <= 1.0, (rel, worst)
+    live = synth.n_live_slots(stc) * wl.block_len
+    assert bool(torch.isfinite(sb.out[:live].float()).all())
+    assert bool((sb.out[live:].float() == 7.0).all())
