@@ -95,7 +95,8 @@ __device__ __forceinline__ bool load_item(const AttnParams& p, int idx, ItemGeom
 // round-to-nearest split x = n + f, f in [-0.5, 0.5], cubic minimax fit of 2^f
 // (max relative error 7.5e-5, far below bf16 resolution), then n is added to
 // the exponent field.  Valid for -120 <= x <= 120.
-constexpr int kPolyOf4 = 1;   // pairs out of every 4 that take this path
+constexpr int kPolyOf4 = 1;   // pairs out of every 4 that take this path (bf16 pages)
+constexpr int kPolyOf4F8 = 1;   // the same share with 8-bit pages (0, 2 and 3 of 4 measured slower)
 __device__ __forceinline__ float2 exp2_poly2(float2 x) {
   x.x = fmaxf(x.x, -120.f);
   x.y = fmaxf(x.y, -120.f);
@@ -652,7 +653,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 const float2 x = __ffma2_rn(make_float2(__uint_as_float(sr[i]), __uint_as_float(sr[i + 1])), sl2v, nmb);
                 xm4[(i >> 1) & 3] = max3(xm4[(i >> 1) & 3], x.x, x.y);
                 float2 pv;
-                if (((i >> 1) & 3) < kPolyOf4) pv = exp2_poly2(x);
+                if (((i >> 1) & 3) < (F8 ? kPolyOf4F8 : kPolyOf4)) pv = exp2_poly2(x);
                 else pv = make_float2(ex2_approx(x.x), ex2_approx(x.y));
                 acc2[(i >> 1) & 1] = __fadd2_rn(acc2[(i >> 1) & 1], pv);
                 if constexpr (F8) {
