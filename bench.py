@@ -252,7 +252,7 @@ def run_ours(args):
     seed = synth.BASE_SEED + wl.index + 1000 * rank     # each rank its own batch
     stc, tokens, n_live, z_live, attn = build_inputs(wl, seed)
     stc_init = stc
-    ctx = B.Context(**synth.config_dict(stc))
+    ctx = B.Context(tuning=dict(attn_pair=1) if args.pair else None, **synth.config_dict(stc))
     st = B.DeviceState.from_numpy(dev, stc.active, stc.prefix_len, stc.L, stc.R, tokens,
                                   np.zeros((wl.n_requests, wl.wmax), np.uint8), stc.page_table)
     pk = B.PackBuffers.alloc(ctx, dev)
@@ -359,14 +359,17 @@ def run_ours(args):
             for p0 in range(0, pool.shape[0], 2048):
                 x = torch.randn(pool[p0:p0 + 2048].shape, device=dev, generator=gen8) / sc[None, :, None, None]
                 pool[p0:p0 + 2048] = x.clamp_(-448.0, 448.0).to(torch.float8_e4m3fn).view(torch.uint8)
+        ctx8 = B.Context(kv_fp8=1, **synth.config_dict(stc, window_in_pages=1))
+        pk8 = B.PackBuffers.alloc(ctx8, dev)
+        ws8 = B.alloc_workspace(ctx8, dev)
         ev8 = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n2)]
         for k in range(3 + n2):
-            B.fb_pack_wavefronts(ctx2, st, pk2, ws2, sb.status, stream)
+            B.fb_pack_wavefronts(ctx8, st, pk8, ws8, sb.status, stream)
             e = ev8[k - 3] if k >= 3 else None
             if e: e[0].record(stream)
-            B.fb_scatter_window_kv_fp8(ctx2, pk2, st.page_table, kw, vw, kp8, vp8, ks8, vs8, sb.status, 10000.0, stream)
+            B.fb_scatter_window_kv_fp8(ctx8, pk8, st.page_table, kw, vw, kp8, vp8, ks8, vs8, sb.status, 10000.0, stream)
             if e: e[1].record(stream)
-            B.fb_wavefront_attn_fp8(ctx2, pk2, q, kp8, vp8, ks8, vs8, st.page_table, sb.out, ws2, sb.status, stream)
+            B.fb_wavefront_attn_fp8(ctx8, pk8, q, kp8, vp8, ks8, vs8, st.page_table, sb.out, ws8, sb.status, stream)
             if e: e[2].record(stream)
         barrier()
         s8_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in ev8]))
@@ -378,7 +381,7 @@ def run_ours(args):
         nxt["attn_fp8_pages"] = {"ms": round(a8_ms, 4), "tflops": round(attn_flops(cur) / a8_ms / 1e9, 2),
                                  "algorithmic_bytes": a8_bytes, "scatter_quantise_ms": round(s8_ms, 4),
                                  "speedup_vs_bf16_pages": round(ra_ms / a8_ms, 3)}
-        del ctx2, pk2, ws2, kp8, vp8
+        del ctx2, pk2, ws2, ctx8, pk8, ws8, kp8, vp8
         # next row: the row pass fused into the LM head GEMM (hidden size of a small dLLM; random inputs)
         hidden = 2048
         gen = torch.Generator(device=dev); gen.manual_seed(seed + 77)
@@ -766,6 +769,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-calibrated", action="store_true", help="skip next_rows.step_calibrated")
+    ap.add_argument("--pair", action="store_true",
+                    help="quads of Q tiles on the CTA-pair attention kernel (fb_tuning.attn_pair): the comparison run")
     ap.add_argument("--dry-run-cpu", action="store_true",
                     help="launcher / reduction plumbing only: gloo ranks on CPU, no kernel, placeholder times")
     ap.add_argument("--requests", type=int, default=0,

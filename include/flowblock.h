@@ -126,6 +126,10 @@ typedef struct {
                                 compare) is revealed (action FB_ACT_FORCED,
                                 counted as M2T).  Not in the paper: Eq. 1 is
                                 threshold-only; off by default               */
+  int32_t kv_fp8;            /* 1: the pools are FP8 E4M3 bytes with per-KV-head
+                                scales (fb_scatter_window_kv_fp8,
+                                fb_wavefront_attn_fp8); needs window_in_pages =
+                                1 and head_dim = 128.  0: bf16 pools          */
 } fb_config;
 
 /* Per-request wavefront state (Sec. 3.2: (L_b, R_b), in-order commit
@@ -173,6 +177,14 @@ typedef struct {
                                     split, large = split down to the minimum  */
   int32_t attn_min_chunk_tiles;  /* shortest key range of a split piece, in
                                     128-key tiles (default 4)                 */
+  int32_t attn_pair;             /* 1: four Q tiles of one request and KV head
+                                    at a time run on a pair of CTAs that share
+                                    every K/V tile (tcgen05 cta_group::2; bf16
+                                    pages and head_dim 128 only), the remaining
+                                    tiles on single CTAs.  Off by default: on
+                                    the measured workloads the single-CTA
+                                    kernel alone is faster                     */
+  int32_t reserved;              /* 0                                         */
   int64_t wait_cycles;           /* limit of every bounded device-side wait
                                     (mbarrier, hand-off flags) in SM clock
                                     cycles (default 2e9, about a second); when
@@ -201,9 +213,11 @@ size_t fb_workspace_bytes(const fb_ctx* ctx);
  * fb_pack_wavefronts runs on the device (the paper has no counterpart: the
  * work list is this library's execution plan).  For n <= max_requests decoding
  * requests with HOST arrays h_prefix_len[n] and h_live_blocks[n] (R - L of
- * each) it writes six int32 to h_out: units, work items and split pieces the
- * batch produces, then the capacities max_units, max_items, max_parts that
- * the workspace of this context is sized for.  No CUDA call is made. */
+ * each) it writes twelve int32 to h_out, six per work list (first the list of
+ * the one-CTA kernel, then the list of the CTA-pair kernel): unit records,
+ * work items and split pieces the batch produces, then the capacities
+ * max_units, max_items, max_parts that the workspace of this context is sized
+ * for.  No CUDA call is made. */
 int fb_attn_plan_host(const fb_ctx* ctx, const int32_t* h_prefix_len,
                       const int32_t* h_live_blocks, int32_t n, int32_t* h_out);
 
@@ -264,7 +278,9 @@ int fb_scatter_window_kv(fb_ctx* ctx, const fb_pack* pk,
  * One scale per head rather than per page: a page is filled by several commits
  * and frozen positions are never rewritten.  Contexts need window_in_pages = 1
  * (the scatter is the quantiser, so every key the attention reads is a paged
- * 8-bit one) and head_dim = 128; FB_ERR_UNSUPPORTED otherwise.
+ * 8-bit one), head_dim = 128 and kv_fp8 = 1 in the configuration;
+ * FB_ERR_UNSUPPORTED otherwise (and fb_wavefront_attn / fb_scatter_window_kv
+ * refuse a kv_fp8 context).
  *   k_pool8, v_pool8  [num_pages, n_kv_heads, 64, head_dim] uint8 (E4M3)
  *   k_scale, v_scale  [n_kv_heads] fp32, positive, DEVICE pointers
  *

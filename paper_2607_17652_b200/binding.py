@@ -41,12 +41,14 @@ class fb_config(C.Structure):
         [(n, C.c_float) for n in ("tau_mask", "tau_edit", "theta_spawn",
                                   "sm_scale")] + \
         [("window_in_pages", C.c_int32), ("batch_sync", C.c_int32),
-         ("delta_literal", C.c_int32), ("force_progress", C.c_int32)]
+         ("delta_literal", C.c_int32), ("force_progress", C.c_int32),
+         ("kv_fp8", C.c_int32)]
 
 
 class fb_tuning(C.Structure):
     _fields_ = [("attn_target_items", C.c_int32),
                 ("attn_min_chunk_tiles", C.c_int32),
+                ("attn_pair", C.c_int32), ("reserved", C.c_int32),
                 ("wait_cycles", C.c_int64)]
 
 
@@ -168,9 +170,12 @@ class Context:
         """fb_attn_plan_host: what the attention work list of such a batch holds."""
         p = np.ascontiguousarray(prefix_len, np.int32)
         w = np.ascontiguousarray(live_blocks, np.int32)
-        out = np.zeros(6, np.int32)
+        out = np.zeros(12, np.int32)
         self.check(lib().fb_attn_plan_host(self._h, p.ctypes.data, w.ctypes.data, len(p), out.ctypes.data))
-        return dict(zip(("units", "items", "parts", "max_units", "max_items", "max_parts"), map(int, out)))
+        names = ("units", "items", "parts", "max_units", "max_items", "max_parts")
+        d = dict(zip(names, map(int, out[:6])))                      # the one-CTA kernel's list
+        d["pair"] = dict(zip(names, map(int, out[6:])))              # the CTA-pair kernel's list
+        return d
 
     def __del__(self):
         try:

@@ -15,7 +15,7 @@ CSRC = os.path.join(HERE, "csrc")
 ROOT = os.path.dirname(HERE)
 LIB = os.path.join(HERE, "libflowblock.so")
 SOURCES = ["api.cu", "pack.cu", "t2t.cu", "gate_commit.cu", "attn_sm100.cu", "scatter.cu", "lm_head.cu",
-           "attn_static.cu"]
+           "attn_static.cu", "attn_pair_sm100.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo",
               "-std=c++17", "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

@@ -23,23 +23,33 @@ int fail(fb_ctx* ctx, int code, const std::string& msg) {
 
 namespace fb {
 
-WsLayout make_ws_layout(const fb_config& c, int tiles_per_slot, int target_items, int min_chunk_tiles) {
+WsLayout make_ws_layout(const fb_config& c, int tiles_per_slot, int target_items, int min_chunk_tiles, int pair_on) {
   WsLayout w{};
   const long long qtiles = (long long)c.max_requests * c.wmax * tiles_per_slot;
-  w.max_units = (int)((qtiles + c.max_requests + 1) / 2) * c.n_kv_heads;
-  // split pieces: the bound that split_rule derives, and never more than every unit cut into
-  // pieces of the minimum length (a unit spans at most the keys its page-table row can address)
   const long long max_tiles = ((long long)c.max_pages_per_req * kPage + kTileN - 1) / kTileN + 2;
-  const long long every = (long long)w.max_units * ((max_tiles + min_chunk_tiles - 1) / min_chunk_tiles);
-  const long long by_target = (long long)kPartsPerTarget * target_items + 8;
-  w.max_parts = (int)(by_target < every ? by_target : every);
-  w.max_items = w.max_units + w.max_parts;
   size_t off = 0;
-  w.header = off;  off = align_up(off + sizeof(SchedHeader), 256);
-  w.items = off;   off = align_up(off + (size_t)w.max_items * sizeof(AttnItem), 256);
-  w.units = off;   off = align_up(off + (size_t)w.max_units * sizeof(AttnUnit), 256);
-  w.part_ml = off; off = align_up(off + (size_t)w.max_parts * 2 * kTileM * 2 * sizeof(float), 256);
-  w.part_o = off;  off = align_up(off + (size_t)w.max_parts * 2 * kTileM * c.head_dim * sizeof(float), 256);
+  for (int l = 0; l < 2; ++l) {
+    WsList& x = w.l[l];
+    // list 0: every two tiles a unit (plus one leftover unit per request and two KV heads);
+    // list 1: every four tiles of a request and KV head two unit records
+    const long long units = l == 0 ? ((qtiles + c.max_requests + 1) / 2) * c.n_kv_heads
+                                   : (pair_on ? (qtiles / 4) * 2 * c.n_kv_heads : 0);
+    const int target = l == 0 ? target_items : (target_items > 1 ? target_items / 2 : 1);
+    const int mult = l + 1;
+    // split pieces: the bound that split_rule derives (per scheduling unit; list 1 has two records
+    // per unit), and never more than every unit cut into pieces of the minimum length (a unit spans
+    // at most the keys its page-table row can address)
+    const long long every = units * ((max_tiles + min_chunk_tiles - 1) / min_chunk_tiles);
+    const long long by_target = mult * ((long long)kPartsPerTarget * target + 8);
+    x.max_units = (int)units;
+    x.max_parts = units ? (int)(by_target < every ? by_target : every) : 0;
+    x.max_items = x.max_units + x.max_parts;
+    x.header = off;  off = align_up(off + sizeof(SchedHeader), 256);
+    x.items = off;   off = align_up(off + (size_t)x.max_items * sizeof(AttnItem), 256);
+    x.units = off;   off = align_up(off + (size_t)x.max_units * sizeof(AttnUnit), 256);
+    x.part_ml = off; off = align_up(off + (size_t)x.max_parts * 2 * kTileM * 2 * sizeof(float), 256);
+    x.part_o = off;  off = align_up(off + (size_t)x.max_parts * 2 * kTileM * c.head_dim * sizeof(float), 256);
+  }
   w.total = off;
   return w;
 }
@@ -103,6 +113,10 @@ int fb_create(const fb_config* cfg, fb_ctx** out) {
     return fail(nullptr, FB_ERR_INVALID_ARG, "window_in_pages must be 0 or 1");
   if (c.batch_sync != 0 && c.batch_sync != 1)
     return fail(nullptr, FB_ERR_INVALID_ARG, "batch_sync must be 0 or 1");
+  if (c.kv_fp8 != 0 && c.kv_fp8 != 1) return fail(nullptr, FB_ERR_INVALID_ARG, "kv_fp8 must be 0 or 1");
+  if (c.kv_fp8 && (!c.window_in_pages || c.head_dim != 128))
+    return fail(nullptr, FB_ERR_UNSUPPORTED,
+                "kv_fp8 = 1 needs window_in_pages = 1 (the scatter is the quantiser) and head_dim = 128");
   if ((long long)c.max_requests * c.wmax * c.block_len > (1ll << 24))
     return fail(nullptr, FB_ERR_UNSUPPORTED, "max_requests * wmax * block_len is too large");
   fb_ctx* ctx = new (std::nothrow) fb_ctx();
@@ -114,8 +128,9 @@ int fb_create(const fb_config* cfg, fb_ctx** out) {
   ctx->target_items = fb::kDefaultTargetItems;
   ctx->min_chunk_tiles = fb::kDefaultMinChunkTiles;
   ctx->wait_cycles = fb::kDefaultWaitCycles;
+  ctx->pair_on = 0;                      // the CTA-pair kernel is opt-in (fb_tuning.attn_pair)
   ctx->sm_scale = c.sm_scale > 0.f ? c.sm_scale : 1.0f / sqrtf((float)c.head_dim);
-  ctx->ws = fb::make_ws_layout(c, ctx->tiles_per_slot, ctx->target_items, ctx->min_chunk_tiles);
+  ctx->ws = fb::make_ws_layout(c, ctx->tiles_per_slot, ctx->target_items, ctx->min_chunk_tiles, ctx->pair_on);
   *out = ctx;
   return FB_OK;
 }
@@ -124,12 +139,13 @@ int fb_set_tuning(fb_ctx* ctx, const fb_tuning* t) {
   if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");
   if (!t) return fail(ctx, FB_ERR_INVALID_ARG, "tuning is null");
   if (t->attn_target_items < 0 || t->attn_target_items > (1 << 20) || t->attn_min_chunk_tiles < 0 ||
-      t->attn_min_chunk_tiles > 4096 || t->wait_cycles < -1)
+      t->attn_min_chunk_tiles > 4096 || t->wait_cycles < -1 || (t->attn_pair != 0 && t->attn_pair != 1))
     return fail(ctx, FB_ERR_INVALID_ARG, "a tuning value is out of range");
   ctx->target_items = t->attn_target_items ? t->attn_target_items : fb::kDefaultTargetItems;
   ctx->min_chunk_tiles = t->attn_min_chunk_tiles ? t->attn_min_chunk_tiles : fb::kDefaultMinChunkTiles;
   ctx->wait_cycles = t->wait_cycles ? (long long)t->wait_cycles : fb::kDefaultWaitCycles;
-  ctx->ws = fb::make_ws_layout(ctx->cfg, ctx->tiles_per_slot, ctx->target_items, ctx->min_chunk_tiles);
+  ctx->pair_on = ctx->cfg.head_dim == 128 && !ctx->cfg.kv_fp8 && t->attn_pair;
+  ctx->ws = fb::make_ws_layout(ctx->cfg, ctx->tiles_per_slot, ctx->target_items, ctx->min_chunk_tiles, ctx->pair_on);
   return FB_OK;
 }
 
@@ -145,29 +161,35 @@ int fb_attn_plan_host(const fb_ctx* ctx, const int32_t* h_prefix_len, const int3
   if (!ctx || !h_prefix_len || !h_live_blocks || !h_out || n < 0 || n > ctx->cfg.max_requests)
     return fail(nullptr, FB_ERR_INVALID_ARG, "fb_attn_plan_host: null argument or n outside [0, max_requests]");
   const fb_config& c = ctx->cfg;
-  long long total = 0, units = 0;
-  for (int r = 0; r < n; ++r) {
+  for (int r = 0; r < n; ++r)
     if (h_live_blocks[r] < 0 || h_live_blocks[r] > c.wmax)
       return fail(nullptr, FB_ERR_INVALID_ARG, "fb_attn_plan_host: live blocks outside [0, wmax]");
-    const fb::ReqGeom g = fb::req_geom_of(h_live_blocks[r], h_prefix_len[r], ctx->tiles_per_slot, c.block_len,
-                                          c.n_kv_heads, c.window_in_pages);
-    total += (long long)g.nunits * g.nt;
-    units += g.nt ? g.nunits : 0;
+  for (int list = 0; list < 2; ++list) {
+    const int target = list == 0 ? ctx->target_items : (ctx->target_items > 1 ? ctx->target_items / 2 : 1);
+    const int mult = list + 1;
+    long long total = 0, units = 0;
+    for (int r = 0; r < n; ++r) {
+      const fb::ReqGeom g = fb::req_geom_of(h_live_blocks[r], h_prefix_len[r], ctx->tiles_per_slot, c.block_len,
+                                            c.n_kv_heads, c.window_in_pages, list, ctx->pair_on);
+      total += (long long)g.nunits * g.nt;
+      units += g.nt ? g.nunits : 0;
+    }
+    if (total > 0x7fffffffll) return fail(nullptr, FB_ERR_UNSUPPORTED, "fb_attn_plan_host: work list too long");
+    const fb::SplitRule rule = fb::split_rule((int)total, (int)units, target, ctx->min_chunk_tiles);
+    long long wbase = 0, items = 0, parts = 0;
+    for (int r = 0; r < n; ++r) {
+      const fb::ReqGeom g = fb::req_geom_of(h_live_blocks[r], h_prefix_len[r], ctx->tiles_per_slot, c.block_len,
+                                            c.n_kv_heads, c.window_in_pages, list, ctx->pair_on);
+      const int nunits = g.nt ? g.nunits : 0;
+      const fb::ReqSplit rs = fb::req_split(rule, (int)wbase, nunits, g.nt);
+      items += rs.items(nunits);
+      parts += rs.parts(nunits);
+      wbase += (long long)nunits * g.nt;
+    }
+    int32_t* o = h_out + 6 * list;
+    o[0] = (int32_t)(mult * units); o[1] = (int32_t)items; o[2] = (int32_t)(mult * parts);
+    o[3] = ctx->ws.l[list].max_units; o[4] = ctx->ws.l[list].max_items; o[5] = ctx->ws.l[list].max_parts;
   }
-  if (total > 0x7fffffffll) return fail(nullptr, FB_ERR_UNSUPPORTED, "fb_attn_plan_host: work list too long");
-  const fb::SplitRule rule = fb::split_rule((int)total, (int)units, ctx->target_items, ctx->min_chunk_tiles);
-  long long wbase = 0, items = 0, parts = 0;
-  for (int r = 0; r < n; ++r) {
-    const fb::ReqGeom g = fb::req_geom_of(h_live_blocks[r], h_prefix_len[r], ctx->tiles_per_slot, c.block_len,
-                                          c.n_kv_heads, c.window_in_pages);
-    const int nunits = g.nt ? g.nunits : 0;
-    const fb::ReqSplit rs = fb::req_split(rule, (int)wbase, nunits, g.nt);
-    items += rs.items(nunits);
-    parts += rs.parts(nunits);
-    wbase += (long long)nunits * g.nt;
-  }
-  h_out[0] = (int32_t)units; h_out[1] = (int32_t)items; h_out[2] = (int32_t)parts;
-  h_out[3] = ctx->ws.max_units; h_out[4] = ctx->ws.max_items; h_out[5] = ctx->ws.max_parts;
   return FB_OK;
 }
 
@@ -191,6 +213,7 @@ int fb_wavefront_attn(fb_ctx* ctx, const fb_pack* pk, const void* q, const void*
                       int32_t* status, void* stream) {
   if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");
   if (int e = check_pack(ctx, pk)) return e;
+  if (ctx->cfg.kv_fp8) return fail(ctx, FB_ERR_UNSUPPORTED, "this context holds 8-bit pages: use fb_wavefront_attn_fp8");
   const bool resident = ctx->cfg.window_in_pages != 0;
   if (!q || !k_pool || !v_pool || !page_table || !out)
     return fail(ctx, FB_ERR_INVALID_ARG, "a tensor pointer is null");
@@ -212,6 +235,7 @@ int fb_scatter_window_kv(fb_ctx* ctx, const fb_pack* pk, const int32_t* page_tab
                          void* stream) {
   if (!ctx) return fail(nullptr, FB_ERR_INVALID_ARG, "ctx is null");
   if (int e = check_pack(ctx, pk)) return e;
+  if (ctx->cfg.kv_fp8) return fail(ctx, FB_ERR_UNSUPPORTED, "this context holds 8-bit pages: use fb_scatter_window_kv_fp8");
   if (!page_table || !k_new || !v_new || !k_pool || !v_pool || !status)
     return fail(ctx, FB_ERR_INVALID_ARG, "a tensor pointer is null");
   if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_pool) || !aligned16(v_pool))
@@ -222,9 +246,8 @@ int fb_scatter_window_kv(fb_ctx* ctx, const fb_pack* pk, const int32_t* page_tab
 }
 
 static int check_fp8_ctx(fb_ctx* ctx) {
-  if (!ctx->cfg.window_in_pages)
-    return fail(ctx, FB_ERR_UNSUPPORTED, "8-bit KV pages need a context with window_in_pages = 1 (the window is quantised into the pages by the scatter)");
-  if (ctx->cfg.head_dim != 128) return fail(ctx, FB_ERR_UNSUPPORTED, "8-bit KV pages: head_dim must be 128");
+  if (!ctx->cfg.kv_fp8)
+    return fail(ctx, FB_ERR_UNSUPPORTED, "8-bit KV pages need a context created with kv_fp8 = 1 (window_in_pages = 1, head_dim = 128)");
   return FB_OK;
 }
 

@@ -33,127 +33,9 @@
 // workspace and a second kernel merges them in a fixed order.
 #include <cudaTypedefs.h>
 
-#include "fb_common.cuh"
-#include "ptx_sm100.cuh"
+#include "attn_common.cuh"
 
 namespace fb {
-
-constexpr int kAttnThreads = 384;   // 3 warpgroups: control, softmax A, softmax B
-constexpr float kLog2eF = 1.4426950408889634f;
-constexpr float kRescaleThreshold = 8.0f;   // log2 units
-// Dynamic shared memory per CTA.  Both sizes exceed half of the 227 KB an SM
-// offers, so two CTAs never share an SM: each CTA allocates all 512 TMEM columns.
-constexpr int kSmem64 = 120 * 1024;
-constexpr int kSmem128 = 6 * 32768 + 8192;
-constexpr int kSmemF8 = 2 * 32768 + 6 * 16384 + 8192;   // Q staging (bf16), Q / K / V tiles in 8 bits
-// 8-bit pages: the exponentials are taken 2^4 above the reference, so that E4M3 (normal down to
-// 2^-6, largest value 448) holds P from 2^-10 of the reference up to the 2^8 bound of the lazy re-base
-constexpr float kF8PShift = 4.0f;
-
-struct AttnParams {
-  SchedHeader* hdr;
-  const AttnItem* items;
-  const AttnUnit* units;
-  const int32_t* page_table;
-  __nv_bfloat16* out;
-  float* part_ml;
-  float* part_o;
-  int32_t* status;
-  int32_t bl, n_q_heads, n_kv_heads, group, max_pages_per_req, num_pages;
-  int32_t resident;     // 1: the window is read from the pages (every key tile is a paged one)
-  const float* k_scale; // 8-bit pages only: value = code * scale of the KV head, [n_kv_heads]
-  const float* v_scale;
-  float scale_log2;
-  long long wait_cycles;
-};
-
-// Geometry of one work item, computed identically by every role.
-struct ItemGeom {
-  AttnUnit un;
-  int jb, n, nA, nB, chunk, kvhA, kvhB;
-};
-
-__device__ __forceinline__ bool load_item(const AttnParams& p, int idx, ItemGeom& g) {
-  const int4 it = *reinterpret_cast<const int4*>(&p.items[idx]);
-  const int4* up = reinterpret_cast<const int4*>(&p.units[it.x]);
-  const int4 u0 = up[0], u1 = up[1], u2 = up[2], u3 = up[3];
-  g.un.req = u0.x; g.un.kvh = u0.y; g.un.slotA = u0.z; g.un.slotB = u0.w;
-  g.kvhA = u0.y & 0xffff; g.kvhB = u0.y >> 16;
-  g.un.t0A = u1.x; g.un.t0B = u1.y; g.un.n_tiles = u1.z; g.un.n_chunks = u1.w;
-  g.un.nvisA = u2.x; g.un.nvisB = u2.y; g.un.part_base = u2.z; g.un.prefix_len = u2.w;
-  g.un.npt = u3.x; g.un.win_row0 = u3.y; g.un.winA = u3.z; g.un.winB = u3.w;
-  g.chunk = it.y; g.jb = it.z;
-  const int je = it.w;
-  g.nA = max(0, min(je, g.un.nvisA) - g.jb);
-  g.nB = g.un.slotB >= 0 ? max(0, min(je, g.un.nvisB) - g.jb) : 0;
-  g.n = max(g.nA, g.nB);
-  return g.n > 0;
-}
-
-// 2^x for a pair of values on the FMA pipe (the MUFU pipe is as busy as the
-// tensor pipe in this kernel, so a share of the exponentials is moved off it):
-// round-to-nearest split x = n + f, f in [-0.5, 0.5], cubic minimax fit of 2^f
-// (max relative error 7.5e-5, far below bf16 resolution), then n is added to
-// the exponent field.  Valid for -120 <= x <= 120.
-constexpr int kPolyOf4 = 1;   // pairs out of every 4 that take this path (bf16 pages)
-constexpr int kPolyOf4F8 = 1;   // the same share with 8-bit pages (0, 2 and 3 of 4 measured slower)
-__device__ __forceinline__ float2 exp2_poly2(float2 x) {
-  x.x = fmaxf(x.x, -120.f);
-  x.y = fmaxf(x.y, -120.f);
-  const float kMagic = 12582912.f;   // 1.5 * 2^23: x + kMagic has round(x) in its low mantissa bits
-  const float2 t = __fadd2_rn(x, make_float2(kMagic, kMagic));
-  const float2 n = __fadd2_rn(t, make_float2(-kMagic, -kMagic));
-  const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
-  float2 q = __ffma2_rn(make_float2(0.05517137795686722f, 0.05517137795686722f), f,
-                        make_float2(0.24261121451854706f, 0.24261121451854706f));
-  q = __ffma2_rn(q, f, make_float2(0.6932610273361206f, 0.6932610273361206f));
-  q = __ffma2_rn(q, f, make_float2(0.9999280571937561f, 0.9999280571937561f));
-  q.x = __int_as_float(__float_as_int(q.x) + (__float_as_int(t.x) << 23));
-  q.y = __int_as_float(__float_as_int(q.y) + (__float_as_int(t.y) << 23));
-  return q;
-}
-
-__device__ __forceinline__ int uni(int x) { return __shfl_sync(0xffffffffu, x, 0); }
-
-// The subset of an item the control warps need, made warp-uniform (every lane
-// holds lane 0's copy) so that the compiler keeps it in uniform registers.
-struct ItemU {
-  int req, kvhA, kvhB, rowA, rowB, jb, n, nA, nB, npt, prefix_len, win_row0, winA, winB;
-  __device__ __forceinline__ bool dual() const { return kvhA != kvhB; }   // two K/V streams
-  // keys of local tile j that a tile with window reach winX may see; `resident`: the
-  // window follows the prefix in the pages, one run of keys [0, prefix_len + winX)
-  __device__ __forceinline__ int limit(int j, int winX, int resident) const {
-    const int gj = jb + j;
-    const int lim = gj < npt ? prefix_len + (resident ? winX : 0) - gj * kTileN : winX - (gj - npt) * kTileN;
-    return min(lim, kTileN);
-  }
-};
-
-__device__ __forceinline__ bool load_item_uniform(const AttnParams& p, int idx, ItemU& u) {
-  ItemGeom g;
-  load_item(p, idx, g);
-  u.req = uni(g.un.req); u.kvhA = uni(g.kvhA); u.kvhB = uni(g.kvhB);
-  u.rowA = uni(g.un.slotA * p.bl + g.un.t0A); u.rowB = uni(g.un.slotB * p.bl + g.un.t0B);
-  u.jb = uni(g.jb); u.n = uni(g.n); u.nA = uni(g.nA); u.nB = uni(g.nB);
-  u.npt = uni(g.un.npt); u.prefix_len = uni(g.un.prefix_len); u.win_row0 = uni(g.un.win_row0);
-  u.winA = uni(g.un.winA); u.winB = uni(g.un.winB);
-  return u.n > 0;
-}
-
-// All lanes of a converged warp wait on the barrier; the result is uniform.
-__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort, long long limit) {
-  const bool ok = mbar_wait(bar, parity, abort, limit);
-  return __all_sync(0xffffffffu, ok);
-}
-
-// number of keys of local tile j that tile X (window reach winX) may see
-__device__ __forceinline__ int tile_limit(const ItemGeom& g, int j, int winX, int resident) {
-  const int gj = g.jb + j;
-  const int lim = gj < g.un.npt ? g.un.prefix_len + (resident ? winX : 0) - gj * kTileN
-                                : winX - (gj - g.un.npt) * kTileN;
-  return min(lim, kTileN);
-}
-__device__ __forceinline__ int round16(int x) { return (x + 15) & ~15; }
 
 // F8: the KV pages hold FP8 E4M3 bytes (window resident in the pages, D = 128).  Both products
 // then run as kind::f8f6f4 MMAs: the softmax warps convert their Q tile to E4M3 once per item
@@ -632,6 +514,9 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           m_ref = fmaxf(fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3])), fmaxf(fmaxf(m8[4], m8[5]), fmaxf(m8[6], m8[7])));
         }
         uint32_t pk[F8 ? 32 : 64];             // P of this tile: packed bf16 pairs, or E4M3 four to a word
+        // 8-bit P saturates at 448, so the largest exponent of the tile is tracked element by
+        // element; bf16 P has the range of fp32 and only needs the tile's sum to stay finite
+        constexpr bool TRACK = F8;
         float tile_sum = 0.f;
 #pragma unroll 1
         for (int attempt = 0; attempt < 2; ++attempt) {
@@ -651,7 +536,7 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
 #pragma unroll
               for (int i = 0; i < 32; i += 2) {
                 const float2 x = __ffma2_rn(make_float2(__uint_as_float(sr[i]), __uint_as_float(sr[i + 1])), sl2v, nmb);
-                xm4[(i >> 1) & 3] = max3(xm4[(i >> 1) & 3], x.x, x.y);
+                if constexpr (TRACK) xm4[(i >> 1) & 3] = max3(xm4[(i >> 1) & 3], x.x, x.y);
                 float2 pv;
                 if (((i >> 1) & 3) < (F8 ? kPolyOf4F8 : kPolyOf4)) pv = exp2_poly2(x);
                 else pv = make_float2(ex2_approx(x.x), ex2_approx(x.y));
@@ -669,8 +554,10 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
               for (int i = 0; i < 32; i += 2) {
                 const bool v0 = 32 * c + i < limit, v1 = 32 * c + i + 1 < limit;
                 const float x0 = fmaf(__uint_as_float(sr[i]), sl2, -mb), x1 = fmaf(__uint_as_float(sr[i + 1]), sl2, -mb);
-                if (v0) xm4[0] = fmaxf(xm4[0], x0);
-                if (v1) xm4[1] = fmaxf(xm4[1], x1);
+                if constexpr (TRACK) {
+                  if (v0) xm4[0] = fmaxf(xm4[0], x0);
+                  if (v1) xm4[1] = fmaxf(xm4[1], x1);
+                }
                 const float p0 = v0 ? ex2_approx(x0) : 0.f, p1 = v1 ? ex2_approx(x1) : 0.f;
                 acc2[0].x += p0 + p1;
                 if constexpr (F8) {
@@ -683,9 +570,21 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             }
           }
           tile_sum = (acc2[0].x + acc2[0].y) + (acc2[1].x + acc2[1].y);
-          const float xmax = fmaxf(fmaxf(xm4[0], xm4[1]), fmaxf(xm4[2], xm4[3]));
-          const bool grow = attempt == 0 && xmax > kRescaleThreshold;
+          float xmax = fmaxf(fmaxf(xm4[0], xm4[1]), fmaxf(xm4[2], xm4[3]));
+          const bool grow = attempt == 0 && (TRACK ? xmax > kRescaleThreshold : !(tile_sum <= kGrowSum));
           if (!__any_sync(0xffffffffu, grow)) break;
+          if constexpr (!TRACK) {
+            // the largest exponent of the tile was not tracked: one more pass over S (whole warp)
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+              uint32_t sr[32];
+              tmem_ld32(tS + 32 * c, sr);
+              tmem_ld_wait();
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (32 * c + i < limit) xmax = fmaxf(xmax, fmaf(__uint_as_float(sr[i]), sl2, -mb));
+            }
+          }
           // rare: re-base this row's reference, rescale what has been accumulated so far
           // (O is quiescent: the commit behind this S also covered the previous P V)
           const float alpha = grow ? ex2_approx(kShift - xmax) : 1.0f;
@@ -870,6 +769,7 @@ int ensure_device(fb_ctx* ctx) {
                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemF8), "smem attr"))
     return e;
   if (int e = lm_head_device_setup(ctx)) return e;
+  if (int e = attn_pair_device_setup(ctx)) return e;
   ctx->device = dev;
   ctx->dev_ready = true;
   return FB_OK;
@@ -887,16 +787,17 @@ static int encode(fb_ctx* ctx, CUtensorMap* m, const void* base, int rank, const
   return FB_OK;
 }
 
-static void fill_params(fb_ctx* ctx, AttnParams& p, const int32_t* page_table, void* out, void* ws, int32_t* status) {
+void fill_attn_params(fb_ctx* ctx, AttnParams& p, const int32_t* page_table, void* out, void* ws, int32_t* status,
+                      int list) {
   const fb_config& c = ctx->cfg;
   uint8_t* w = static_cast<uint8_t*>(ws);
-  p.hdr = reinterpret_cast<SchedHeader*>(w + ctx->ws.header);
-  p.items = reinterpret_cast<const AttnItem*>(w + ctx->ws.items);
-  p.units = reinterpret_cast<const AttnUnit*>(w + ctx->ws.units);
+  p.hdr = reinterpret_cast<SchedHeader*>(w + ctx->ws.l[list].header);
+  p.items = reinterpret_cast<const AttnItem*>(w + ctx->ws.l[list].items);
+  p.units = reinterpret_cast<const AttnUnit*>(w + ctx->ws.l[list].units);
   p.page_table = page_table;
   p.out = static_cast<__nv_bfloat16*>(out);
-  p.part_ml = reinterpret_cast<float*>(w + ctx->ws.part_ml);
-  p.part_o = reinterpret_cast<float*>(w + ctx->ws.part_o);
+  p.part_ml = reinterpret_cast<float*>(w + ctx->ws.l[list].part_ml);
+  p.part_o = reinterpret_cast<float*>(w + ctx->ws.l[list].part_o);
   p.status = status;
   p.bl = c.block_len; p.n_q_heads = c.n_q_heads; p.n_kv_heads = c.n_kv_heads; p.group = ctx->group;
   p.max_pages_per_req = c.max_pages_per_req; p.num_pages = c.num_pages;
@@ -904,6 +805,13 @@ static void fill_params(fb_ctx* ctx, AttnParams& p, const int32_t* page_table, v
   p.k_scale = nullptr; p.v_scale = nullptr;
   p.scale_log2 = ctx->sm_scale * kLog2eF;
   p.wait_cycles = ctx->wait_cycles;
+}
+
+int launch_attn_combine(fb_ctx* ctx, const AttnParams& p, int list, cudaStream_t stream) {
+  const int grid = min(max(ctx->ws.l[list].max_units, 1) * kCombineSplit, kCombineCtasPerSm * ctx->num_sms);
+  if (ctx->cfg.head_dim == 64)
+    return cuda_err(ctx, launch_pdl(attn_combine_kernel<64>, grid, 256, 0, stream, p), "attn_combine_kernel launch");
+  return cuda_err(ctx, launch_pdl(attn_combine_kernel<128>, grid, 256, 0, stream, p), "attn_combine_kernel launch");
 }
 
 static int encode_q(fb_ctx* ctx, const void* q) {
@@ -933,6 +841,8 @@ int launch_attn(fb_ctx* ctx, const fb_pack* pk, const void* q, const void* k_win
       // window resident in the pages: no window tensors; the two maps are never used then
       if (int e = encode(ctx, &ctx->tm_kwin, k_win ? k_win : k_pool, 3, dims, str, box)) return e;
       if (int e = encode(ctx, &ctx->tm_vwin, v_win ? v_win : v_pool, 3, dims, str, box)) return e;
+      cuuint32_t half[3] = {64, 1, 64};       // the CTA-pair kernel: each CTA takes 64 of a tile's 128 window keys
+      if (int e = encode(ctx, &ctx->tm_kwin_half, k_win ? k_win : k_pool, 3, dims, str, half)) return e;
     }
     {
       cuuint64_t dims[2] = {D, (cuuint64_t)c.num_pages * c.n_kv_heads * kPage};
@@ -945,23 +855,23 @@ int launch_attn(fb_ctx* ctx, const fb_pack* pk, const void* q, const void* k_win
     ctx->maps_f8 = false;
   }
   AttnParams p;
-  fill_params(ctx, p, page_table, out, ws, status);
+  fill_attn_params(ctx, p, page_table, out, ws, status, 0);
   const int grid = ctx->num_sms;
-  const int combine_grid = min(ctx->ws.max_units * kCombineSplit, kCombineCtasPerSm * ctx->num_sms);
   if (c.head_dim == 64) {
     if (int e = cuda_err(ctx, launch_pdl(wavefront_attn_kernel<64, false>, grid, kAttnThreads, kSmem64, stream, ctx->tm_q,
                                          ctx->tm_kwin, ctx->tm_vwin, ctx->tm_kpool, ctx->tm_vpool, p),
                          "wavefront_attn_kernel launch"))
       return e;
-    return cuda_err(ctx, launch_pdl(attn_combine_kernel<64>, combine_grid, 256, 0, stream, p),
-                    "attn_combine_kernel launch");
+    return launch_attn_combine(ctx, p, 0, stream);
   }
+  // quads first (the CTA-pair kernel), then everything else
+  if (ctx->pair_on)
+    if (int e = launch_attn_pair(ctx, page_table, out, ws, status, stream)) return e;
   if (int e = cuda_err(ctx, launch_pdl(wavefront_attn_kernel<128, false>, grid, kAttnThreads, kSmem128, stream, ctx->tm_q,
                                        ctx->tm_kwin, ctx->tm_vwin, ctx->tm_kpool, ctx->tm_vpool, p),
                        "wavefront_attn_kernel launch"))
     return e;
-  return cuda_err(ctx, launch_pdl(attn_combine_kernel<128>, combine_grid, 256, 0, stream, p),
-                  "attn_combine_kernel launch");
+  return launch_attn_combine(ctx, p, 0, stream);
 }
 
 // Attention over 8-bit pages (window resident in the pages, head_dim 128): the pools are E4M3
@@ -985,15 +895,13 @@ int launch_attn_fp8(fb_ctx* ctx, const fb_pack* pk, const void* q, const void* k
     ctx->maps_f8 = true;
   }
   AttnParams p;
-  fill_params(ctx, p, page_table, out, ws, status);
+  fill_attn_params(ctx, p, page_table, out, ws, status, 0);
   p.k_scale = k_scale; p.v_scale = v_scale;
-  const int combine_grid = min(ctx->ws.max_units * kCombineSplit, kCombineCtasPerSm * ctx->num_sms);
   if (int e = cuda_err(ctx, launch_pdl(wavefront_attn_kernel<128, true>, ctx->num_sms, kAttnThreads, (size_t)kSmemF8, stream,
                                        ctx->tm_q, ctx->tm_kwin, ctx->tm_vwin, ctx->tm_kpool, ctx->tm_vpool, p),
                        "wavefront_attn_kernel (8-bit pages) launch"))
     return e;
-  return cuda_err(ctx, launch_pdl(attn_combine_kernel<128>, combine_grid, 256, 0, stream, p),
-                  "attn_combine_kernel launch");
+  return launch_attn_combine(ctx, p, 0, stream);
 }
 
 }  // namespace fb

@@ -39,15 +39,21 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 fb::WsLayout unsplit_layout(const fb_ctx* c) {
   fb::WsLayout w{};
   const long long qtiles = (long long)c->cfg.max_requests * c->cfg.wmax * c->tiles_per_slot;
-  w.max_units = (int)((qtiles + c->cfg.max_requests + 1) / 2) * c->cfg.n_kv_heads;
-  w.max_items = w.max_units + 8;
-  w.max_parts = 2;        // never used: no unit is split
+  fb::WsList& x = w.l[0];
+  x.max_units = (int)((qtiles + c->cfg.max_requests + 1) / 2) * c->cfg.n_kv_heads;
+  x.max_items = x.max_units + 8;
+  x.max_parts = 2;        // never used: no unit is split
   size_t off = 0;
-  w.header = off;  off = align_up(off + sizeof(fb::SchedHeader), 256);
-  w.items = off;   off = align_up(off + (size_t)w.max_items * sizeof(fb::AttnItem), 256);
-  w.units = off;   off = align_up(off + (size_t)w.max_units * sizeof(fb::AttnUnit), 256);
-  w.part_ml = off; off = align_up(off + (size_t)w.max_parts * 2 * fb::kTileM * 2 * sizeof(float), 256);
-  w.part_o = off;  off = align_up(off + (size_t)w.max_parts * 2 * fb::kTileM * c->cfg.head_dim * sizeof(float), 256);
+  x.header = off;  off = align_up(off + sizeof(fb::SchedHeader), 256);
+  x.items = off;   off = align_up(off + (size_t)x.max_items * sizeof(fb::AttnItem), 256);
+  x.units = off;   off = align_up(off + (size_t)x.max_units * sizeof(fb::AttnUnit), 256);
+  x.part_ml = off; off = align_up(off + (size_t)x.max_parts * 2 * fb::kTileM * 2 * sizeof(float), 256);
+  x.part_o = off;  off = align_up(off + (size_t)x.max_parts * 2 * fb::kTileM * c->cfg.head_dim * sizeof(float), 256);
+  // the second work list (CTA-pair kernel) stays empty here: a header and nothing else
+  fb::WsList& y = w.l[1];
+  y.max_units = y.max_items = y.max_parts = 0;
+  y.header = off;  off = align_up(off + sizeof(fb::SchedHeader), 256);
+  y.items = y.units = y.part_ml = y.part_o = off;
   w.total = off;
   return w;
 }
@@ -106,6 +112,7 @@ extern "C" int fb_wavefront_attn_static(fb_ctx* ctx, const fb_state* st, const f
     sh->sm_scale = ctx->sm_scale;
     sh->target_items = 1;                 // chunk length = all tiles: nothing is split
     sh->min_chunk_tiles = 1 << 20;
+    sh->pair_on = 0;                      // one work list, one kernel
     sh->ws = lay;
   }
   sh->wait_cycles = ctx->wait_cycles;

@@ -40,9 +40,15 @@ struct SchedHeader {
   int32_t pad[9];
 };
 
-struct WsLayout {
-  size_t header, items, units, part_ml, part_o, total;
+// The workspace holds two work lists: list 0 for the one-CTA kernel, list 1 ("quads": four Q
+// tiles of one request and KV head) for the CTA-pair kernel.  List 1 is empty when pairing is off.
+struct WsList {
+  size_t header, items, units, part_ml, part_o;
   int32_t max_items, max_units, max_parts;
+};
+struct WsLayout {
+  WsList l[2];
+  size_t total;
 };
 
 // ---------------------------------------------------------------------------
@@ -54,19 +60,28 @@ struct WsLayout {
 // An odd tile left over is paired with itself across two adjacent KV heads
 // instead: the two halves stream different K/V but keep both tile slots of a
 // CTA busy, which a lone tile cannot.  nunits counts both kinds.
+// With pairing on, the first 4 * nquad tiles of a request go to list 1 as quads (one scheduling
+// unit per quad and KV head, run by a pair of CTAs: tiles 4q + r and 4q + 2 + r in CTA r); list 0
+// takes the remaining ntq tiles, starting at tile0.
 struct ReqGeom {
-  int w, ntq, npairs, P, npt, nt;
-  int nfull, odd, nunits;   // full pairs per KV head; leftover tile; units of the request
+  int w, ntq, tile0, nquad, P, npt, nt;
+  int nfull, odd, nunits;   // full pairs per KV head; leftover tile; scheduling units of the request in this list
 };
 __host__ __device__ inline ReqGeom req_geom_of(int w, int prefix_len, int tiles_per_slot, int bl, int n_kv_heads,
-                                               int resident) {
+                                               int resident, int list, int pair_on) {
   ReqGeom g;
   g.w = w;
-  g.ntq = g.w * tiles_per_slot;
-  g.npairs = (g.ntq + 1) >> 1;
-  g.nfull = g.ntq >> 1;
-  g.odd = g.ntq & 1;
-  g.nunits = g.nfull * n_kv_heads + g.odd * ((n_kv_heads + 1) >> 1);
+  const int ntq_all = g.w * tiles_per_slot;
+  g.nquad = pair_on ? ntq_all >> 2 : 0;
+  if (list == 1) {
+    g.ntq = 4 * g.nquad; g.tile0 = 0; g.nfull = 0; g.odd = 0;
+    g.nunits = g.nquad * n_kv_heads;
+  } else {
+    g.ntq = ntq_all - 4 * g.nquad; g.tile0 = 4 * g.nquad;
+    g.nfull = g.ntq >> 1;
+    g.odd = g.ntq & 1;
+    g.nunits = g.nfull * n_kv_heads + g.odd * ((n_kv_heads + 1) >> 1);
+  }
   g.P = g.w ? (prefix_len > 0 ? prefix_len : 0) : 0;
   g.npt = (g.P + kTileN - 1) / kTileN;
   g.nt = g.w ? g.npt + (g.w * bl + kTileN - 1) / kTileN : 0;
@@ -74,6 +89,7 @@ __host__ __device__ inline ReqGeom req_geom_of(int w, int prefix_len, int tiles_
     g.nt = g.w ? (g.P + g.w * bl + kTileN - 1) / kTileN : 0;
     g.npt = g.nt;
   }
+  if (g.nunits == 0) g.nt = 0;
   return g;
 }
 
@@ -139,8 +155,9 @@ struct fb_ctx {
   int group;            // G = n_q_heads / n_kv_heads
   int tiles_per_slot;   // bl * G / 128
   int tokens_per_tile;  // 128 / G
-  int target_items;
+  int target_items;       // list 0; list 1 aims for target_items / 2 (half as many executors)
   int min_chunk_tiles;
+  int pair_on;            // quads go to the CTA-pair kernel (bf16 pages, head_dim 128)
   long long wait_cycles;  // limit of every bounded device-side wait, in SM clock cycles
   float sm_scale;
   fb::WsLayout ws;
@@ -151,6 +168,7 @@ struct fb_ctx {
   int num_sms = 0;
   void* encode_fn = nullptr;
   // cached tensor maps (re-encoded when a base pointer changes)
+  CUtensorMap tm_kwin_half;   // 64-row boxes of the window keys (CTA-pair kernel)
   const void* map_ptrs[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
   bool maps_f8 = false;   // the cached pool maps describe 8-bit pages
   CUtensorMap tm_q, tm_kwin, tm_vwin, tm_kpool, tm_vpool;
@@ -223,7 +241,9 @@ int launch_gate(fb_ctx*, const fb_pack*, const int32_t* slot_stats, const fb_sta
 
 constexpr long long kDefaultWaitCycles = 2000000000LL;   // about a second at the SM clock
 
-fb::WsLayout make_ws_layout(const fb_config& c, int tiles_per_slot, int target_items, int min_chunk_tiles);
+fb::WsLayout make_ws_layout(const fb_config& c, int tiles_per_slot, int target_items, int min_chunk_tiles, int pair_on);
+int launch_attn_pair(fb_ctx*, const int32_t* page_table, void* out, void* ws, int32_t* status, cudaStream_t);
+int attn_pair_device_setup(fb_ctx*);
 int check_state(fb_ctx* ctx, const fb_state* st);   // every member non-null, else FB_ERR_INVALID_ARG
 int check_pack(fb_ctx* ctx, const fb_pack* pk);
 void static_forget(const fb_ctx* ctx);              // drops what fb_wavefront_attn_static keeps per context

@@ -52,10 +52,12 @@ def test_create_validates_configuration():
            dict(n_kv_heads=3), dict(wmax=0), dict(vocab=1001), dict(wmax=9),
            dict(tau_edit=0.5), dict(s_pe=300), dict(max_requests=-1),
            dict(tau_mask=float("nan")), dict(window_in_pages=2), dict(batch_sync=2),
-           dict(delta_literal=2), dict(force_progress=-1)]
+           dict(delta_literal=2), dict(force_progress=-1), dict(kv_fp8=1), dict(kv_fp8=2),
+           dict(kv_fp8=1, window_in_pages=1, head_dim=64)]
     for delta in bad:
         with pytest.raises(B.FlowBlockError):
             B.Context(**dict(GOOD, **delta))
+    B.Context(**dict(GOOD, kv_fp8=1, window_in_pages=1))      # 8-bit pages: window in the pages, head_dim 128
     # thresholds the other way round are accepted only with Delta taken literally
     B.Context(**dict(GOOD, tau_edit=0.5, delta_literal=1))
     assert B.lib().fb_create(None, None) == B.FB_ERR_INVALID_ARG
@@ -164,16 +166,23 @@ def test_split_pieces_never_exceed_the_workspace_bound():
     ctx = B.Context(**_llm_cfg())
     for P in range(16384, 32768 + 1, 64):
         pl = ctx.attn_plan([P], [3])
-        assert pl["parts"] <= pl["max_parts"] and pl["items"] <= pl["max_items"], (P, pl)
-        assert pl["units"] == 24 and pl["items"] >= pl["units"]
+        for lst in (pl, pl["pair"]):
+            assert lst["parts"] <= lst["max_parts"] and lst["items"] <= lst["max_items"], (P, pl)
+        assert pl["units"] == 24 and pl["pair"]["units"] == 0 and pl["items"] >= pl["units"]
     # the batch-64 shape with one request of prefix 65536 and four live blocks
     ctx = B.Context(**_llm_cfg(max_requests=64, wmax=4, block_len=32, max_pages_per_req=1030,
                                num_pages=64 * 1030))
     pl = ctx.attn_plan([65536], [4])
-    assert 0 < pl["parts"] <= pl["max_parts"], pl
+    assert pl["pair"]["units"] == 0 and 0 < pl["parts"] <= pl["max_parts"], pl
+    ctx.set_tuning(attn_pair=1)                              # quads go to the CTA-pair kernel's list
+    pl = ctx.attn_plan([65536], [4])
+    assert pl["units"] == 0 and 0 < pl["pair"]["parts"] <= pl["pair"]["max_parts"], pl
+    lc = B.Context(tuning=dict(attn_pair=1), **_llm_cfg())
+    pl = lc.attn_plan([20000], [3])                          # six Q tiles per KV head: a quad (two records) + a pair
+    assert pl["units"] == 8 and pl["pair"]["units"] == 16
     # random batches, several tuning settings
-    for target, min_chunk in ((0, 0), (1, 0), (7, 1), (100000, 1), (296, 16), (50, 2)):
-        ctx.set_tuning(attn_target_items=target, attn_min_chunk_tiles=min_chunk)
+    for target, min_chunk, pair in ((0, 0, 1), (1, 0, 1), (7, 1, 0), (100000, 1, 1), (296, 16, 0), (50, 2, 1)):
+        ctx.set_tuning(attn_target_items=target, attn_min_chunk_tiles=min_chunk, attn_pair=pair)
         for _ in range(300):
             n = int(rg.integers(1, 65))
             P = rg.integers(0, 65536, size=n)
@@ -181,7 +190,9 @@ def test_split_pieces_never_exceed_the_workspace_bound():
                 P[:] = rg.integers(0, 400)             # many short requests
             w = rg.integers(0, 5, size=n)
             pl = ctx.attn_plan(P, w)
-            assert pl["units"] <= pl["max_units"], pl
-            assert pl["items"] <= pl["max_items"], pl
-            assert pl["parts"] <= pl["max_parts"], (target, min_chunk, pl)
+            for lst in (pl, pl["pair"]):
+                assert lst["units"] <= lst["max_units"], pl
+                assert lst["items"] <= lst["max_items"], pl
+                assert lst["parts"] <= lst["max_parts"], (target, min_chunk, pl)
+            assert (pl["pair"]["units"] == 0) == (pair == 0 or (np.asarray(w) < 4).all())
     assert B.lib().fb_attn_plan_host(ctx.handle, None, None, 0, None) == B.FB_ERR_INVALID_ARG

@@ -59,7 +59,7 @@ def _setup(wl, tuning=None, seed=None):
     tokens = synth.make_tokens(stc)
     q, kw, vw, _, _ = synth.make_attn_inputs(stc)
     k8, v8, ks, vs = synth.make_fp8_kv(stc)
-    ctx = B.Context(tuning=tuning, **H.common_cfg(stc, window_in_pages=1))
+    ctx = B.Context(tuning=tuning, kv_fp8=1, **H.common_cfg(stc, window_in_pages=1))
     st = B.DeviceState.from_numpy(DEV, stc.active, stc.prefix_len, stc.L, stc.R, tokens,
                                   np.zeros((wl.n_requests, wl.wmax), np.uint8), stc.page_table)
     pk = B.PackBuffers.alloc(ctx, DEV)
