@@ -236,6 +236,55 @@ def run_dry(args):
         dist.destroy_process_group()
 
 
+def run_fp8_only(args):
+    """`--only attn_fp8`: fb_wavefront_attn_fp8 alone on the workload's structure (8-bit pools of
+    N(0,1) values quantised on the device, window scattered once), for profiler captures."""
+    import torch
+    from paper_2607_17652_b200 import binding as B, synth
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    wl = pick_workload(args)
+    stc = synth.make_structure(wl, synth.BASE_SEED + wl.index)
+    tokens = synth.make_tokens(stc)
+    ctx = B.Context(kv_fp8=1, **synth.config_dict(stc, window_in_pages=1))
+    st = B.DeviceState.from_numpy(dev, stc.active, stc.prefix_len, stc.L, stc.R, tokens,
+                                  np.zeros((wl.n_requests, wl.wmax), np.uint8), stc.page_table)
+    pk = B.PackBuffers.alloc(ctx, dev)
+    sb = B.StepBuffers(ctx, dev)
+    gen = torch.Generator(device=dev); gen.manual_seed(stc.seed)
+    rows = ctx.max_slots * wl.block_len
+    q = torch.randn(rows, wl.n_q_heads, wl.head_dim, device=dev, generator=gen).to(torch.bfloat16)
+    kw = torch.randn(rows, wl.n_kv_heads, wl.head_dim, device=dev, generator=gen).to(torch.bfloat16)
+    vw = torch.randn(rows, wl.n_kv_heads, wl.head_dim, device=dev, generator=gen).to(torch.bfloat16)
+    ks = torch.full((wl.n_kv_heads,), 6.0 / 448.0, device=dev)
+    vs = ks.clone()
+    shape = (stc.num_pages, wl.n_kv_heads, wl.page_size, wl.head_dim)
+    pools = []
+    for _ in range(2):
+        pool = torch.empty(shape, dtype=torch.uint8, device=dev)
+        for p0 in range(0, shape[0], 2048):
+            x = torch.randn(pool[p0:p0 + 2048].shape, device=dev, generator=gen) / ks[None, :, None, None]
+            pool[p0:p0 + 2048] = x.clamp_(-448.0, 448.0).to(torch.float8_e4m3fn).view(torch.uint8)
+        pools.append(pool)
+    k8, v8 = pools
+    B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+    B.fb_scatter_window_kv_fp8(ctx, pk, st.page_table, kw, vw, k8, v8, ks, vs, sb.status)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for i in range(args.warmup + args.steps):
+        e = ev[i - args.warmup] if i >= args.warmup else None
+        if e: e[0].record()
+        B.fb_wavefront_attn_fp8(ctx, pk, q, k8, v8, ks, vs, st.page_table, sb.out, sb.ws, sb.status)
+        if e: e[1].record()
+    torch.cuda.synchronize()
+    ms = float(np.mean([a.elapsed_time(b) for a, b in ev]))
+    peaks = load_peaks()
+    tf = attn_flops(stc) / ms / 1e9
+    print(json.dumps({"metric": METRIC, "only": "attn_fp8", "config": {"workload": wl.name, "requests": wl.n_requests},
+                      "kernels": {"attn_ms": round(ms, 4), "attn_tflops": round(tf, 2)},
+                      "frac_of_fp8_peak": round(tf / (2.0 * peaks["bf16_tflops"]), 4),
+                      "device_status": int(sb.status.item())}), flush=True)
+
+
 # ---------------------------------------------------------------- our arm
 def run_ours(args):
     import torch
@@ -775,7 +824,7 @@ def main():
                     help="launcher / reduction plumbing only: gloo ranks on CPU, no kernel, placeholder times")
     ap.add_argument("--requests", type=int, default=0,
                     help="override the workload's request count (small cases for profiler captures)")
-    ap.add_argument("--only", default="all", choices=["all", "attn", "t2t"],
+    ap.add_argument("--only", default="all", choices=["all", "attn", "t2t", "attn_fp8"],
                     help="time one call only (profiler captures); the JSON line then has no step metric")
     ap.add_argument("--cpu-budget", type=float, default=12.0)
     ap.add_argument("--ref-requests", type=int, default=2)
@@ -800,6 +849,8 @@ def main():
         run_reference(args)
     elif args.dry_run_cpu:
         run_dry(args)
+    elif args.only == "attn_fp8":
+        run_fp8_only(args)
     elif args.sweep:
         run_sweep(args)
     else:
