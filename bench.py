@@ -397,40 +397,42 @@ def run_ours(args):
                                      "gbs": round(sc_bytes / sc_ms / 1e6, 1)},
                "attn_window_in_pages": {"ms": round(ra_ms, 4),
                                         "tflops": round(attn_flops(device_structure()) / ra_ms / 1e9, 2)}}
-        # next row: the KV pages in 8 bits (FP8 E4M3, per-KV-head scales): scatter = quantiser, attention
-        # with both products as 8-bit MMAs.  Pools of N(0,1) values quantised on the device.
-        gen8 = torch.Generator(device=dev); gen8.manual_seed(seed + 78)
-        ks8 = torch.full((wl.n_kv_heads,), 6.0 / 448.0, device=dev) * (0.5 + 1.5 * torch.rand(wl.n_kv_heads, device=dev, generator=gen8))
-        vs8 = torch.full((wl.n_kv_heads,), 6.0 / 448.0, device=dev) * (0.5 + 1.5 * torch.rand(wl.n_kv_heads, device=dev, generator=gen8))
-        kp8 = torch.empty(kp.shape, dtype=torch.uint8, device=dev)
-        vp8 = torch.empty(vp.shape, dtype=torch.uint8, device=dev)
-        for pool, sc in ((kp8, ks8), (vp8, vs8)):
-            for p0 in range(0, pool.shape[0], 2048):
-                x = torch.randn(pool[p0:p0 + 2048].shape, device=dev, generator=gen8) / sc[None, :, None, None]
-                pool[p0:p0 + 2048] = x.clamp_(-448.0, 448.0).to(torch.float8_e4m3fn).view(torch.uint8)
-        ctx8 = B.Context(kv_fp8=1, **synth.config_dict(stc, window_in_pages=1))
-        pk8 = B.PackBuffers.alloc(ctx8, dev)
-        ws8 = B.alloc_workspace(ctx8, dev)
-        ev8 = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n2)]
-        for k in range(3 + n2):
-            B.fb_pack_wavefronts(ctx8, st, pk8, ws8, sb.status, stream)
-            e = ev8[k - 3] if k >= 3 else None
-            if e: e[0].record(stream)
-            B.fb_scatter_window_kv_fp8(ctx8, pk8, st.page_table, kw, vw, kp8, vp8, ks8, vs8, sb.status, 10000.0, stream)
-            if e: e[1].record(stream)
-            B.fb_wavefront_attn_fp8(ctx8, pk8, q, kp8, vp8, ks8, vs8, st.page_table, sb.out, ws8, sb.status, stream)
-            if e: e[2].record(stream)
-        barrier()
-        s8_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in ev8]))
-        a8_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in ev8]))
-        cur = device_structure()
-        kv_tokens = sum(int(cur.prefix_len[r]) + int(cur.R[r] - cur.L[r]) * wl.block_len
-                        for r in range(wl.n_requests) if cur.active[r] == 1)
-        a8_bytes = 2.0 * kv_tokens * wl.n_kv_heads * wl.head_dim + 2.0 * 2 * live_now * wl.block_len * wl.n_q_heads * wl.head_dim
-        nxt["attn_fp8_pages"] = {"ms": round(a8_ms, 4), "tflops": round(attn_flops(cur) / a8_ms / 1e9, 2),
-                                 "algorithmic_bytes": a8_bytes, "scatter_quantise_ms": round(s8_ms, 4),
-                                 "speedup_vs_bf16_pages": round(ra_ms / a8_ms, 3)}
-        del ctx2, pk2, ws2, ctx8, pk8, ws8, kp8, vp8
+        if wl.head_dim == 128:
+            # next row: the KV pages in 8 bits (FP8 E4M3, per-KV-head scales): scatter = quantiser, attention
+            # with both products as 8-bit MMAs.  Pools of N(0,1) values quantised on the device.
+            gen8 = torch.Generator(device=dev); gen8.manual_seed(seed + 78)
+            ks8 = torch.full((wl.n_kv_heads,), 6.0 / 448.0, device=dev) * (0.5 + 1.5 * torch.rand(wl.n_kv_heads, device=dev, generator=gen8))
+            vs8 = torch.full((wl.n_kv_heads,), 6.0 / 448.0, device=dev) * (0.5 + 1.5 * torch.rand(wl.n_kv_heads, device=dev, generator=gen8))
+            kp8 = torch.empty(kp.shape, dtype=torch.uint8, device=dev)
+            vp8 = torch.empty(vp.shape, dtype=torch.uint8, device=dev)
+            for pool, sc in ((kp8, ks8), (vp8, vs8)):
+                for p0 in range(0, pool.shape[0], 2048):
+                    x = torch.randn(pool[p0:p0 + 2048].shape, device=dev, generator=gen8) / sc[None, :, None, None]
+                    pool[p0:p0 + 2048] = x.clamp_(-448.0, 448.0).to(torch.float8_e4m3fn).view(torch.uint8)
+            ctx8 = B.Context(kv_fp8=1, **synth.config_dict(stc, window_in_pages=1))
+            pk8 = B.PackBuffers.alloc(ctx8, dev)
+            ws8 = B.alloc_workspace(ctx8, dev)
+            ev8 = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n2)]
+            for k in range(3 + n2):
+                B.fb_pack_wavefronts(ctx8, st, pk8, ws8, sb.status, stream)
+                e = ev8[k - 3] if k >= 3 else None
+                if e: e[0].record(stream)
+                B.fb_scatter_window_kv_fp8(ctx8, pk8, st.page_table, kw, vw, kp8, vp8, ks8, vs8, sb.status, 10000.0, stream)
+                if e: e[1].record(stream)
+                B.fb_wavefront_attn_fp8(ctx8, pk8, q, kp8, vp8, ks8, vs8, st.page_table, sb.out, ws8, sb.status, stream)
+                if e: e[2].record(stream)
+            barrier()
+            s8_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in ev8]))
+            a8_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in ev8]))
+            cur = device_structure()
+            kv_tokens = sum(int(cur.prefix_len[r]) + int(cur.R[r] - cur.L[r]) * wl.block_len
+                            for r in range(wl.n_requests) if cur.active[r] == 1)
+            a8_bytes = 2.0 * kv_tokens * wl.n_kv_heads * wl.head_dim + 2.0 * 2 * live_now * wl.block_len * wl.n_q_heads * wl.head_dim
+            nxt["attn_fp8_pages"] = {"ms": round(a8_ms, 4), "tflops": round(attn_flops(cur) / a8_ms / 1e9, 2),
+                                     "algorithmic_bytes": a8_bytes, "scatter_quantise_ms": round(s8_ms, 4),
+                                     "speedup_vs_bf16_pages": round(ra_ms / a8_ms, 3)}
+            del ctx8, pk8, ws8, kp8, vp8
+        del ctx2, pk2, ws2
         # next row: the row pass fused into the LM head GEMM (hidden size of a small dLLM; random inputs)
         hidden = 2048
         gen = torch.Generator(device=dev); gen.manual_seed(seed + 77)
@@ -561,10 +563,11 @@ def run_ours(args):
         if nxt:
             nxt["lm_head_t2t"]["frac_of_measured_bf16"] = round(nxt["lm_head_t2t"]["tflops"] / peaks["bf16_tflops"], 4)
             nxt["scatter_window_kv"]["frac_of_measured_hbm"] = round(nxt["scatter_window_kv"]["gbs"] / peaks["hbm_gbs"], 4)
-            f8 = nxt["attn_fp8_pages"]
+            f8 = nxt.get("attn_fp8_pages", {})
             f8["peak_fp8_tflops"] = round(2.0 * peaks["bf16_tflops"], 1)      # measured bf16 burst x the nominal fp8 : bf16 ratio (4.5 : 2.25)
-            f8["frac_of_fp8_peak"] = round(f8["tflops"] / f8["peak_fp8_tflops"], 4)
-            f8["hbm_floor_ms"] = round(f8["algorithmic_bytes"] / peaks["hbm_gbs"] / 1e6, 4)
+            if "tflops" in f8:
+                f8["frac_of_fp8_peak"] = round(f8["tflops"] / f8["peak_fp8_tflops"], 4)
+                f8["hbm_floor_ms"] = round(f8["algorithmic_bytes"] / peaks["hbm_gbs"] / 1e6, 4)
             line["next_rows"] = nxt
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(wl, stc_init, tokens, z_live, attn, budget_s=args.cpu_budget)
