@@ -235,3 +235,72 @@ def test_contexts_that_cannot_hold_8_bit_pages_are_refused():
         with pytest.raises(B.FlowBlockError) as e:
             B.fb_wavefront_attn_fp8(ctx, pk, d, d, d, d, d, d, d, d, d)
         assert e.value.code == B.FB_ERR_UNSUPPORTED
+
+
+def test_multi_step_trajectory_with_8_bit_pages():
+    """Eight consecutive steps with the pages in 8 bits: pack -> scatter (the
+    quantiser, Eq. 6 every step) -> attention over the pages -> T2T ->
+    gate/commit as a pointer bump.  After every step the pools must hold exactly
+    the oracle's bytes (so the K/V of every block that retires is frozen as it
+    was quantised in its last step, and nothing else moves), the state and the
+    decisions must be bit-exact, the attention within the derived bound."""
+    wl = synth.tiny_workload(head_dim=128, n_q_heads=8, n_kv_heads=2, n_requests=5, wmax=3, w_lo=1, w_hi=2,
+                             prefix_lo=40, prefix_hi=400, max_blocks=10)
+    stc = synth.make_structure(wl, n_inactive=2)
+    late = [int(r) for r in np.flatnonzero(stc.active == 0)]
+    tokens = synth.make_tokens(stc)
+    ctx = B.Context(kv_fp8=1, **H.common_cfg(stc, window_in_pages=1, s_pe=1))
+    st = B.DeviceState.from_numpy(DEV, stc.active, stc.prefix_len, stc.L, stc.R, tokens,
+                                  np.zeros((wl.n_requests, wl.wmax), np.uint8), stc.page_table)
+    pk = B.PackBuffers.alloc(ctx, DEV)
+    sb = B.StepBuffers(ctx, DEV)
+    ocfg = H.oracle_cfg(stc, s_pe=1)
+    ost = H.oracle_state(stc, tokens)
+    q, kw, vw, _, _ = synth.make_attn_inputs(stc)
+    k8, v8, ks, vs = synth.make_fp8_kv(stc)
+    ok8, ov8 = k8.numpy().copy(), v8.numpy().copy()
+    dk8, dv8, dks, dvs = k8.to(DEV), v8.to(DEV), ks.to(DEV), vs.to(DEV)
+    total_commits = 0
+    for step in range(8):
+        if step in (2, 4):
+            r = late[step // 2 - 1]
+            ost.active[r] = 1
+            st.active[r] = 1
+        cur = dataclasses.replace(stc)
+        cur.active, cur.prefix_len, cur.L, cur.R = (ost.active.copy(), ost.prefix_len.copy(),
+                                                   ost.L.copy(), ost.R.copy())
+        z, tok2 = synth.make_logits(cur, ost.tokens, "calibrated", seed_shift=step, conf_shift=0.05 * step)
+        ost.tokens[:] = tok2
+        st.tokens.copy_(torch.from_numpy(tok2))
+        q = synth.randn_bf16(q.shape, stc.seed + step, 1)
+        kw = synth.randn_bf16(kw.shape, stc.seed + step, 2)
+        vw = synth.randn_bf16(vw.shape, stc.seed + step, 3)
+        B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+        B.fb_scatter_window_kv_fp8(ctx, pk, st.page_table, kw.to(DEV), vw.to(DEV), dk8, dv8, dks, dvs, sb.status)
+        B.fb_wavefront_attn_fp8(ctx, pk, q.to(DEV), dk8, dv8, dks, dvs, st.page_table, sb.out, sb.ws, sb.status)
+        B.fb_t2t_step(ctx, pk, z.to(DEV), st, sb.argmax, sb.conf, sb.action, sb.slot_stats, sb.status)
+        B.fb_gate_commit(ctx, pk, sb.slot_stats, st, None, None, None, None, sb.n_committed, sb.spawned,
+                         sb.step_counters, sb.status)
+        torch.cuda.synchronize()
+        assert int(sb.status.item()) == 0
+        opk = O.pack_wavefronts(ocfg, ost)
+        O.scatter_window_kv_fp8(ocfg, opk, H.f64(kw), H.f64(vw), ok8, ov8, ks.numpy(), vs.numpy(), ost.page_table)
+        ref = O.wavefront_attn_fp8(ocfg, opk, H.f64(q), ok8, ov8, ks.numpy(), vs.numpy(), ost.page_table)
+        rows = H.live_rows(opk, wl.block_len)
+        g_out = sb.out.float().cpu().numpy().astype(np.float64)[rows]
+        rel = float(np.linalg.norm(g_out - ref[rows]) / np.linalg.norm(ref[rows]))
+        assert rel <= F8_REL_L2, (step, rel)
+        xhat, conf = O.t2t_rows(ocfg, opk, H.f64(z))
+        action, stats = O.t2t_update(ocfg, opk, ost, xhat, conf)
+        ncom, spawned, ctr = O.gate_commit(ocfg, opk, stats, ost)          # window in the pages: nothing to copy
+        np.testing.assert_array_equal(sb.action.cpu().numpy(), action)
+        np.testing.assert_array_equal(sb.n_committed.cpu().numpy(), ncom)
+        np.testing.assert_array_equal(sb.spawned.cpu().numpy(), spawned)
+        np.testing.assert_array_equal(sb.step_counters.cpu().numpy(), ctr)
+        g = st.to_numpy()
+        for name in ("active", "prefix_len", "L", "R", "tokens", "pe_done"):
+            np.testing.assert_array_equal(g[name], getattr(ost, name), err_msg=f"{name}@{step}")
+        np.testing.assert_array_equal(dk8.cpu().numpy(), ok8, err_msg=f"K bytes@{step}")
+        np.testing.assert_array_equal(dv8.cpu().numpy(), ov8, err_msg=f"V bytes@{step}")
+        total_commits += int(ncom.sum())
+    assert total_commits >= 3, "the trajectory never committed a block"
