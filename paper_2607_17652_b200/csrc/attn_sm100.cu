@@ -670,11 +670,11 @@ wavefront_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
 }
 
 // Merge of the split-KV partials, chunks in index order.  A unit is cut into
-// eight pieces of 32 of its 256 rows; the CTAs of a fixed-size grid loop over
+// 32 pieces of 8 of its 256 rows; the CTAs of a fixed-size grid loop over
 // the pieces (nothing to do, and an immediate return, when no unit was split).
 // A warp takes one row at a time and keeps the loads of four chunks in flight.
-constexpr int kCombineSplit = 8;
-constexpr int kCombineCtasPerSm = 4;
+constexpr int kCombineSplit = 32;        // pieces of 8 rows: one row per warp, no serial row loop
+constexpr int kCombineCtasPerSm = 8;
 template <int D>
 __global__ void __launch_bounds__(256) attn_combine_kernel(const AttnParams p) {
   pdl_wait();

@@ -346,7 +346,9 @@ int launch_pack(fb_ctx* ctx, const fb_state* st, const fb_pack* out, void* ws, i
   p.min_chunk_tiles = ctx->min_chunk_tiles;
   p.resident = ctx->cfg.window_in_pages;
   p.n_gather_blocks = (p.max_slots + kSlotsPerBlock - 1) / kSlotsPerBlock;
-  return cuda_err(ctx, launch_pdl(pack_kernel, p.n_gather_blocks + 2, kPackThreads, 0, stream, p), "pack_kernel launch");
+  // one more block per work list in use (the CTA-pair kernel's list only when that kernel is on)
+  return cuda_err(ctx, launch_pdl(pack_kernel, p.n_gather_blocks + 1 + (p.pair_on ? 1 : 0), kPackThreads, 0, stream, p),
+                  "pack_kernel launch");
 }
 
 }  // namespace fb
