@@ -456,6 +456,39 @@ def run_ours(args):
                               "logits_bytes_not_moved": 2.0 * live_now * wl.block_len * wl.vocab * 2}
         del hx, hw, lws
 
+    # ------------- the same step replayed from a CUDA graph (one graph launch instead of seven launches)
+    if only == "all" and world == 1 and not args.no_graph:
+        def step_current():
+            B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
+            B.fb_wavefront_attn(ctx, pk, q, kw, vw, kp, vp, st.page_table, sb.out, sb.ws, sb.status)
+            B.fb_t2t_step(ctx, pk, logits, st, sb.argmax, sb.conf, sb.action, sb.slot_stats, sb.status)
+            B.fb_gate_commit(ctx, pk, sb.slot_stats, st, kw, vw, kp, vp, sb.n_committed, sb.spawned,
+                             sb.step_counters, sb.status)
+        graph = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            step_current()                       # per-device set-up already happened: nothing but launches
+            side.synchronize()
+            with torch.cuda.graph(graph, stream=side):
+                step_current()
+        stream.wait_stream(side)
+        ng = max(3, min(args.steps, 20))
+        evg = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(ng)]
+        for k in range(3 + ng):
+            if flush is not None:
+                flush.fill_(k & 0xFF)
+            e = evg[k - 3] if k >= 3 else None
+            if e: e[0].record(stream)
+            graph.replay()
+            if e: e[1].record(stream)
+        barrier()
+        g_ms = [a.elapsed_time(b) for a, b in evg]
+        nxt["step_graph_replay"] = {"ms_per_step": round(float(np.mean(g_ms)), 4), "ms_per_step_min": round(float(np.min(g_ms)), 4),
+                                    "direct_launch_ms_per_step": round(float(per_step.mean()), 4), "timed_steps": ng,
+                                    "device_status": int(sb.status.item())}
+        del graph
+
     # ------------- a step that commits: calibrated confidences, state reset before every timed step
     if only == "all" and world == 1 and not args.no_calibrated:
         nxt["step_calibrated"] = calibrated_step(args, wl, stc_init, dev, stream, q, kw, vw, kp, vp, logits, sb)
@@ -821,6 +854,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-calibrated", action="store_true", help="skip next_rows.step_calibrated")
+    ap.add_argument("--no-graph", action="store_true", help="skip next_rows.step_graph_replay")
     ap.add_argument("--pair", action="store_true",
                     help="quads of Q tiles on the CTA-pair attention kernel (fb_tuning.attn_pair): the comparison run")
     ap.add_argument("--dry-run-cpu", action="store_true",
