@@ -301,7 +301,8 @@ def run_ours(args):
     seed = synth.BASE_SEED + wl.index + 1000 * rank     # each rank its own batch
     stc, tokens, n_live, z_live, attn = build_inputs(wl, seed)
     stc_init = stc
-    ctx = B.Context(tuning=dict(attn_pair=1) if args.pair else None, **synth.config_dict(stc))
+    tuning = dict(attn_pair=int(args.pair), attn_target_items=args.target_items, attn_min_chunk_tiles=args.min_chunk)
+    ctx = B.Context(tuning=tuning if any(tuning.values()) else None, **synth.config_dict(stc))
     st = B.DeviceState.from_numpy(dev, stc.active, stc.prefix_len, stc.L, stc.R, tokens,
                                   np.zeros((wl.n_requests, wl.wmax), np.uint8), stc.page_table)
     pk = B.PackBuffers.alloc(ctx, dev)
@@ -855,6 +856,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-calibrated", action="store_true", help="skip next_rows.step_calibrated")
     ap.add_argument("--no-graph", action="store_true", help="skip next_rows.step_graph_replay")
+    ap.add_argument("--target-items", type=int, default=0, help="fb_tuning.attn_target_items (0: default)")
+    ap.add_argument("--min-chunk", type=int, default=0, help="fb_tuning.attn_min_chunk_tiles (0: default)")
     ap.add_argument("--pair", action="store_true",
                     help="quads of Q tiles on the CTA-pair attention kernel (fb_tuning.attn_pair): the comparison run")
     ap.add_argument("--dry-run-cpu", action="store_true",
