@@ -16,7 +16,7 @@
 //               (3-stage rings); in the first CTA it also draws the work items
 //               and publishes them to both CTAs
 //   warp 1      first CTA only: issues every MMA of the pair and the commits,
-//               which arrive on the barriers of both CTAs
+//               which arrive on the barriers of both CTAs (one commit per CTA)
 //   warps 4-7   softmax + epilogue of this CTA's tile A, 8-11 of its tile B
 //               (one thread per query row; as in the one-CTA kernel)
 // Streams: A = (tile A of CTA 0, tile A of CTA 1), B likewise; the MMA warp
@@ -276,7 +276,7 @@ wavefront_attn_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid
           const uint32_t boff = ((ks >> 2) * 8192 + (ks & 3) * 32) >> 4;      // K: 64 rows per half of d
           umma_ss_pair(d, qa + aoff, kb + boff, idesc_qk, ks > 0 ? 1u : 0u);
         }
-        umma_commit_pair(&s_full[X], 3);
+        umma_commit_pair(&s_full[X], true);
       }
       __syncwarp();
     };
@@ -291,7 +291,7 @@ wavefront_attn_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid
       }
       __syncwarp();
     };
-    auto commit = [&](uint64_t* bar) { if (leader) umma_commit_pair(bar, 3); __syncwarp(); };
+    auto commit = [&](uint64_t* bar) { if (leader) umma_commit_pair(bar, true); __syncwarp(); };
     for (int k = 0; ok; ++k) {
       if (!warp_wait(&item_full[k & 1], (k >> 1) & 1, abortf, LIM)) { ok = false; break; }
       const int idx = s_item[k & 1];
@@ -535,7 +535,7 @@ wavefront_attn_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid
     // tensor memory goes back, copies in flight land while the CTA sleeps
     if (tid == 0) atomicOr(p.status, FB_ST_DEV_TIMEOUT);
     if (warp == 1 && first) {
-      if (elect_one()) umma_commit_pair(drain, 1);
+      if (elect_one()) umma_commit_pair(drain, false);
       __syncwarp();
       for (int i = 0; i < 4096 && !mbar_test(drain, 0); ++i) __nanosleep(200);
     }

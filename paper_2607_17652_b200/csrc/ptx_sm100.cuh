@@ -303,13 +303,17 @@ __device__ __forceinline__ void umma_ts_pair(uint32_t d_tmem, uint32_t a_tmem, u
       "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// everything issued so far -> one arrival on the barrier at this offset in each CTA of `mask`
-__device__ __forceinline__ void umma_commit_pair(uint64_t* bar, uint16_t mask) {
-  asm volatile(
-      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
-          smem_u32(bar)),
-      "h"(mask)
-      : "memory");
+// everything this thread has issued so far (MMAs over both CTAs) -> one arrival on a barrier given
+// by its shared::cluster address, i.e. of either CTA of the pair
+__device__ __forceinline__ void umma_commit_pair_addr(uint32_t bar_cluster) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_cluster)
+               : "memory");
+}
+// ... on the barrier at this offset in this CTA (`both` = false) or in both CTAs of the pair:
+// two commits, one per CTA, each an arrival of its own
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar, bool both) {
+  umma_commit_pair_addr(mapa_u32(bar, 0));
+  if (both) umma_commit_pair_addr(mapa_u32(bar, 1));
 }
 
 // Shared-memory matrix descriptor for a 128-byte-swizzled operand tile whose
