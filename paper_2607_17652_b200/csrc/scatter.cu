@@ -5,12 +5,14 @@
 // (all KV heads), optionally with the rotary embedding applied to the keys.
 // HBM-bound: 2 x rows x Hkv x d x 2 bytes read and as many written.
 //
-// One to four CTAs per slot (the KV heads are dealt among them).  For a (token, head) the head_dim elements are contiguous
+// One to four CTAs per slot (the slot's tokens are dealt among them).  For a (token, head) the head_dim elements are contiguous
 // in the source (slot-order rows) and in the destination (pool row of that
 // position), so a thread moves 16-byte pieces: with the rotary embedding a
 // thread owns the two pieces that hold elements i and i + d/2 of eight pairs,
 // and the rotation angles come from a per-slot table in shared memory.
 #include <cuda_fp8.h>
+
+#include <cmath>
 
 #include "fb_common.cuh"
 
@@ -27,6 +29,7 @@ struct ScatterParams {
   int32_t bl, n_kv_heads, head_dim, max_pages_per_req, num_pages;
   float rope_base;
   const float *k_scale, *v_scale;   // 8-bit pages: [n_kv_heads]
+  double inv_freq[64];              // rope_base^(-2k/d), k < d/2 (formed on the host in fp64)
 };
 
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
@@ -53,6 +56,7 @@ __device__ __forceinline__ uint2 quant8(const uint4 v, float scale) {
 // the scale of its KV head before it is rounded.
 template <bool F8>
 __global__ void __launch_bounds__(kScatterThreads) scatter_window_kv_kernel(const ScatterParams p) {
+  pdl_wait();
   const int slot = blockIdx.x;
   if (slot >= *p.n_live) return;
   const int r = p.slot_req[slot], pos0 = p.slot_pos0[slot];
@@ -65,20 +69,21 @@ __global__ void __launch_bounds__(kScatterThreads) scatter_window_kv_kernel(cons
   constexpr int kTokBatch = 32;
   __shared__ float2 cs[kTokBatch * 64];              // [token of the batch][pair] (cos, sin), d/2 <= 64
   const int half = p.head_dim / 2;
-  __shared__ double inv_freq[64];                    // base^(-2k/d)
-  if (rope && threadIdx.x < half)
-    inv_freq[threadIdx.x] = exp2(-2.0 * (double)threadIdx.x / (double)p.head_dim * log2((double)p.rope_base));
   // work item = (token, head, piece); with the rotary embedding only the lower half of the
   // pieces is enumerated and each item also handles its partner piece + d/16
   const int per_head = rope ? vph / 2 : vph;
-  for (int t0 = 0; t0 < p.bl; t0 += kTokBatch) {
-  const int nt = min(kTokBatch, p.bl - t0);
+  // the slot's tokens are dealt to the gridDim.y CTAs of the slot (each builds the table of its
+  // own tokens only)
+  const int tpc = (p.bl + (int)gridDim.y - 1) / (int)gridDim.y;
+  const int tbeg = (int)blockIdx.y * tpc, tend = min(p.bl, tbeg + tpc);
+  for (int t0 = tbeg; t0 < tend; t0 += kTokBatch) {
+  const int nt = min(kTokBatch, tend - t0);
   if (rope) {
     __syncthreads();                                 // the previous batch has been read
     for (int i = threadIdx.x; i < nt * half; i += kScatterThreads) {
       const int t = i / half, k = i % half;
       // angle in fp64, reduced to [-pi, pi] there; sine and cosine of the remainder in fp32
-      const double ang = (double)(pos0 + t0 + t) * inv_freq[k];
+      const double ang = (double)(pos0 + t0 + t) * p.inv_freq[k];
       const double red = fma(-rint(ang * 0.15915494309189535), 6.283185307179586, ang);
       float sf, cf;
       sincosf((float)red, &sf, &cf);
@@ -86,13 +91,12 @@ __global__ void __launch_bounds__(kScatterThreads) scatter_window_kv_kernel(cons
     }
     __syncthreads();
   }
-  // the KV heads are dealt to the gridDim.y CTAs of the slot
-  const int nh = (p.n_kv_heads - (int)blockIdx.y + (int)gridDim.y - 1) / (int)gridDim.y;
+  const int nh = p.n_kv_heads;
   const int total = nt * nh * per_head;
   for (int i = threadIdx.x; i < total; i += kScatterThreads) {
     const int tb = i / (nh * per_head), rem = i % (nh * per_head);
     const int t = t0 + tb;
-    const int h = (rem / per_head) * gridDim.y + blockIdx.y, v = rem % per_head;
+    const int h = rem / per_head, v = rem % per_head;
     const int pos = pos0 + t, pidx = pos / kPage;
     if (pidx >= p.max_pages_per_req) { atomicOr(p.status, FB_ST_BAD_PAGE); continue; }
     const int page = p.page_table[(size_t)r * p.max_pages_per_req + pidx];
@@ -150,6 +154,15 @@ __global__ void __launch_bounds__(kScatterThreads) scatter_window_kv_kernel(cons
   }
 }
 
+static void fill_inv_freq(ScatterParams& p, int head_dim, float rope_base) {
+  for (int k = 0; k < 64; ++k)
+    p.inv_freq[k] = (rope_base > 0.f && k < head_dim / 2)
+                        ? exp2(-2.0 * (double)k / (double)head_dim * log2((double)rope_base)) : 0.0;
+}
+// enough (token, head, piece) items per CTA to keep 256 threads busy: four CTAs per slot once a
+// slot holds 32 tokens of at least four KV heads
+static int scatter_ctas_per_slot(const fb_config& c) { return c.block_len >= 32 && c.n_kv_heads >= 4 ? 4 : 1; }
+
 int launch_scatter(fb_ctx* ctx, const fb_pack* pk, const int32_t* page_table, const void* k_new,
                    const void* v_new, void* k_pool, void* v_pool, float rope_base, int32_t* status,
                    cudaStream_t stream) {
@@ -164,9 +177,10 @@ int launch_scatter(fb_ctx* ctx, const fb_pack* pk, const int32_t* page_table, co
   p.max_pages_per_req = c.max_pages_per_req; p.num_pages = c.num_pages;
   p.rope_base = rope_base;
   p.k_scale = p.v_scale = nullptr;
-  const dim3 grid(c.max_requests * c.wmax, c.n_kv_heads >= 4 ? 4 : 1);
-  scatter_window_kv_kernel<false><<<grid, kScatterThreads, 0, stream>>>(p);
-  return cuda_err(ctx, cudaGetLastError(), "scatter_window_kv_kernel launch");
+  fill_inv_freq(p, c.head_dim, rope_base);
+  const dim3 grid(c.max_requests * c.wmax, scatter_ctas_per_slot(c));
+  return cuda_err(ctx, launch_pdl(scatter_window_kv_kernel<false>, grid, kScatterThreads, 0, stream, p),
+                  "scatter_window_kv_kernel launch");
 }
 
 int launch_scatter_fp8(fb_ctx* ctx, const fb_pack* pk, const int32_t* page_table, const void* k_new,
@@ -183,9 +197,10 @@ int launch_scatter_fp8(fb_ctx* ctx, const fb_pack* pk, const int32_t* page_table
   p.max_pages_per_req = c.max_pages_per_req; p.num_pages = c.num_pages;
   p.rope_base = rope_base;
   p.k_scale = k_scale; p.v_scale = v_scale;
-  const dim3 grid(c.max_requests * c.wmax, c.n_kv_heads >= 4 ? 4 : 1);
-  scatter_window_kv_kernel<true><<<grid, kScatterThreads, 0, stream>>>(p);
-  return cuda_err(ctx, cudaGetLastError(), "scatter_window_kv_kernel (8-bit pages) launch");
+  fill_inv_freq(p, c.head_dim, rope_base);
+  const dim3 grid(c.max_requests * c.wmax, scatter_ctas_per_slot(c));
+  return cuda_err(ctx, launch_pdl(scatter_window_kv_kernel<true>, grid, kScatterThreads, 0, stream, p),
+                  "scatter_window_kv_kernel (8-bit pages) launch");
 }
 
 // fb_embed_gather: x[i, :] = table[qtok[i], :] for live rows; one warp per row, 16-byte pieces.
