@@ -691,7 +691,8 @@ def run_sweep(args):
     n_steps = args.steps if args.steps != 20 else 48
     rise = tuple(float(x) for x in args.rise_range.split(",")) if args.rise_range else None
     inp = sweep.SweepInputs(wl, n_steps=n_steps, arrive_hi=1 if args.static_batch else 24, rise_range=rise)
-    run = sweep.SweepRunner(inp, dev, window_in_pages=args.window_in_pages, batch_sync=args.batch_sync)
+    run = sweep.SweepRunner(inp, dev, window_in_pages=args.window_in_pages, batch_sync=args.batch_sync,
+                            kv_fp8=args.kv_fp8)
 
     def one_pass(timed):
         seg, flops, live, committed = [], [], [], 0
@@ -733,8 +734,10 @@ def run_sweep(args):
         "metric": METRIC, "value": round(float(flops.sum()) / total_ms / 1e9, 3),
         "unit": "TFLOP/s (attention FLOPs / whole-step time)",
         "n_gpus": 1, "steps": n_steps, "warmup": n_steps, "ms_per_step": round(total_ms / n_steps, 4),
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": wl.name + (" (sweep, window in pages)" if args.window_in_pages else " (sweep)"), "requests": wl.n_requests, "block_len": wl.block_len,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "fp8 e4m3 (K/V pages, Q, P; fp32 accumulation)" if args.kv_fp8 else "bf16", "data": "synthetic",
+        "config": {"workload": wl.name + (" (sweep, FP8 E4M3 pages)" if args.kv_fp8 else
+                                          " (sweep, window in pages)" if args.window_in_pages else " (sweep)"), "requests": wl.n_requests, "block_len": wl.block_len,
                    "wmax": wl.wmax, "theta_spawn": wl.theta_spawn,
                    "policy": "batch-synchronous wavefront" if args.batch_sync else "per-sequence wavefronts",
                    "arrivals": "all at step 0" if args.static_batch else "uniform over the first 24 steps",
@@ -871,6 +874,8 @@ def main():
     ap.add_argument("--window-in-pages", action="store_true",
                     help="with --sweep: scatter the window K/V into the pages every step (Eq. 6), attention "
                          "over the pages, retirement as a pointer bump")
+    ap.add_argument("--kv-fp8", action="store_true",
+                    help="with --sweep: KV pages in FP8 E4M3 (scatter = quantiser every step, 8-bit attention products)")
     ap.add_argument("--batch-sync", action="store_true",
                     help="with --sweep: the batch-synchronous wavefront of the packing ablation (fb_config.batch_sync)")
     ap.add_argument("--static-batch", action="store_true", help="with --sweep: every request arrives at step 0")

@@ -172,11 +172,15 @@ class SweepRunner:
     and the four calls of a step."""
 
     def __init__(self, inp: SweepInputs, device="cuda:0", window_in_pages: bool = False,
-                 batch_sync: bool = False, **cfg_over):
+                 batch_sync: bool = False, kv_fp8: bool = False, **cfg_over):
+        """``kv_fp8``: the pages hold FP8 E4M3 bytes (implies the window in the pages: the
+        scatter is the quantiser)."""
         self.inp, self.dev = inp, device
-        self.resident = bool(window_in_pages)
+        self.fp8 = bool(kv_fp8)
+        self.resident = bool(window_in_pages) or self.fp8
         stc, wl = inp.stc, inp.wl
-        self.ctx = B.Context(**synth.config_dict(stc, window_in_pages=int(self.resident),
+        self.ctx = B.Context(kv_fp8=int(self.fp8),
+                             **synth.config_dict(stc, window_in_pages=int(self.resident),
                                                  batch_sync=int(bool(batch_sync)), **cfg_over))
         self.st = B.DeviceState.from_numpy(device, stc.active, stc.prefix_len, stc.L, stc.R, inp.tokens0(),
                                            np.zeros((wl.n_requests, wl.wmax), np.uint8), stc.page_table)
@@ -184,6 +188,9 @@ class SweepRunner:
         self.sb = B.StepBuffers(self.ctx, device)
         q, kw, vw, kp, vp = synth.make_attn_inputs(stc)
         self.q, self.kw, self.vw, self.kp, self.vp = (t.to(device) for t in (q, kw, vw, kp, vp))
+        if self.fp8:                     # 8-bit pools of the same N(0,1) values, per-KV-head scales
+            k8, v8, ks, vs = synth.make_fp8_kv(stc)
+            self.kp, self.vp, self.ks, self.vs = (t.to(device) for t in (k8, v8, ks, vs))
         self.z = inp.bank.to(device)
         self.ev = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
         # written before every timed step: keeps the GPU busy while the host enqueues the
@@ -216,7 +223,12 @@ class SweepRunner:
         ev[0].record()
         B.fb_pack_wavefronts(ctx, st, pk, sb.ws, sb.status)
         ev[1].record()
-        if self.resident:      # Eq. 6 every step, attention over the pages
+        if self.fp8:           # Eq. 6 every step into 8-bit pages, attention with 8-bit products
+            B.fb_scatter_window_kv_fp8(ctx, pk, st.page_table, self.kw, self.vw, self.kp, self.vp, self.ks, self.vs,
+                                       sb.status)
+            B.fb_wavefront_attn_fp8(ctx, pk, self.q, self.kp, self.vp, self.ks, self.vs, st.page_table, sb.out,
+                                    sb.ws, sb.status)
+        elif self.resident:    # Eq. 6 every step, attention over the pages
             B.fb_scatter_window_kv(ctx, pk, st.page_table, self.kw, self.vw, self.kp, self.vp, sb.status)
             B.fb_wavefront_attn(ctx, pk, self.q, None, None, self.kp, self.vp, st.page_table, sb.out, sb.ws,
                                 sb.status)
